@@ -1,0 +1,137 @@
+/*
+ * seer.h -- C ABI of the B200 (sm_100a) SeerAttention prefill hot path.
+ *
+ *   seer_gate_scores : Q, K, Wq, Wk        -> block-level gating scores   (Sec. 3.1, Eq. 1)
+ *   seer_block_mask  : scores, TopK | thr  -> per-row sorted KV-block index lists (Sec. 3.3, Eq. 3 / Eq. 4)
+ *   seer_sparse_attn : Q, K, V, lists      -> O, visiting only listed blocks (Sec. 3.3, "Block Sparse Flash-Attn Kernel")
+ *
+ * General rules
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller and must stay valid until the work
+ *    enqueued by the call has completed on `stream`.  `cu_seqlens_host` and the parameter structs are
+ *    HOST memory and are consumed before the call returns.
+ *  - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*; NULL = default stream) and return
+ *    without synchronising.  The library allocates device memory only in seer_create; per-call scratch
+ *    comes from the caller's workspace `ws` (>= seer_workspace_bytes(shape), 256-byte aligned).
+ *  - Nothing throws across the ABI.  Host-detectable errors are returned at once and enqueue nothing.
+ *    Errors only the device can see (list capacity exceeded, a list entry out of range, a bounded wait
+ *    that ran out) are recorded in a status word owned by the context; the offending work is skipped and
+ *    the kernel exits normally.  seer_poll_device_status reads that word.
+ *  - bf16 tensors are passed as const void* / void*; element type is the 16-bit bfloat16 bit pattern.
+ *
+ * Shapes and layouts ("THD", packed variable-length batch)
+ *    T            total tokens of all sequences = cu_seqlens[batch]
+ *    q, o         [T, num_q_heads,  head_dim]   row-major bf16
+ *    k, v         [T, num_kv_heads, head_dim]   row-major bf16
+ *    Wq           [num_q_heads,  head_dim, gate_dim] fp32,  gate input x Wq[h] (row vector times matrix, no bias)
+ *    Wk           [num_kv_heads, head_dim, gate_dim] fp32;  query head h pairs with KV head h / (Hq/Hkv)
+ *    nb_b         ceil(len_b / block) blocks in sequence b
+ *    scores       sequence after sequence, each [num_q_heads][nb_b][nb_b] fp32; entry (h,i,j) is defined for
+ *                 j <= i only, the rest is never written nor read
+ *    mask rows    row id of (b, h, i) = num_q_heads * (blocks of sequences before b) + h * nb_b + i
+ *    row_ptr      int32 [rows + 1], col_idx int32 [nnz]: CSR lists of KV block indices, local to the sequence,
+ *                 ascending, unique, 0 <= j <= i
+ *
+ * Supported: head_dim = 128, gate_dim = 128, block = 64, num_q_heads a multiple of num_kv_heads, batch <= 4096.
+ * Anything else returns SEER_ERR_UNSUPPORTED.
+ */
+#ifndef SEER_H_
+#define SEER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SEER_OK = 0,
+  SEER_ERR_INVALID_ARG = 1,   /* null pointer, negative size, non-monotone cu_seqlens, bad mode */
+  SEER_ERR_UNSUPPORTED = 2,   /* shape outside the supported set (see above), or more than 2^31-1 mask rows / score elements per sequence */
+  SEER_ERR_WORKSPACE = 3,     /* ws too small or misaligned */
+  SEER_ERR_CAPACITY = 4,      /* device: nnz exceeds col_capacity; row_ptr and nnz_out are still complete */
+  SEER_ERR_INVALID_INDEX = 5, /* device: a list entry outside [0, i] */
+  SEER_ERR_TIMEOUT = 6,       /* device: a bounded wait expired */
+  SEER_ERR_CUDA = 7           /* a CUDA runtime / driver call failed (including: no device, no sm_100 device) */
+} seer_status;
+
+typedef struct seer_ctx seer_ctx;
+
+/* Creates a context on CUDA device `device`: queries the SM count, raises the kernels' shared-memory limits,
+ * allocates the device status word and a small metadata buffer.  Not thread-safe per context: use one
+ * context per host thread or serialise calls. */
+seer_status seer_create(seer_ctx** out, int device);
+void seer_destroy(seer_ctx* ctx);
+const char* seer_status_string(seer_status s);
+
+typedef struct {
+  int32_t batch;                  /* number of packed sequences, >= 1 */
+  const int32_t* cu_seqlens_host; /* HOST [batch + 1], cu[0] = 0, non-decreasing; empty sequences are allowed */
+  int32_t num_q_heads;
+  int32_t num_kv_heads;
+  int32_t head_dim;               /* 128 */
+  int32_t block;                  /* 64: gate pooling window = attention tile (Sec. 4: B fixed at 64) */
+  int32_t gate_dim;               /* 128: output width of the gate's linear layers */
+  float softmax_scale;            /* attention logit scale; <= 0 selects 1/sqrt(head_dim) (Sec. 2) */
+} seer_shape;
+
+/* Sizing helpers (pure host arithmetic; return 0 / -1 on an invalid shape). */
+size_t seer_workspace_bytes(const seer_shape* shape); /* enough for any of the three calls */
+size_t seer_scores_elems(const seer_shape* shape);    /* num_q_heads * sum_b nb_b^2 */
+int64_t seer_mask_rows(const seer_shape* shape);      /* num_q_heads * sum_b nb_b   */
+int64_t seer_causal_blocks(const seer_shape* shape);  /* num_q_heads * sum_b nb_b (nb_b + 1) / 2: capacity that always suffices */
+
+/* 1. AttnGate (Sec. 3.1, Eq. 1): score = softmax((Pq(Q) Wq)(Pk(K) Wk)^T / sqrt(gate_dim)).
+ *    Pq, Pk: average pooling over non-overlapping blocks of `block` tokens (a ragged last block averages the
+ *    tokens it has).  The softmax of row i runs over the causal blocks j <= i, so each row sums to 1.
+ *    All gate arithmetic is fp32.  Writes `scores` (layout above). */
+seer_status seer_gate_scores(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k,
+                             const float* Wq, const float* Wk, float* scores, void* ws, size_t ws_bytes,
+                             void* stream);
+
+enum { SEER_TOPK_RATIO = 0, SEER_TOPK_COUNT = 1, SEER_THRESHOLD = 2 };
+enum { SEER_FORCE_DIAG = 1u, SEER_FORCE_SINK = 2u };
+
+typedef struct {
+  int32_t mode;      /* SEER_TOPK_RATIO: keep k_i = clamp(ceil(keep_num * (i+1) / keep_den), 1, i+1) blocks in row i;
+                        SEER_TOPK_COUNT: keep min(k, i+1);  SEER_THRESHOLD: keep score > threshold (strict, fp32) */
+  int32_t keep_num;  /* ratio numerator   (>= 0) */
+  int32_t keep_den;  /* ratio denominator (>= 1) */
+  int32_t k;
+  float threshold;
+  uint32_t flags;    /* SEER_FORCE_DIAG keeps block i, SEER_FORCE_SINK keeps block 0, in every row.  In the TopK modes
+                        forced blocks count toward k_i; the other places go to the best remaining blocks ordered by
+                        (score descending, block index ascending).  NaN scores are never selected. */
+} seer_mask_params;
+
+/* 2. Binary block mask (Sec. 3.3, Eq. 3 TopK / Eq. 4 threshold) as CSR index lists.
+ *    row_ptr [rows+1] and nnz_out (device int64, may be NULL) are always written in full.  col_idx receives the lists
+ *    of the rows that fit entirely below col_capacity; if nnz > col_capacity the device status becomes
+ *    SEER_ERR_CAPACITY and the caller may re-allocate and call again. */
+seer_status seer_block_mask(seer_ctx* ctx, const seer_shape* shape, const float* scores,
+                            const seer_mask_params* params, int32_t* row_ptr, int32_t* col_idx,
+                            int64_t col_capacity, int64_t* nnz_out, void* ws, size_t ws_bytes, void* stream);
+
+/* 3. Causal GQA block-sparse attention (Sec. 3.3): for every query token, softmax(scale * q k^T) v over the keys of the
+ *    blocks listed for its (sequence, head, query block) row that are not later than the query.  bf16 operands, fp32
+ *    accumulation and softmax, probabilities rounded to bf16 before the P V product, o written as bf16.
+ *    lse (optional, may be NULL): [num_q_heads, T] fp32, natural log of the softmax denominator of the scaled logits.
+ *    A row with an empty list yields o = 0 and lse = -inf. */
+seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k, const void* v,
+                             const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, void* ws,
+                             size_t ws_bytes, void* stream);
+
+/* Selects the attention kernel used by seer_sparse_attn: 0 = tcgen05 / TMEM / TMA kernel (default),
+ * 1 = mma.sync kernel kept as an on-device cross-check.  Returns SEER_ERR_INVALID_ARG for other values. */
+seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);
+
+/* Synchronises `stream`, returns the device status word (SEER_OK if nothing was raised) and clears it. */
+seer_status seer_poll_device_status(seer_ctx* ctx, void* stream);
+
+/* Number of kernels the library has launched through this context since creation (for launch accounting). */
+int64_t seer_launch_count(const seer_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEER_H_ */

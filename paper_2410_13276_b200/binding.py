@@ -1,0 +1,207 @@
+"""ctypes binding of the C ABI in include/seer.h: same names, argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device buffers; every step of the
+path runs inside libseer.so.  There is no CPU fallback: if the shared library
+has not been built, or no B200 is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libseer.so")
+
+SEER_OK = 0
+SEER_TOPK_RATIO, SEER_TOPK_COUNT, SEER_THRESHOLD = 0, 1, 2
+SEER_FORCE_DIAG, SEER_FORCE_SINK = 1, 2
+STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER_ERR_WORKSPACE", "SEER_ERR_CAPACITY",
+                "SEER_ERR_INVALID_INDEX", "SEER_ERR_TIMEOUT", "SEER_ERR_CUDA"]
+
+# every symbol include/seer.h declares
+EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
+           "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
+           "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count"]
+
+
+class SeerError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name}")
+
+
+class seer_shape(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("cu_seqlens_host", C.POINTER(C.c_int32)), ("num_q_heads", C.c_int32),
+                ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("block", C.c_int32), ("gate_dim", C.c_int32),
+                ("softmax_scale", C.c_float)]
+
+
+class seer_mask_params(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("keep_num", C.c_int32), ("keep_den", C.c_int32), ("k", C.c_int32),
+                ("threshold", C.c_float), ("flags", C.c_uint32)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads libseer.so (built in-tree by `python -m paper_2410_13276_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_13276_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, sz, i64, i32 = C.c_void_p, C.c_size_t, C.c_int64, C.c_int32
+    shp = C.POINTER(seer_shape)
+    lib.seer_create.argtypes = [C.POINTER(vp), C.c_int]
+    lib.seer_create.restype = C.c_int
+    lib.seer_destroy.argtypes = [vp]
+    lib.seer_destroy.restype = None
+    lib.seer_status_string.argtypes = [C.c_int]
+    lib.seer_status_string.restype = C.c_char_p
+    lib.seer_workspace_bytes.argtypes = [shp]
+    lib.seer_workspace_bytes.restype = sz
+    lib.seer_scores_elems.argtypes = [shp]
+    lib.seer_scores_elems.restype = sz
+    lib.seer_mask_rows.argtypes = [shp]
+    lib.seer_mask_rows.restype = i64
+    lib.seer_causal_blocks.argtypes = [shp]
+    lib.seer_causal_blocks.restype = i64
+    lib.seer_gate_scores.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.seer_gate_scores.restype = C.c_int
+    lib.seer_block_mask.argtypes = [vp, shp, vp, C.POINTER(seer_mask_params), vp, vp, i64, vp, vp, sz, vp]
+    lib.seer_block_mask.restype = C.c_int
+    lib.seer_sparse_attn.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.seer_sparse_attn.restype = C.c_int
+    lib.seer_set_attn_impl.argtypes = [vp, C.c_int]
+    lib.seer_set_attn_impl.restype = C.c_int
+    lib.seer_poll_device_status.argtypes = [vp, vp]
+    lib.seer_poll_device_status.restype = C.c_int
+    lib.seer_launch_count.argtypes = [vp]
+    lib.seer_launch_count.restype = i64
+    _lib = lib
+    return lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Device (or host) address of a tensor / raw int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != SEER_OK:
+        raise SeerError(status, where)
+
+
+def make_shape(cu_seqlens: Sequence[int], num_q_heads: int, num_kv_heads: int, *, head_dim: int = 128,
+               block: int = 64, gate_dim: int = 128, softmax_scale: float = 0.0) -> seer_shape:
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    s = seer_shape(len(cu) - 1, cu.ctypes.data_as(C.POINTER(C.c_int32)), num_q_heads, num_kv_heads, head_dim, block,
+                   gate_dim, softmax_scale)
+    s._keepalive = cu          # the struct points into this array
+    return s
+
+
+def make_mask_params(mode: int, *, keep_num: int = 1, keep_den: int = 1, k: int = 0, threshold: float = 0.0,
+                     flags: int = SEER_FORCE_DIAG) -> seer_mask_params:
+    return seer_mask_params(mode, keep_num, keep_den, k, threshold, flags)
+
+
+def seer_workspace_bytes(shape: seer_shape) -> int:
+    return int(load_library().seer_workspace_bytes(C.byref(shape)))
+
+
+def seer_scores_elems(shape: seer_shape) -> int:
+    return int(load_library().seer_scores_elems(C.byref(shape)))
+
+
+def seer_mask_rows(shape: seer_shape) -> int:
+    return int(load_library().seer_mask_rows(C.byref(shape)))
+
+
+def seer_causal_blocks(shape: seer_shape) -> int:
+    return int(load_library().seer_causal_blocks(C.byref(shape)))
+
+
+def seer_status_string(status: int) -> str:
+    return load_library().seer_status_string(status).decode()
+
+
+class Context:
+    """Owns a seer_ctx on one device."""
+
+    def __init__(self, device: int = 0):
+        self._lib = load_library()
+        self._h = C.c_void_p()
+        _check(self._lib.seer_create(C.byref(self._h), device), "seer_create")
+        self.device = device
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.seer_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+
+def seer_gate_scores(ctx: Context, shape: seer_shape, q, k, wq, wk, scores, ws, stream=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(ctx._lib.seer_gate_scores(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(wq), _ptr(wk), _ptr(scores),
+                                     _ptr(ws), ws_bytes, _stream(stream)), "seer_gate_scores")
+
+
+def seer_block_mask(ctx: Context, shape: seer_shape, scores, params: seer_mask_params, row_ptr, col_idx,
+                    col_capacity: Optional[int] = None, nnz_out=None, ws=None, stream=None) -> None:
+    if col_capacity is None:
+        col_capacity = 0 if col_idx is None else col_idx.numel()
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(ctx._lib.seer_block_mask(ctx.handle, C.byref(shape), _ptr(scores), C.byref(params), _ptr(row_ptr),
+                                    _ptr(col_idx), col_capacity, _ptr(nnz_out), _ptr(ws), ws_bytes, _stream(stream)),
+           "seer_block_mask")
+
+
+def seer_sparse_attn(ctx: Context, shape: seer_shape, q, k, v, row_ptr, col_idx, o, lse=None, ws=None,
+                     stream=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(ctx._lib.seer_sparse_attn(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(row_ptr),
+                                     _ptr(col_idx), _ptr(o), _ptr(lse), _ptr(ws), ws_bytes, _stream(stream)),
+           "seer_sparse_attn")
+
+
+def seer_set_attn_impl(ctx: Context, impl: int) -> None:
+    _check(ctx._lib.seer_set_attn_impl(ctx.handle, impl), "seer_set_attn_impl")
+
+
+def seer_poll_device_status(ctx: Context, stream=None) -> int:
+    return int(ctx._lib.seer_poll_device_status(ctx.handle, _stream(stream)))
+
+
+def seer_launch_count(ctx: Context) -> int:
+    return int(ctx._lib.seer_launch_count(ctx.handle))

@@ -1,0 +1,220 @@
+// Binary block mask (Sec. 3.3, Eq. 3 TopK / Eq. 4 threshold) as CSR index lists.
+//   count_kernel : one warp per (sequence, head, query-block) row -> number of kept blocks
+//   scan_kernel  : exclusive prefix sum of the counts -> row_ptr, nnz, capacity check
+//   fill_kernel  : one warp per row repeats the selection and writes the ascending list by ballot compaction
+// Selection order in the TopK modes is (score descending, block index ascending): scores become order-preserving
+// 32-bit keys, the key of the last kept candidate is found by a bitwise search over the row held in shared
+// memory, and ties at that key are resolved by rank in index order.
+#include "seer_internal.cuh"
+
+namespace seer {
+
+constexpr int kMaskWarps = 4;
+constexpr int kMaskSmemRowMax = 8192;   // rows up to this many blocks are staged in shared memory
+
+struct RowInfo {
+  const float* s;   // scores of this row
+  int i;            // query block index (row has n = i + 1 causal blocks)
+  bool valid;
+};
+
+__device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const float* __restrict__ scores, int64_t r) {
+  RowInfo ri;
+  ri.valid = r < m.rows;
+  if (!ri.valid) { ri.s = nullptr; ri.i = 0; return ri; }
+  const int b = find_sequence(m.blk_off, m.batch, (int)(r / m.num_q_heads));
+  const int nb = m.blk_off[b + 1] - m.blk_off[b];
+  const int64_t local = r - (int64_t)m.num_q_heads * m.blk_off[b];
+  const int h = (int)(local / nb);
+  ri.i = (int)(local - (int64_t)h * nb);
+  ri.s = scores + m.score_off[b] + ((size_t)h * nb + ri.i) * nb;
+  return ri;
+}
+
+// Order-preserving map fp32 -> uint32 (larger score = larger key); -0 equals +0; NaN -> 0 (never a candidate).
+__device__ __forceinline__ uint32_t score_key(float s) {
+  uint32_t u = __float_as_uint(s);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return 0u;
+  if (u == 0x80000000u) u = 0u;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ bool is_forced(int j, int i, uint32_t flags) {
+  return ((flags & SEER_FORCE_DIAG) && j == i) || ((flags & SEER_FORCE_SINK) && j == 0);
+}
+
+__device__ __forceinline__ int num_forced(int i, uint32_t flags) {
+  int nf = (flags & SEER_FORCE_DIAG) ? 1 : 0;
+  if ((flags & SEER_FORCE_SINK) && !((flags & SEER_FORCE_DIAG) && i == 0)) nf += 1;
+  return nf;
+}
+
+__device__ __forceinline__ int keep_count(int n, const seer_mask_params& p) {
+  if (p.mode == SEER_TOPK_RATIO) {
+    long long k = ((long long)p.keep_num * n + p.keep_den - 1) / p.keep_den;
+    if (k < 1) k = 1;
+    if (k > n) k = n;
+    return (int)k;
+  }
+  int k = p.k < 0 ? 0 : p.k;
+  return k < n ? k : n;
+}
+
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void __launch_bounds__(kMaskWarps * 32)
+count_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, int32_t* __restrict__ row_ptr) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * kMaskWarps + (threadIdx.x >> 5);
+  const RowInfo ri = decode_row(m, scores, r);
+  if (!ri.valid) return;
+  const int n = ri.i + 1;
+  int c = 0;
+  if (p.mode == SEER_THRESHOLD) {
+    for (int j = lane; j < n; j += 32) c += (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold) ? 1 : 0;
+    c = warp_sum(c);
+  } else {
+    for (int j = lane; j < n; j += 32) c += (!is_forced(j, ri.i, p.flags) && score_key(ri.s[j]) != 0u) ? 1 : 0;
+    const int ncand = warp_sum(c);
+    const int nf = num_forced(ri.i, p.flags);
+    const int take = max(keep_count(n, p) - nf, 0);
+    c = nf + min(take, ncand);
+  }
+  if (lane == 0) row_ptr[r + 1] = c;
+}
+
+// Single CTA: in-place inclusive scan of row_ptr[1..rows]; row_ptr[0] = 0.
+__global__ void __launch_bounds__(1024)
+scan_kernel(int64_t rows, int32_t* __restrict__ row_ptr, int64_t col_capacity, int64_t* __restrict__ nnz_out,
+            int* __restrict__ status) {
+  __shared__ long long part[1024];
+  const int t = threadIdx.x;
+  const int64_t per = (rows + 1023) / 1024;
+  const int64_t lo = min(rows, t * per), hi = min(rows, lo + per);
+  long long s = 0;
+  for (int64_t r = lo; r < hi; ++r) s += row_ptr[r + 1];
+  part[t] = s;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {
+    long long v = t >= off ? part[t - off] : 0;
+    __syncthreads();
+    part[t] += v;
+    __syncthreads();
+  }
+  long long run = part[t] - s;   // exclusive prefix of this thread's segment
+  for (int64_t r = lo; r < hi; ++r) {
+    run += row_ptr[r + 1];
+    row_ptr[r + 1] = (int32_t)run;
+  }
+  if (t == 0) {
+    row_ptr[0] = 0;
+    const long long nnz = part[1023];
+    if (nnz_out) *nnz_out = nnz;
+    if (nnz > col_capacity) atomicCAS(status, 0, (int)SEER_ERR_CAPACITY);
+  }
+}
+
+__global__ void __launch_bounds__(kMaskWarps * 32)
+fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, const int32_t* __restrict__ row_ptr,
+            int32_t* __restrict__ col_idx, int64_t col_capacity, int stage_cap) {
+  extern __shared__ uint32_t key_smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t r = (int64_t)blockIdx.x * kMaskWarps + warp;
+  const RowInfo ri = decode_row(m, scores, r);
+  if (!ri.valid) return;
+  const int n = ri.i + 1;
+  const int32_t out0 = row_ptr[r], out1 = row_ptr[r + 1];
+  if ((int64_t)out1 > col_capacity) return;   // this row (and all later ones) do not fit; status already raised
+  int32_t* __restrict__ out = col_idx + out0;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+
+  if (p.mode == SEER_THRESHOLD) {
+    int written = 0;
+    for (int base = 0; base < n; base += 32) {
+      const int j = base + lane;
+      const bool keep = j < n && (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold);
+      const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+      if (keep) out[written + __popc(bal & lt_mask)] = j;
+      written += __popc(bal);
+    }
+    return;
+  }
+
+  // ---- TopK
+  const int nf = num_forced(ri.i, p.flags);
+  const int take = max(keep_count(n, p) - nf, 0);
+  uint32_t* keys = key_smem + (size_t)warp * stage_cap;
+  const bool staged = n <= stage_cap;
+  int c = 0;
+  for (int j = lane; j < n; j += 32) {
+    const uint32_t kk = is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]);
+    if (staged) keys[j] = kk;
+    c += kk != 0u;
+  }
+  const int ncand = warp_sum(c);
+  __syncwarp();
+  auto key_at = [&](int j) -> uint32_t {
+    return staged ? keys[j] : (is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]));
+  };
+
+  uint32_t T = 0u;      // key of the last kept candidate; kept: key > T, plus the first need_eq with key == T
+  int need_eq = 0;
+  if (take >= ncand) {
+    T = 0u; need_eq = 0;            // every candidate is kept (key >= 1 > 0)
+  } else if (take == 0) {
+    T = 0xffffffffu; need_eq = 0;   // nothing beyond the forced blocks
+  } else {
+    for (int bit = 31; bit >= 0; --bit) {
+      const uint32_t cand = T | (1u << bit);
+      int cnt = 0;
+      for (int j = lane; j < n; j += 32) cnt += key_at(j) >= cand;
+      if (warp_sum(cnt) >= take) T = cand;
+    }
+    int gt = 0;
+    for (int j = lane; j < n; j += 32) gt += key_at(j) > T;
+    need_eq = take - warp_sum(gt);
+  }
+  int written = 0, eq_seen = 0;
+  for (int base = 0; base < n; base += 32) {
+    const int j = base + lane;
+    const uint32_t kk = j < n ? key_at(j) : 0u;
+    const bool forced = j < n && is_forced(j, ri.i, p.flags);
+    const bool eq = kk != 0u && kk == T;
+    const uint32_t eq_bal = __ballot_sync(0xffffffffu, eq);
+    const bool keep = forced || (kk != 0u && kk > T) || (eq && eq_seen + __popc(eq_bal & lt_mask) < need_eq);
+    const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+    if (keep) out[written + __popc(bal & lt_mask)] = j;
+    written += __popc(bal);
+    eq_seen += __popc(eq_bal);
+  }
+}
+
+int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer_mask_params& p, int32_t* row_ptr,
+                int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream) {
+  if (m.rows == 0) {
+    cudaMemsetAsync(row_ptr, 0, sizeof(int32_t), stream);
+    if (nnz_out) cudaMemsetAsync(nnz_out, 0, sizeof(int64_t), stream);
+    return 0;
+  }
+  const unsigned grid = (unsigned)((m.rows + kMaskWarps - 1) / kMaskWarps);
+  count_kernel<<<grid, kMaskWarps * 32, 0, stream>>>(m, scores, p, row_ptr);
+  scan_kernel<<<1, 1024, 0, stream>>>(m.rows, row_ptr, col_capacity, nnz_out, ctx->d_status);
+  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // longer rows re-read their scores instead
+  const size_t smem = (size_t)kMaskWarps * stage_cap * sizeof(uint32_t);
+  fill_kernel<<<grid, kMaskWarps * 32, smem, stream>>>(m, scores, p, row_ptr, col_idx, col_capacity, stage_cap);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 3 : -(int)e;
+}
+
+seer_status init_mask(seer_ctx* ctx) {
+  (void)ctx;
+  cudaError_t e = cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kMaskWarps * kMaskSmemRowMax * (int)sizeof(uint32_t));
+  return e == cudaSuccess ? SEER_OK : SEER_ERR_CUDA;
+}
+
+}  // namespace seer

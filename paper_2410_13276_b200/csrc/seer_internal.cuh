@@ -1,0 +1,104 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "seer.h"
+
+namespace seer {
+
+constexpr int kBlock = 64;      // gate block = attention tile
+constexpr int kHeadDim = 128;
+constexpr int kGateDim = 128;
+constexpr int kMaxBatch = 4096;
+constexpr int kMetaSlots = 8;
+constexpr int kPoolChunk = 16;  // blocks pooled and projected by one CTA of the gate's first kernel
+constexpr int kScoreTile = 64;  // score rows handled by one CTA of the gate's second kernel
+
+// Per-batch metadata the kernels read from device memory.
+struct SeqMeta {
+  const int32_t* cu_seqlens;   // [batch+1] token offsets
+  const int32_t* blk_off;      // [batch+1] cumulative number of blocks
+  const int64_t* score_off;    // [batch+1] Hq * cumulative nb^2
+  const int32_t* chunk_off;    // [batch+1] cumulative ceil(nb / kPoolChunk)
+  const int32_t* tile_off;     // [batch+1] cumulative ceil(nb / kScoreTile)
+  int32_t batch;
+  int32_t num_q_heads;
+  int32_t num_kv_heads;
+  int32_t group;               // Hq / Hkv
+  int32_t total_tokens;
+  int32_t total_blocks;
+  int32_t total_chunks;
+  int32_t total_tiles;
+  int32_t max_nb;
+  int64_t rows;                // Hq * total_blocks
+  int64_t score_elems;
+  float softmax_scale;
+};
+
+struct MetaSlot {
+  std::vector<int32_t> key;    // cu_seqlens + Hq: what the slot currently describes
+  void* dev = nullptr;
+  void* pinned = nullptr;
+  cudaEvent_t ready = nullptr;     // upload finished
+  cudaEvent_t last_use = nullptr;  // last library call that read the slot
+  uint64_t stamp = 0;
+};
+
+}  // namespace seer
+
+struct seer_ctx {
+  int device = 0;
+  int num_sms = 0;
+  int* d_status = nullptr;
+  int attn_impl = 0;
+  int64_t launches = 0;
+  uint64_t clock = 0;
+  seer::MetaSlot slots[seer::kMetaSlots];
+  void* tmap_encode = nullptr;   // cuTensorMapEncodeTiled, resolved at run time
+};
+
+namespace seer {
+
+// Validates the shape, makes its metadata resident on the device (ordered before later work on `stream`)
+// and fills `m`.  `slot_out` identifies the slot to pass to finish_call.
+seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream, SeqMeta* m, int* slot_out);
+void finish_call(seer_ctx* ctx, int slot, cudaStream_t stream);
+
+// Host-only shape arithmetic (no CUDA calls): returns SEER_OK and fills totals.
+struct ShapeTotals {
+  int64_t total_tokens, total_blocks, total_chunks, total_tiles, rows, score_elems, causal_blocks;
+  int32_t max_nb;
+};
+seer_status shape_totals(const seer_shape* shape, ShapeTotals* t);
+
+size_t gate_workspace_bytes(const ShapeTotals& t, const seer_shape* shape);
+
+// Kernel launchers (each returns the number of kernels it launched, or a negative cudaError).
+int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const float* Wq, const float* Wk,
+                float* scores, void* ws, cudaStream_t stream);
+int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer_mask_params& p, int32_t* row_ptr,
+                int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream);
+int launch_attn_mma(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
+                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
+int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
+                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
+seer_status init_gate(seer_ctx* ctx);
+seer_status init_mask(seer_ctx* ctx);
+seer_status init_attn_mma(seer_ctx* ctx);
+seer_status init_attn_tc(seer_ctx* ctx);
+
+// Sequence that owns global block index gb: largest b with blk_off[b] <= gb (empty sequences are skipped).
+__device__ __forceinline__ int find_sequence(const int32_t* __restrict__ off, int batch, int x) {
+  int lo = 0, hi = batch;  // off[lo] <= x < off[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (off[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+}  // namespace seer

@@ -1,0 +1,320 @@
+"""GPU-vs-oracle parity through the C ABI (needs a B200).
+
+Tolerances (stated by the benchmark spec): block index lists bit-exact when built from
+identical scores; gate scores within 1e-3 relative; attention output within
+2e-2 absolute + 1e-2 relative (bf16 I/O, fp32 accumulation).  Attention is
+additionally held to a relative RMS error <= 1e-2 per (head, query block),
+because at long context |o| is itself ~1e-2 and the absolute term alone would
+accept anything.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import seer_oracle as O
+from paper_2410_13276_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rt():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("no CUDA device: the gpu tests must run on a B200")
+    from paper_2410_13276_b200 import binding as B
+    from paper_2410_13276_b200.prefill import Prefill
+    ctx = B.Context(0)
+    yield B, Prefill, ctx
+    ctx.close()
+
+
+def make_prefill(rt, w, **kw):
+    B, Prefill, ctx = rt
+    p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx, **kw)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    return p
+
+
+def params_of(B, spec, threshold=None):
+    thr = spec.threshold if threshold is None else threshold
+    return B.make_mask_params(spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                              threshold=0.0 if thr is None else thr, flags=spec.flags)
+
+
+def check_scores(got_flat, ref_list, w):
+    got = O.unflatten_scores(got_flat, w.cu_seqlens, w.block, w.num_q_heads)
+    for g, r in zip(got, ref_list):
+        nb = r.shape[-1]
+        il = np.tril_indices(nb)
+        gg, rr = g[:, il[0], il[1]].astype(np.float64), r[:, il[0], il[1]].astype(np.float64)
+        tol = np.where(np.abs(rr) < 1e-30, 1e-33, 1e-3 * np.abs(rr))
+        bad = np.abs(gg - rr) > tol
+        assert not bad.any(), f"{bad.sum()} scores off, worst rel {np.max(np.abs(gg - rr) / np.maximum(np.abs(rr), 1e-300)):.3e}"
+
+
+def check_attention(o_gpu, lse_gpu, o_ref, lse_ref, w, rows=None):
+    """o_gpu [T,Hq,d] fp32 (widened bf16), o_ref fp64 with NaN where not computed."""
+    done = ~np.isnan(o_ref[..., 0])
+    assert done.any()
+    x, r = o_gpu[done].astype(np.float64), o_ref[done]
+    err = np.abs(x - r)
+    assert np.all(err <= 2e-2 + 1e-2 * np.abs(r)), f"max abs err {err.max():.3e}"
+    # per (token, head) relative RMS, then the worst over rows
+    rms = np.sqrt((err ** 2).sum(-1)) / np.maximum(np.sqrt((r ** 2).sum(-1)), 1e-30)
+    assert rms.max() <= 1e-2, f"worst relative RMS {rms.max():.3e}"
+    assert err.max() <= 2.0 ** -6 * np.abs(r).max()
+    if lse_gpu is not None:
+        lr = lse_ref.T[done]
+        lg = lse_gpu.T[done].astype(np.float64)
+        fin = np.isfinite(lr)
+        assert np.all(np.abs(lg[fin] - lr[fin]) <= 2e-3 + 1e-3 * np.abs(lr[fin]))
+        assert np.all(lg[~fin] == lr[~fin])
+
+
+SMALL = [
+    dict(seed=100, seqlens=[64], hq=1, hkv=1),
+    dict(seed=101, seqlens=[1], hq=2, hkv=1),
+    dict(seed=102, seqlens=[200], hq=4, hkv=2),
+    dict(seed=103, seqlens=[130, 0, 777, 64, 65], hq=6, hkv=2),
+    dict(seed=104, seqlens=[1500, 333], hq=5, hkv=1),
+    dict(seed=105, seqlens=[4099], hq=8, hkv=4, q_gain=3.0),
+]
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: f"s{c['seed']}")
+def test_gate_small(rt, cfg):
+    w = W.make_small(**cfg)
+    p = make_prefill(rt, w)
+    p.gate()
+    assert p.status() == 0
+    check_scores(p.scores_host(), O.gate_scores(w.q, w.k, w.wq, w.wk, w.cu_seqlens, 64), w)
+
+
+@pytest.mark.parametrize("name", ["c1", "c2s", "c4s", "c5s"])
+def test_gate_workloads(rt, name):
+    w = W.make_workload(name)
+    p = make_prefill(rt, w)
+    p.gate()
+    check_scores(p.scores_host(), O.gate_scores(w.q, w.k, w.wq, w.wk, w.cu_seqlens, 64), w)
+
+
+def mask_cases(B):
+    D, S = B.SEER_FORCE_DIAG, B.SEER_FORCE_SINK
+    cases = []
+    for flags in (0, D, D | S, S):
+        for num, den in ((1, 2), (1, 10), (1, 1), (3, 7)):
+            cases.append(dict(mode=B.SEER_TOPK_RATIO, keep_num=num, keep_den=den, flags=flags))
+        for k in (0, 1, 3, 40):
+            cases.append(dict(mode=B.SEER_TOPK_COUNT, k=k, flags=flags))
+        for thr in (-np.inf, 0.0, 0.02, 0.25, 1.0, np.inf):
+            cases.append(dict(mode=B.SEER_THRESHOLD, threshold=float(thr), flags=flags))
+    return cases
+
+
+@pytest.mark.parametrize("kind", ["random", "ties", "nan", "softmax"])
+def test_mask_bit_exact_from_oracle_scores(rt, kind):
+    B, Prefill, ctx = rt
+    cu = np.array([0, 64 * 37 + 5, 64 * 37 + 5, 64 * 37 + 5 + 64 * 70, 64 * 37 + 5 + 64 * 70 + 1], np.int32)
+    hq = 3
+    rng = np.random.default_rng(7)
+    nbs = O.blocks_per_sequence(cu, 64)
+    scores = []
+    for nb in nbs:
+        nb = int(nb)
+        s = rng.random((hq, nb, nb)).astype(np.float32)
+        if kind == "ties":
+            s = (np.floor(s * 5) / 5).astype(np.float32)
+            s[0] = 0.0
+            s[1, :, ::2] = -0.0
+        elif kind == "nan":
+            s[rng.random(s.shape) < 0.2] = np.nan
+            s[rng.random(s.shape) < 0.05] = -np.inf
+        elif kind == "softmax":
+            s = O.causal_softmax_rows(rng.standard_normal((hq, nb, nb)) * 3).astype(np.float32)
+        scores.append(s)
+    p = Prefill(cu, hq, 1, ctx=ctx)
+    p.set_scores(O.flatten_scores(scores))
+    for case in mask_cases(B):
+        p.mask(B.make_mask_params(**case))
+        assert p.status() == 0
+        rp, col = p.lists_host()
+        orp, ocol = O.block_mask(scores, case["mode"], keep_num=case.get("keep_num", 1), keep_den=case.get("keep_den", 1),
+                                 k=case.get("k", 0), threshold=case.get("threshold", 0.0), flags=case["flags"])
+        assert np.array_equal(rp, orp), case
+        assert np.array_equal(col, ocol), case
+        assert int(p.nnz.item()) == len(ocol)
+
+
+@pytest.mark.parametrize("name", ["c1", "c3s", "c5s"])
+def test_mask_bit_exact_from_gpu_scores(rt, name):
+    B, Prefill, ctx = rt
+    w = W.make_workload(name)
+    p = make_prefill(rt, w)
+    p.gate()
+    gs = O.unflatten_scores(p.scores_host(), w.cu_seqlens, 64, w.num_q_heads)
+    specs = list(w.masks) + [W.MaskSpec(W.MODE_THRESHOLD, threshold=2e-3, flags=W.FORCE_DIAG)]
+    for spec in specs:
+        thr = spec.threshold if spec.threshold is not None else 5e-3
+        p.mask(params_of(B, spec, thr))
+        rp, col = p.lists_host()
+        orp, ocol = O.block_mask(gs, spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                                 threshold=thr, flags=spec.flags)
+        assert np.array_equal(rp, orp) and np.array_equal(col, ocol)
+
+
+def test_mask_capacity_overflow_is_reported_and_row_ptr_complete(rt):
+    B, Prefill, ctx = rt
+    cu = np.array([0, 640], np.int32)
+    scores = [np.random.default_rng(0).random((2, 10, 10)).astype(np.float32)]
+    p = Prefill(cu, 2, 1, ctx=ctx, col_capacity=17)
+    p.set_scores(O.flatten_scores(scores))
+    p.col_idx.fill_(-7)
+    p.mask(B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=1))
+    assert p.status() == 4                         # SEER_ERR_CAPACITY
+    assert p.status() == 0                         # polling clears it
+    orp, ocol = O.block_mask(scores, O.MODE_TOPK_RATIO, keep_num=1, keep_den=1)
+    rp = p.row_ptr.cpu().numpy()
+    assert np.array_equal(rp, orp) and int(p.nnz.item()) == 110
+    col = p.col_idx.cpu().numpy()
+    fits = int(np.searchsorted(orp, 17, side="right")) - 1      # rows that end at or below the capacity
+    assert np.array_equal(col[: orp[fits]], ocol[: orp[fits]]) and np.all(col[orp[fits]:] == -7)
+
+
+def run_attention(rt, w, row_ptr, col, impl):
+    B, Prefill, ctx = rt
+    B.seer_set_attn_impl(ctx, impl)
+    try:
+        p = make_prefill(rt, w)
+        p.set_lists(row_ptr, col)
+        p.o.fill_(float("nan"))
+        p.attn()
+        st = p.status()
+        return p.o_host(), p.lse_host(), st
+    finally:
+        B.seer_set_attn_impl(ctx, 0)
+
+
+IMPLS = [0, 1]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: f"s{c['seed']}")
+@pytest.mark.parametrize("lists", ["full", "topk", "diag"])
+def test_attention_small(rt, cfg, lists, impl):
+    w = W.make_small(**cfg)
+    if lists == "full":
+        rp, col = O.full_causal_lists(w.cu_seqlens, 64, w.num_q_heads)
+    else:
+        rng = np.random.default_rng(cfg["seed"])
+        scores = [rng.random((w.num_q_heads, int(nb), int(nb))).astype(np.float32) for nb in w.num_blocks]
+        if lists == "topk":
+            rp, col = O.block_mask(scores, O.MODE_TOPK_RATIO, keep_num=1, keep_den=3, flags=O.FORCE_DIAG | O.FORCE_SINK)
+        else:
+            rp, col = O.block_mask(scores, O.MODE_TOPK_COUNT, k=1, flags=O.FORCE_DIAG)
+    o, lse, st = run_attention(rt, w, rp, col, impl)
+    assert st == 0
+    o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64,
+                                        1 / math.sqrt(128))
+    check_attention(o, lse, o_ref, lse_ref, w)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_attention_config1_end_to_end_lists(rt, impl):
+    """Config 1 in full: oracle gate -> oracle mask -> both attention paths on identical lists."""
+    B, Prefill, ctx = rt
+    w = W.make_workload("c1")
+    spec = w.masks[0]
+    s = O.gate_scores(w.q, w.k, w.wq, w.wk, w.cu_seqlens, 64)
+    rp, col = O.block_mask(s, spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, flags=spec.flags)
+    assert len(col) == 1088
+    o, lse, st = run_attention(rt, w, rp, col, impl)
+    assert st == 0
+    o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, 4, 1, 64, 1 / math.sqrt(128))
+    check_attention(o, lse, o_ref, lse_ref, w)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_attention_empty_rows_and_unsorted_lists(rt, impl):
+    w = W.make_small(110, [256], 2, 1)
+    # head 0: rows 0..3 with lists [], [1,0], [2], [3,0,1]; head 1: all empty
+    rp = np.array([0, 0, 2, 3, 6, 6, 6, 6, 6], np.int64)
+    col = np.array([1, 0, 2, 3, 0, 1], np.int32)
+    o, lse, st = run_attention(rt, w, rp, col, impl)
+    assert st == 0
+    o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, 2, 1, 64, 1 / math.sqrt(128))
+    check_attention(o, lse, o_ref, lse_ref, w)
+    assert np.all(o[:64, 0] == 0) and np.all(o[:, 1] == 0) and np.all(np.isneginf(lse[1]))
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_attention_flags_out_of_range_index_without_touching_it(rt, impl):
+    w = W.make_small(111, [192], 1, 1)
+    rp = np.array([0, 1, 3, 5], np.int64)
+    col = np.array([0, 0, 5, -3, 2], np.int32)      # row 1 lists block 5 (> i), row 2 lists block -3
+    o, lse, st = run_attention(rt, w, rp, col, impl)
+    assert st == 5                                   # SEER_ERR_INVALID_INDEX
+    good_rp = np.array([0, 1, 2, 3], np.int64)
+    good_col = np.array([0, 0, 2], np.int32)
+    o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, good_rp, good_col, 1, 1, 64, 1 / math.sqrt(128))
+    check_attention(o, lse, o_ref, lse_ref, w)      # the bad entries were skipped
+
+
+@pytest.mark.parametrize("name", ["c2s", "c3s", "c4s", "c5s"])
+def test_attention_reduced_twins_gpu_pipeline(rt, name):
+    """Whole GPU path (gate -> mask -> attention); the oracle attends over the GPU's own lists."""
+    B, Prefill, ctx = rt
+    w = W.make_workload(name)
+    p = make_prefill(rt, w)
+    for spec in w.masks:
+        thr = {0.90: 6.5e-3, 0.85: 2.5e-3, 0.92: 3e-3}.get(spec.target_sparsity, 0.0)
+        p.run(params_of(B, spec, thr))
+        assert p.status() == 0
+        rp, col = p.lists_host()
+        o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64,
+                                            1 / math.sqrt(128))
+        check_attention(p.o_host(), p.lse_host(), o_ref, lse_ref, w)
+
+
+def test_tc_and_mma_kernels_agree_on_device(rt):
+    B, Prefill, ctx = rt
+    w = W.make_workload("c3s")
+    p = make_prefill(rt, w)
+    p.run(params_of(B, w.masks[2]))
+    o0 = p.o_host().copy()
+    B.seer_set_attn_impl(ctx, 1)
+    try:
+        p.attn()
+        o1 = p.o_host()
+    finally:
+        B.seer_set_attn_impl(ctx, 0)
+    assert np.abs(o0 - o1).max() <= 2e-2
+
+
+def test_invalid_arguments_are_rejected_on_the_host(rt):
+    B, Prefill, ctx = rt
+    import torch
+    buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    for bad in (dict(head_dim=64), dict(block=128), dict(gate_dim=64)):
+        s = B.make_shape([0, 128], 2, 1, **bad)
+        with pytest.raises(B.SeerError) as e:
+            B.seer_gate_scores(ctx, s, buf, buf, buf, buf, buf, buf)
+        assert e.value.status == 2
+    with pytest.raises(B.SeerError) as e:
+        B.seer_gate_scores(ctx, B.make_shape([0, 128], 3, 2), buf, buf, buf, buf, buf, buf)
+    assert e.value.status == 2
+    with pytest.raises(B.SeerError) as e:
+        B.seer_gate_scores(ctx, B.make_shape([0, 128, 64], 2, 1), buf, buf, buf, buf, buf, buf)
+    assert e.value.status == 1
+    s = B.make_shape([0, 128], 2, 1)
+    with pytest.raises(B.SeerError) as e:
+        B.seer_gate_scores(ctx, s, buf, buf, buf, buf, buf, buf[:16])
+    assert e.value.status == 3
+    with pytest.raises(B.SeerError) as e:
+        B.seer_gate_scores(ctx, s, None, buf, buf, buf, buf, buf)
+    assert e.value.status == 1
+    with pytest.raises(B.SeerError) as e:
+        B.seer_block_mask(ctx, s, buf, B.make_mask_params(7), buf, buf, 16)
+    assert e.value.status == 1
+    assert B.seer_poll_device_status(ctx) == 0

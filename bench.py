@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the SeerAttention prefill hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3] [--keep 1/10]
+
+One step = one pass of the whole hot path (seer_gate_scores -> seer_block_mask -> seer_sparse_attn) over one
+synthetic layer.  Default workload: Llama-3-8B-shaped layer at 131072 tokens, TopK keeping 1/10 of the causal
+blocks (90 % block sparsity), diagonal and sink forced.  Prints ONE JSON line on rank 0.
+
+value  = kept-block attention FLOPs (4 * 64 * 64 * 128 per kept block) of all ranks / step time, inputs resident in HBM.
+e2e    = same, through seer_prefill_host: pinned host buffers in, pinned host buffer out, copies inside the timed region.
+roofline = the attention kernel alone (CUDA events around its launch) against the measured bf16 dense peak.
+cpu_baseline = the fp64 CPU oracle's attention on a sample of rows of the same workload, on this machine's host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FLOP_PER_BLOCK = 4 * 64 * 64 * 128
+METRIC = "sparse_prefill_attention_effective_tflops_128k_90pct_block_sparsity"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--keep", default="1/10", help="TopK ratio for the c3 workload")
+    ap.add_argument("--attn-impl", type=int, default=0, help="0 tcgen05 kernel, 1 mma.sync cross-check kernel")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense-list run of the attention kernel")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def pick_mask(w, args):
+    from paper_2410_13276_b200 import workloads as W
+    if w.name.startswith("c3"):
+        num, den = (int(x) for x in args.keep.split("/"))
+        return W.MaskSpec(W.MODE_TOPK_RATIO, num, den, flags=W.FORCE_DIAG | W.FORCE_SINK)
+    spec = w.masks[0]
+    if spec.mode == W.MODE_THRESHOLD and spec.threshold is None:
+        with open(os.path.join(ROOT, "tests", "golden", "thresholds.json")) as f:
+            spec.threshold = float.fromhex(json.load(f)[w.name]["threshold_hex"])
+    return spec
+
+
+def workload_desc(w, spec):
+    return {"workload": f"{w.name}: 1 attention layer, batch {len(w.cu_seqlens) - 1}, tokens {w.total_tokens}, "
+                        f"{w.num_q_heads} q heads / {w.num_kv_heads} kv heads, head_dim 128, block 64, causal",
+            "mask": ({0: "topk_ratio", 1: "topk_count", 2: "threshold"}[spec.mode]
+                     + (f" {spec.keep_num}/{spec.keep_den}" if spec.mode == 0 else
+                        f" {spec.threshold!r}" if spec.mode == 2 else f" {spec.k}")
+                     + f", flags {spec.flags}"),
+            "l2": "inputs larger than L2 (no flush)"}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d["bf16_tflops"], d.get("bf16_tflops_sustained"), d["hbm_gbs"], "measured"
+    return 1590.0, 1400.0, 6650.0, "fallback"
+
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.strip().lower() == "active":
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "power_w_max": max(power), "samples": len(sm)}
+
+
+def cpu_oracle_sample(w, rp, col, budget_rows=None):
+    """Times the oracle's attention on a sample of (head, query-block) rows.  Returns (tflops, seconds, description, cores)."""
+    from oracle import seer_oracle as O
+    from paper_2410_13276_b200 import workloads as W
+    rows = W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=1234, per_head_random=2, heads=range(0, w.num_q_heads, 4))
+    if budget_rows:
+        rows = rows[:: max(1, len(rows) // budget_rows)]
+    blocks = int(sum(int(rp[r + 1] - rp[r]) for r in rows))
+    t0 = time.perf_counter()
+    O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64, w.softmax_scale, rows=rows)
+    dt = time.perf_counter() - t0
+    cores = len(os.sched_getaffinity(0))
+    return blocks * FLOP_PER_BLOCK / dt / 1e12, dt, f"oracle attention on {len(rows)} sampled (head, query-block) rows = {blocks} kept blocks; gate and mask oracle not included", cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import seer_oracle as O
+    from paper_2410_13276_b200 import workloads as W
+    w = W.make_workload(args.workload)
+    spec = pick_mask(w, args)
+    # lists for the sampled rows come from the oracle's own gate + mask on a slice of heads would take minutes at
+    # this size; the sample uses TopK lists of seeded random scores with the same keep ratio instead (same row lengths).
+    nbs = w.num_blocks
+    rng = np.random.default_rng(99)
+    heads = list(range(0, w.num_q_heads, 4))
+    rp = np.zeros(int(nbs.sum()) * w.num_q_heads + 1, dtype=np.int64)
+    cols = []
+    picks = []
+    base = 0
+    for nb in nbs:
+        nb = int(nb)
+        for h in range(w.num_q_heads):
+            for i in range(nb):
+                rp[base + h * nb + i + 1] = 0
+        for h in heads:
+            for i in {0, nb // 2, nb - 1}:
+                picks.append(base + h * nb + i)
+        base += nb * w.num_q_heads
+    picks = sorted(set(picks))
+    lists = {}
+    for r in picks:
+        # decode i from r for the single-sequence / multi-sequence layout
+        b = 0
+        off = 0
+        for bb, nb in enumerate(nbs):
+            if r < off + int(nb) * w.num_q_heads:
+                b = bb
+                break
+            off += int(nb) * w.num_q_heads
+        i = (r - off) % int(nbs[b])
+        s = rng.random(i + 1).astype(np.float32)
+        lists[r] = O.select_row(s, i, spec.mode if spec.mode != W.MODE_THRESHOLD else O.MODE_TOPK_RATIO,
+                                keep_num=spec.keep_num if spec.mode == 0 else 1, keep_den=spec.keep_den if spec.mode == 0 else 10,
+                                k=spec.k, flags=spec.flags)
+    counts = np.zeros(len(rp) - 1, dtype=np.int64)
+    for r, l in lists.items():
+        counts[r] = len(l)
+    rp[1:] = np.cumsum(counts)
+    col = np.concatenate([np.asarray(lists[r], np.int32) for r in picks])
+    blocks = int(counts.sum())
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64, w.softmax_scale, rows=picks)
+        if it >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    ms = 1e3 * float(np.mean(times))
+    val = blocks * FLOP_PER_BLOCK / (ms * 1e-3) / 1e12
+    cores = len(os.sched_getaffinity(0))
+    sample = f"oracle attention on {len(picks)} sampled (head, query-block) rows = {blocks} kept blocks per step"
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                      "config": workload_desc(w, spec),
+                      "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+                      "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    from paper_2410_13276_b200 import binding as B, workloads as W
+    from paper_2410_13276_b200.prefill import Prefill
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # every rank runs the same layer on its own GPU: shards are independent (no data-path collective) -> weak scaling
+    w = W.make_workload(args.workload)
+    spec = pick_mask(w, args)
+    p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, device=local, want_lse=False)
+    B.seer_set_attn_impl(p.ctx, args.attn_impl)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    params = B.make_mask_params(spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                                threshold=spec.threshold or 0.0, flags=spec.flags)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        p.run(params)
+    barrier()
+    assert p.status() == 0, "device status raised during warm-up"
+    nnz = int(p.nnz.item())
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    l0 = B.seer_launch_count(p.ctx)
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for s in range(args.steps):
+        ev[s][0].record(stream); p.gate()
+        ev[s][1].record(stream); p.mask(params)
+        ev[s][2].record(stream); p.attn()
+        ev[s][3].record(stream)
+    t_end.record(stream)
+    barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    launches = B.seer_launch_count(p.ctx) - l0
+    clocks = sampler.stop() if sampler else None
+    assert p.status() == 0
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_step = total_ms / args.steps
+    gate_ms = float(np.median([e[0].elapsed_time(e[1]) for e in ev]))
+    mask_ms = float(np.median([e[1].elapsed_time(e[2]) for e in ev]))
+    attn_all = [e[2].elapsed_time(e[3]) for e in ev]
+    attn_ms = float(np.mean(attn_all))
+    flops = nnz * FLOP_PER_BLOCK
+    value = world * flops / (ms_step * 1e-3) / 1e12
+
+    # dense-list run of the same attention kernel (speedup column), outside the timed region
+    dense_ms = None
+    if not args.no_dense and rank == 0:
+        dparams = B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=1, flags=B.SEER_FORCE_DIAG)
+        p.mask(dparams)
+        p.attn(); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); p.attn(); p.attn(); b.record(stream); torch.cuda.synchronize()
+        dense_ms = a.elapsed_time(b) / 2
+        p.mask(params)
+
+    # end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        shape = p.shape
+        hq = torch.from_numpy(w.q.view(np.int16)).pin_memory()
+        hk = torch.from_numpy(w.k.view(np.int16)).pin_memory()
+        hv = torch.from_numpy(w.v.view(np.int16)).pin_memory()
+        hwq = torch.from_numpy(w.wq).pin_memory(); hwk = torch.from_numpy(w.wk).pin_memory()
+        ho = torch.empty((w.total_tokens, w.num_q_heads, 128), dtype=torch.int16).pin_memory()
+        arena = torch.empty(B.seer_prefill_host_arena_bytes(shape), dtype=torch.uint8, device="cuda")
+        n_e2e = max(2, min(args.steps, 5))
+        for _ in range(2):
+            B.seer_prefill_host(p.ctx, shape, hq, hk, hv, hwq, hwk, params, ho, None, arena)
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n_e2e):
+            B.seer_prefill_host(p.ctx, shape, hq, hk, hv, hwq, hwk, params, ho, None, arena)
+        b.record(stream)
+        barrier()
+        e_ms = a.elapsed_time(b) / n_e2e
+        if world > 1:
+            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2 + hwq.numel() * 4 + hwk.numel() * 4
+        e2e = {"value": world * flops / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e_ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(ho.numel() * 2), "steps": n_e2e}
+        del arena
+
+    if rank == 0:
+        burst, sustained, hbm, src = peaks()
+        achieved = flops / (attn_ms * 1e-3) / 1e12
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "attn_traffic.json")
+        if os.path.exists(tpath):
+            with open(tpath) as f:
+                tj = json.load(f)
+            traffic = tj.get("dram_bytes_per_kept_block", 0) * nnz or None
+        out = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+               "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_desc(w, spec),
+               "kept_blocks": nnz, "stage_ms": {"gate": gate_ms, "mask": mask_ms, "attn": attn_ms,
+                                                "attn_min": float(min(attn_all))},
+               "attn_kernel": "tcgen05" if args.attn_impl == 0 else "mma.sync",
+               "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
+                            "frac": achieved / burst, "peak_source": f"bf16 dense burst, of {src}",
+                            "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
+                            "kernel": "seer_sparse_attn"},
+               "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
+               "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
+        if dense_ms:
+            dense_blocks = B.seer_causal_blocks(p.shape)
+            out["dense"] = {"attn_ms": dense_ms, "tflops": dense_blocks * FLOP_PER_BLOCK / (dense_ms * 1e-3) / 1e12,
+                            "speedup_sparse_over_dense": dense_ms / attn_ms}
+        if not args.no_cpu:
+            rp, col = p.lists_host()
+            v, dt, desc, cores = cpu_oracle_sample(w, rp, col)
+            out["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc,
+                                   "seconds": dt}
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

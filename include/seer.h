@@ -128,6 +128,18 @@ seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);
 /* Synchronises `stream`, returns the device status word (SEER_OK if nothing was raised) and clears it. */
 seer_status seer_poll_device_status(seer_ctx* ctx, void* stream);
 
+/* Whole path from HOST buffers: copies q, k, v, Wq, Wk to the device, runs seer_gate_scores -> seer_block_mask ->
+ * seer_sparse_attn and copies o (and lse if lse_host is not NULL) back, all enqueued on `stream` (Sec. 3.3: "Inference with
+ * SeerAttention").  Host buffers should be page-locked for the copies to be asynchronous; they must stay valid, and
+ * o_host must not be read, until the stream has been synchronised.  `arena` is a caller-owned DEVICE buffer of at least
+ * seer_prefill_host_arena_bytes(shape) bytes, 256-byte aligned, that holds every intermediate; the call allocates nothing.
+ * col_idx inside the arena is sized for the full causal mask, so SEER_ERR_CAPACITY cannot occur. */
+size_t seer_prefill_host_arena_bytes(const seer_shape* shape);
+seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void* q_host, const void* k_host,
+                              const void* v_host, const float* Wq_host, const float* Wk_host,
+                              const seer_mask_params* params, void* o_host, float* lse_host, void* arena,
+                              size_t arena_bytes, void* stream);
+
 /* Number of kernels the library has launched through this context since creation (for launch accounting). */
 int64_t seer_launch_count(const seer_ctx* ctx);
 

@@ -24,7 +24,8 @@ STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER
 # every symbol include/seer.h declares
 EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
-           "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count"]
+           "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
+           "seer_prefill_host"]
 
 
 class SeerError(RuntimeError):
@@ -85,6 +86,10 @@ def load_library() -> C.CDLL:
     lib.seer_poll_device_status.restype = C.c_int
     lib.seer_launch_count.argtypes = [vp]
     lib.seer_launch_count.restype = i64
+    lib.seer_prefill_host_arena_bytes.argtypes = [shp]
+    lib.seer_prefill_host_arena_bytes.restype = sz
+    lib.seer_prefill_host.argtypes = [vp, shp, vp, vp, vp, vp, vp, C.POINTER(seer_mask_params), vp, vp, vp, sz, vp]
+    lib.seer_prefill_host.restype = C.c_int
     _lib = lib
     return lib
 
@@ -205,3 +210,16 @@ def seer_poll_device_status(ctx: Context, stream=None) -> int:
 
 def seer_launch_count(ctx: Context) -> int:
     return int(ctx._lib.seer_launch_count(ctx.handle))
+
+
+def seer_prefill_host_arena_bytes(shape: seer_shape) -> int:
+    return int(load_library().seer_prefill_host_arena_bytes(C.byref(shape)))
+
+
+def seer_prefill_host(ctx: Context, shape: seer_shape, q_host, k_host, v_host, wq_host, wk_host,
+                      params: seer_mask_params, o_host, lse_host, arena, stream=None) -> None:
+    """Host tensors (ideally pinned) in, host tensors out; `arena` is a device tensor."""
+    _check(ctx._lib.seer_prefill_host(ctx.handle, C.byref(shape), _ptr(q_host), _ptr(k_host), _ptr(v_host),
+                                      _ptr(wq_host), _ptr(wk_host), C.byref(params), _ptr(o_host), _ptr(lse_host),
+                                      _ptr(arena), arena.numel() * arena.element_size(), _stream(stream)),
+           "seer_prefill_host")

@@ -307,4 +307,78 @@ seer_status seer_poll_device_status(seer_ctx* ctx, void* stream_) {
 
 int64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
+namespace {
+struct ArenaLayout {
+  size_t q, k, v, o, wq, wk, scores, row_ptr, col_idx, nnz, lse, ws, total;
+};
+ArenaLayout arena_layout(const seer_shape* s, const ShapeTotals& t) {
+  ArenaLayout a;
+  size_t p = 0;
+  auto take = [&](size_t bytes) { size_t at = p; p = align_up(p + bytes, 256); return at; };
+  const size_t T = (size_t)t.total_tokens;
+  a.q = take(T * s->num_q_heads * kHeadDim * 2);
+  a.k = take(T * s->num_kv_heads * kHeadDim * 2);
+  a.v = take(T * s->num_kv_heads * kHeadDim * 2);
+  a.o = take(T * s->num_q_heads * kHeadDim * 2);
+  a.wq = take((size_t)s->num_q_heads * kHeadDim * kGateDim * 4);
+  a.wk = take((size_t)s->num_kv_heads * kHeadDim * kGateDim * 4);
+  a.scores = take((size_t)t.score_elems * 4);
+  a.row_ptr = take(((size_t)t.rows + 1) * 4);
+  a.col_idx = take((size_t)t.causal_blocks * 4);
+  a.nnz = take(8);
+  a.lse = take(T * s->num_q_heads * 4);
+  a.ws = take(gate_workspace_bytes(t, s));
+  a.total = p;
+  return a;
+}
+}  // namespace
+
+size_t seer_prefill_host_arena_bytes(const seer_shape* shape) {
+  ShapeTotals t;
+  if (shape_totals(shape, &t) != SEER_OK) return 0;
+  return arena_layout(shape, t).total;
+}
+
+seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void* q_host, const void* k_host,
+                              const void* v_host, const float* Wq_host, const float* Wk_host,
+                              const seer_mask_params* params, void* o_host, float* lse_host, void* arena,
+                              size_t arena_bytes, void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!ctx || !shape || !params) return SEER_ERR_INVALID_ARG;
+  ShapeTotals t;
+  seer_status st = shape_totals(shape, &t);
+  if (st != SEER_OK) return st;
+  if (t.total_blocks == 0) return SEER_OK;
+  if (!q_host || !k_host || !v_host || !Wq_host || !Wk_host || !o_host) return SEER_ERR_INVALID_ARG;
+  const ArenaLayout a = arena_layout(shape, t);
+  if (!ws_ok(arena, arena_bytes, a.total)) return SEER_ERR_WORKSPACE;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return SEER_ERR_CUDA;
+  char* d = (char*)arena;
+  const size_t T = (size_t)t.total_tokens;
+  const size_t qb = T * shape->num_q_heads * kHeadDim * 2, kb = T * shape->num_kv_heads * kHeadDim * 2;
+  bool ok = cudaMemcpyAsync(d + a.q, q_host, qb, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+            cudaMemcpyAsync(d + a.k, k_host, kb, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+            cudaMemcpyAsync(d + a.v, v_host, kb, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+            cudaMemcpyAsync(d + a.wq, Wq_host, (size_t)shape->num_q_heads * kHeadDim * kGateDim * 4,
+                            cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+            cudaMemcpyAsync(d + a.wk, Wk_host, (size_t)shape->num_kv_heads * kHeadDim * kGateDim * 4,
+                            cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (!ok) return SEER_ERR_CUDA;
+  st = seer_gate_scores(ctx, shape, d + a.q, d + a.k, (const float*)(d + a.wq), (const float*)(d + a.wk),
+                        (float*)(d + a.scores), d + a.ws, a.total - a.ws, stream);
+  if (st != SEER_OK) return st;
+  st = seer_block_mask(ctx, shape, (const float*)(d + a.scores), params, (int32_t*)(d + a.row_ptr),
+                       (int32_t*)(d + a.col_idx), t.causal_blocks, (int64_t*)(d + a.nnz), nullptr, 0, stream);
+  if (st != SEER_OK) return st;
+  st = seer_sparse_attn(ctx, shape, d + a.q, d + a.k, d + a.v, (const int32_t*)(d + a.row_ptr),
+                        (const int32_t*)(d + a.col_idx), d + a.o, lse_host ? (float*)(d + a.lse) : nullptr, nullptr, 0,
+                        stream);
+  if (st != SEER_OK) return st;
+  if (cudaMemcpyAsync(o_host, d + a.o, qb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SEER_ERR_CUDA;
+  if (lse_host &&
+      cudaMemcpyAsync(lse_host, d + a.lse, T * shape->num_q_heads * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return SEER_ERR_CUDA;
+  return SEER_OK;
+}
+
 }  // extern "C"

@@ -240,3 +240,28 @@ def make_small(seed: int, seqlens, hq: int, hkv: int, *, block: int = BLOCK, hea
     wk = (r.standard_normal((hkv, head_dim, gate_dim), dtype=np.float32) * np.float32(w_std))
     return Workload(f"small{seed}", cu, hq, hkv, f32_to_bf16_bits(q), f32_to_bf16_bits(k), f32_to_bf16_bits(v),
                     wq, wk, [], block=block, head_dim=head_dim, gate_dim=gate_dim)
+
+
+def sample_rows(cu_seqlens, num_q_heads: int, row_ptr: np.ndarray, seed: int, per_head_random: int = 8,
+                heads=None, block: int = BLOCK) -> np.ndarray:
+    """Stratified sample of mask rows for full-size checks: for every (sequence, head) the first two query
+    blocks, the last, the row with the longest list, the row with the shortest, and a few seeded-random ones.
+    Pure index selection; returns sorted unique row ids."""
+    lens = np.diff(np.asarray(cu_seqlens, dtype=np.int64))
+    nbs = (lens + block - 1) // block
+    counts = np.diff(np.asarray(row_ptr, dtype=np.int64))
+    rng = np.random.default_rng(seed)
+    out = []
+    base = 0
+    for nb in nbs:
+        nb = int(nb)
+        for h in (range(num_q_heads) if heads is None else heads):
+            if nb == 0:
+                continue
+            r0 = base + h * nb
+            c = counts[r0:r0 + nb]
+            picks = {0, min(1, nb - 1), nb - 1, int(np.argmax(c)), int(np.argmin(c))}
+            picks |= set(rng.integers(0, nb, size=per_head_random).tolist())
+            out.extend(r0 + i for i in picks)
+        base += num_q_heads * nb
+    return np.unique(np.asarray(out, dtype=np.int64))

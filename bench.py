@@ -39,6 +39,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--keep", default="1/10", help="TopK ratio for the c3 workload")
+    ap.add_argument("--seq", type=int, default=None, help="override the sequence length (profiling on a smaller case)")
     ap.add_argument("--attn-impl", type=int, default=0, help="0 tcgen05 kernel, 1 mma.sync cross-check kernel")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-list run of the attention kernel")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
@@ -137,7 +138,7 @@ def run_reference(args):
         return
     from oracle import seer_oracle as O
     from paper_2410_13276_b200 import workloads as W
-    w = W.make_workload(args.workload)
+    w = W.make_workload(args.workload, seq=args.seq)
     spec = pick_mask(w, args)
     # lists for the sampled rows come from the oracle's own gate + mask on a slice of heads would take minutes at
     # this size; the sample uses TopK lists of seeded random scores with the same keep ratio instead (same row lengths).
@@ -217,7 +218,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # every rank runs the same layer on its own GPU: shards are independent (no data-path collective) -> weak scaling
-    w = W.make_workload(args.workload)
+    w = W.make_workload(args.workload, seq=args.seq)
     spec = pick_mask(w, args)
     p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, device=local, want_lse=False)
     B.seer_set_attn_impl(p.ctx, args.attn_impl)

@@ -14,8 +14,10 @@
 // work group computes exact column maxima, rebases m, rescales its partial sums and the O accumulator, and recomputes
 // the tile.  Row sums are per-thread partials combined once per work item.
 //
-// Roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2-5 = softmax / correction /
-// epilogue.  One persistent CTA per SM walks the work items (longest rows first within each KV head).
+// Roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2-5 and 6-9 = two softmax
+// groups.  The tiles of a work item alternate between the groups (even tiles -> A, odd -> B); each group keeps its own
+// S^T buffers, P^T buffer, O^T accumulator, references and row sums, and the epilogue merges the two partial results
+// through their references.  One persistent CTA per SM walks the work items (longest rows first within each KV head).
 // Every wait is bounded; a wait that runs out raises SEER_ERR_TIMEOUT and the CTA drains and exits.
 #include <cuda.h>
 #include <math_constants.h>
@@ -27,35 +29,33 @@
 namespace seer {
 namespace tc {
 
-constexpr int kThreads = 192;
-constexpr int kSoftmaxThreads = 128;
-constexpr int kStages = 2;
+constexpr int kThreads = 320;               // warp 0 producer, warp 1 MMA issuer, warps 2-5 / 6-9 softmax groups A / B
+constexpr int kGroupThreads = 128;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
 constexpr uint32_t kQBytes = 2 * kHalfQ;         // 16 KB
-constexpr uint32_t kKVBytes = 2 * kHalfKV;       // 32 KB (K or V of one stage)
+constexpr uint32_t kKVBytes = 2 * kHalfKV;       // 32 KB (K or V tile of 128 keys)
 constexpr uint32_t kPBytes = 128 * 128;          // 16 KB  P^T [128 keys][64 q] bf16
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffK = kOffQ + kQBytes;                       // kStages x 32 KB
-constexpr uint32_t kOffV = kOffK + kStages * kKVBytes;            // kStages x 32 KB
-constexpr uint32_t kOffP = kOffV + kStages * kKVBytes;            // 16 KB (also epilogue staging)
-constexpr uint32_t kOffRed = kOffP + kPBytes;                     // 128 x 65 floats for the row-sum reduction
-constexpr uint32_t kRedBytes = 128 * 65 * 4;
-constexpr uint32_t kOffMref = kOffRed + kRedBytes;                // 64 floats
-constexpr uint32_t kOffAlpha = kOffMref + 256;                    // 64 floats
-constexpr uint32_t kOffColmax = kOffAlpha + 256;                  // 64 ints
-constexpr uint32_t kOffInvL = kOffColmax + 256;                   // 64 floats
-constexpr uint32_t kOffBar = kOffInvL + 256;                      // mbarriers
-constexpr uint32_t kNumBars = 16;
+constexpr uint32_t kOffQ = 0;                                     // 2 x 16 KB (items alternate)
+constexpr uint32_t kOffK = kOffQ + 2 * kQBytes;                   // 2 x 32 KB ring
+constexpr uint32_t kOffV = kOffK + 2 * kKVBytes;                  // 2 x 32 KB ring
+constexpr uint32_t kOffP = kOffV + 2 * kKVBytes;                  // 2 x 16 KB, one per softmax group (also epilogue staging)
+constexpr uint32_t kOffGrp = kOffP + 2 * kPBytes;                 // per-group small arrays
+constexpr uint32_t kGrpMref = 0, kGrpAlpha = 256, kGrpColmax = 512, kGrpLfin = 768, kGrpLsum = 1024;   // lsum: 4 x 64 floats
+constexpr uint32_t kGrpBytes = 2048;
+constexpr uint32_t kOffW = kOffGrp + 2 * kGrpBytes;               // merge weights wA[64], wB[64]
+constexpr uint32_t kOffBar = kOffW + 512;                         // mbarriers
+constexpr uint32_t kNumBars = 24;
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag
 constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;             // + alignment slack
 
-enum Bar { Q_FULL = 0, Q_EMPTY, KV_FULL0, KV_FULL1, KV_EMPTY0, KV_EMPTY1, S_FULL0, S_FULL1, S_EMPTY0, S_EMPTY1,
-           P_FULL, PV_DONE };
+enum Bar { Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 6, V_FULL = 8, V_EMPTY = 10, S_FULL = 12 /* + 2*group + buf */,
+           S_EMPTY = 16, P_FULL = 20 /* + group */, PV_DONE = 22 };
 
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS0 = 0, kColS1 = 64, kColO = 128;
+constexpr uint32_t kTmemCols = 512;
+__device__ __forceinline__ uint32_t col_s(int group, uint32_t buf) { return (uint32_t)group * 192u + buf * 64u; }
+__device__ __forceinline__ uint32_t col_o(int group) { return (uint32_t)group * 192u + 128u; }
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is declared lost
 
@@ -145,6 +145,13 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
                  "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Same wait, with the loaded registers as in/out operands so that no use of them can be scheduled above it.
+__device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void named_bar_sync(int id, int threads) {
@@ -188,13 +195,6 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-// Wait used by the 128 softmax threads: all of them wait, then agree on the outcome, so that after a lost wait
-// nobody is left behind at a named barrier.
-__device__ __forceinline__ bool wg_wait(const Shared& sh, int bar, uint32_t parity, int* status) {
-  const bool fail = !mbar_wait(sh, bar, parity, status);
-  return !named_bar_or(3, kSoftmaxThreads, fail);
-}
-
 struct Item {
   int b, h, g, i, nb, s0, slen, l0, nlist, ntiles, q_valid;
   int64_t row;
@@ -219,11 +219,130 @@ __device__ __forceinline__ Item decode_item(const SeqMeta& m, const int32_t* __r
   return it;
 }
 
-// Block index of list position p of an item, or -1 when the position is past the list or the entry is out of range.
+// Block index of list position p of an item: -1 past the end of the list, -2 for an entry outside [0, i].
 __device__ __forceinline__ int list_block(const Item& it, const int32_t* __restrict__ col_idx, int p) {
   if (p >= it.nlist) return -1;
   const int j = col_idx[it.l0 + p];
   return (j < 0 || j > it.i) ? -2 : j;
+}
+
+// Walks the tiles of this CTA's work items in order.  The producer and the MMA issuer each keep cursors of their
+// own; they see the same sequence because it depends only on the lists.
+struct Cursor {
+  int64_t w;
+  Item it;
+  int t;             // tile within the item
+  uint32_t k;        // ordinal of the item among this CTA's non-empty items
+  uint32_t g;        // ordinal of the tile among all tiles of this CTA
+  uint32_t cnt[2];   // tiles handed to softmax group 0 / 1 so far
+  bool valid;
+};
+__device__ __forceinline__ void cursor_seek(Cursor& c, const SeqMeta& m, const int32_t* __restrict__ row_ptr) {
+  c.valid = false;
+  while (c.w < m.rows) {
+    c.it = decode_item(m, row_ptr, c.w);
+    if (c.it.ntiles > 0) { c.valid = true; return; }
+    c.w += gridDim.x;
+  }
+}
+__device__ __forceinline__ void cursor_init(Cursor& c, const SeqMeta& m, const int32_t* __restrict__ row_ptr) {
+  c.w = blockIdx.x; c.t = 0; c.k = 0; c.g = 0; c.cnt[0] = c.cnt[1] = 0;
+  cursor_seek(c, m, row_ptr);
+}
+__device__ __forceinline__ void cursor_next(Cursor& c, const SeqMeta& m, const int32_t* __restrict__ row_ptr) {
+  c.cnt[c.t & 1] += 1;
+  c.g += 1;
+  if (++c.t >= c.it.ntiles) {
+    c.t = 0; c.k += 1; c.w += gridDim.x;
+    cursor_seek(c, m, row_ptr);
+  }
+}
+
+// One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]), packed to bf16 pairs.
+// Returns the largest exponent seen.  MASKED applies the causal mask of a diagonal block / drops a dead row.
+template <bool MASKED>
+__device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __restrict__ mref, float sl2, bool row_live,
+                                              bool diag, int key_local, uint32_t (&pk)[32]) {
+  float xmax = -CUDART_INF_F;
+  uint32_t sv[2][16];
+  tc_ld16(s_addr, sv[0]);
+#pragma unroll
+  for (int ch = 0; ch < 4; ++ch) {
+    tc_wait_ld(sv[ch & 1]);
+    if (ch < 3) tc_ld16(s_addr + (ch + 1) * 16, sv[(ch + 1) & 1]);
+#pragma unroll
+    for (int e = 0; e < 16; e += 4) {
+      const int c = ch * 16 + e;
+      const float4 mr = *reinterpret_cast<const float4*>(&mref[c]);
+      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -mr.x);
+      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -mr.y);
+      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -mr.z);
+      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -mr.w);
+      if (MASKED) {
+        if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
+        if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
+        if (!row_live || (diag && key_local > c + 2)) x2 = -CUDART_INF_F;
+        if (!row_live || (diag && key_local > c + 3)) x3 = -CUDART_INF_F;
+      }
+      xmax = fmaxf(xmax, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
+      pk[c >> 1] = pack_bf16(ex2f(x0), ex2f(x1));
+      pk[(c >> 1) + 1] = pack_bf16(ex2f(x2), ex2f(x3));
+    }
+  }
+  return xmax;
+}
+
+// Sums l[0..63] over the 32 lanes of a warp; lane ends with the totals of columns (2*bitrev-ish) base, base+1
+// where base = 32*b4 + 16*b3 + 8*b2 + 4*b1 + 2*b0 (b_i = bit i of the lane id).
+__device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out0, float& out1, int& base) {
+  float a[32];
+  {
+    const bool up = (lane & 16) != 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float send = up ? l[i] : l[i + 32];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
+      a[i] = (up ? l[i + 32] : l[i]) + recv;
+    }
+  }
+  float b[16];
+  {
+    const bool up = (lane & 8) != 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float send = up ? a[i] : a[i + 16];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, 8);
+      b[i] = (up ? a[i + 16] : a[i]) + recv;
+    }
+  }
+  float c[8];
+  {
+    const bool up = (lane & 4) != 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float send = up ? b[i] : b[i + 8];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, 4);
+      c[i] = (up ? b[i + 8] : b[i]) + recv;
+    }
+  }
+  float d[4];
+  {
+    const bool up = (lane & 2) != 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float send = up ? c[i] : c[i + 4];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, 2);
+      d[i] = (up ? c[i + 4] : c[i]) + recv;
+    }
+  }
+  {
+    const bool up = (lane & 1) != 0;
+    const float s0 = up ? d[0] : d[2], s1 = up ? d[1] : d[3];
+    const float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+    out0 = (up ? d[2] : d[0]) + r0;
+    out1 = (up ? d[3] : d[1]) + r1;
+  }
+  base = ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
 }
 
 // ------------------------------------------------------------------------------------------------ kernel
@@ -240,16 +359,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
 
   if (threadIdx.x == 0) {
-    mbar_init(sh.bar(Q_FULL), 1);
-    mbar_init(sh.bar(Q_EMPTY), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(sh.bar(KV_FULL0 + s), 1);
-      mbar_init(sh.bar(KV_EMPTY0 + s), 1);
-      mbar_init(sh.bar(S_FULL0 + s), 1);
-      mbar_init(sh.bar(S_EMPTY0 + s), kSoftmaxThreads);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(sh.bar(Q_FULL + i), 1);
+      mbar_init(sh.bar(Q_EMPTY + i), 1);
+      mbar_init(sh.bar(K_FULL + i), 1);
+      mbar_init(sh.bar(K_EMPTY + i), 1);
+      mbar_init(sh.bar(V_FULL + i), 1);
+      mbar_init(sh.bar(V_EMPTY + i), 1);
+      mbar_init(sh.bar(P_FULL + i), kGroupThreads);
+      mbar_init(sh.bar(PV_DONE + i), 1);
     }
-    mbar_init(sh.bar(P_FULL), kSoftmaxThreads);
-    mbar_init(sh.bar(PV_DONE), 1);
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(sh.bar(S_FULL + i), 1);
+      mbar_init(sh.bar(S_EMPTY + i), kGroupThreads);
+    }
     st_shared_u32(sh.abort_flag(), 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -265,163 +388,180 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // ============================================================================================ producer
   if (warp == 0) {
     if (lane == 0) {
-      uint32_t n_item = 0, n_tile = 0;
-      for (int64_t w = blockIdx.x; w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
-        if (it.ntiles == 0) continue;   // empty list: nothing to load; only items with tiles advance n_item
-        if (!mbar_wait(sh, Q_EMPTY, (n_item & 1u) ^ 1u, status)) break;
-        ++n_item;
-        mbar_expect_tx(sh.bar(Q_FULL), kQBytes);
-        const int tq = it.s0 + it.i * kBlock;
-        tma_load_3d(sh.base + kOffQ, &map_q, sh.bar(Q_FULL), 0, it.h, tq);
-        tma_load_3d(sh.base + kOffQ + kHalfQ, &map_q, sh.bar(Q_FULL), 64, it.h, tq);
-        bool ok = true;
-        for (int t = 0; t < it.ntiles; ++t, ++n_tile) {
-          const uint32_t st = n_tile & 1u;
-          if (!mbar_wait(sh, KV_EMPTY0 + st, ((n_tile >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
-          int ja = list_block(it, col_idx, 2 * t), jb = list_block(it, col_idx, 2 * t + 1);
-          if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
-          const bool has_b = jb != -1;
-          if (ja < 0) ja = 0;            // a rejected entry is replaced by block 0 and masked out in the softmax
-          if (jb < 0) jb = 0;
-          mbar_expect_tx(sh.bar(KV_FULL0 + st), has_b ? 2 * kKVBytes : kKVBytes);
-          const uint32_t kdst = sh.base + kOffK + st * kKVBytes, vdst = sh.base + kOffV + st * kKVBytes;
-          const uint32_t fb = sh.bar(KV_FULL0 + st);
-          const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
-          tma_load_3d(kdst, &map_k, fb, 0, it.g, ta);
-          tma_load_3d(kdst + kHalfKV, &map_k, fb, 64, it.g, ta);
-          if (has_b) {
-            tma_load_3d(kdst + kHalfQ, &map_k, fb, 0, it.g, tb);
-            tma_load_3d(kdst + kHalfKV + kHalfQ, &map_k, fb, 64, it.g, tb);
-          }
-          tma_load_3d(vdst, &map_v, fb, 0, it.g, ta);
-          tma_load_3d(vdst + kHalfKV, &map_v, fb, 64, it.g, ta);
-          if (has_b) {
-            tma_load_3d(vdst + kHalfQ, &map_v, fb, 0, it.g, tb);
-            tma_load_3d(vdst + kHalfKV + kHalfQ, &map_v, fb, 64, it.g, tb);
-          }
+      Cursor kc, vc;                       // K runs one tile ahead of V
+      cursor_init(kc, m, row_ptr);
+      vc = kc;
+      auto load_k = [&](const Cursor& c) -> bool {
+        const Item& it = c.it;
+        if (c.t == 0) {                    // first tile of an item: its Q block
+          const uint32_t qb = c.k & 1u;
+          if (!mbar_wait(sh, Q_EMPTY + qb, ((c.k >> 1) & 1u) ^ 1u, status)) return false;
+          mbar_expect_tx(sh.bar(Q_FULL + qb), kQBytes);
+          const int tq = it.s0 + it.i * kBlock;
+          tma_load_3d(sh.base + kOffQ + qb * kQBytes, &map_q, sh.bar(Q_FULL + qb), 0, it.h, tq);
+          tma_load_3d(sh.base + kOffQ + qb * kQBytes + kHalfQ, &map_q, sh.bar(Q_FULL + qb), 64, it.h, tq);
         }
-        if (!ok) break;
+        int ja = list_block(it, col_idx, 2 * c.t), jb = list_block(it, col_idx, 2 * c.t + 1);
+        if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
+        const bool has_b = jb != -1;
+        if (ja < 0) ja = 0;                // a rejected entry is replaced by block 0 and masked out in the softmax
+        if (jb < 0) jb = 0;
+        const uint32_t st = c.g & 1u;
+        if (!mbar_wait(sh, K_EMPTY + st, ((c.g >> 1) & 1u) ^ 1u, status)) return false;
+        const uint32_t fb = sh.bar(K_FULL + st), dst = sh.base + kOffK + st * kKVBytes;
+        mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
+        const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
+        tma_load_3d(dst, &map_k, fb, 0, it.g, ta);
+        tma_load_3d(dst + kHalfKV, &map_k, fb, 64, it.g, ta);
+        if (has_b) {
+          tma_load_3d(dst + kHalfQ, &map_k, fb, 0, it.g, tb);
+          tma_load_3d(dst + kHalfKV + kHalfQ, &map_k, fb, 64, it.g, tb);
+        }
+        return true;
+      };
+      auto load_v = [&](const Cursor& c) -> bool {
+        const Item& it = c.it;
+        int ja = list_block(it, col_idx, 2 * c.t), jb = list_block(it, col_idx, 2 * c.t + 1);
+        const bool has_b = jb != -1;
+        if (ja < 0) ja = 0;
+        if (jb < 0) jb = 0;
+        const uint32_t st = c.g & 1u;
+        if (!mbar_wait(sh, V_EMPTY + st, ((c.g >> 1) & 1u) ^ 1u, status)) return false;
+        const uint32_t fb = sh.bar(V_FULL + st), dst = sh.base + kOffV + st * kKVBytes;
+        mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
+        const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
+        tma_load_3d(dst, &map_v, fb, 0, it.g, ta);
+        tma_load_3d(dst + kHalfKV, &map_v, fb, 64, it.g, ta);
+        if (has_b) {
+          tma_load_3d(dst + kHalfQ, &map_v, fb, 0, it.g, tb);
+          tma_load_3d(dst + kHalfKV + kHalfQ, &map_v, fb, 64, it.g, tb);
+        }
+        return true;
+      };
+      bool ok = true;
+      if (kc.valid) { ok = load_k(kc); cursor_next(kc, m, row_ptr); }
+      while (ok && vc.valid) {
+        if (kc.valid) { ok = load_k(kc); cursor_next(kc, m, row_ptr); }
+        if (ok) { ok = load_v(vc); cursor_next(vc, m, row_ptr); }
       }
     }
   }
   // ============================================================================================ MMA issuer
   else if (warp == 1) {
     if (lane == 0) {
-      uint32_t n_item = 0, n_tile = 0;
-      const uint32_t q_addr = sh.base + kOffQ;
-      auto issue_s = [&](uint32_t n) -> bool {       // S^T(n) = K_tile * Q^T into S buffer n & 1
-        const uint32_t st = n & 1u, use = n >> 1;
-        if (!mbar_wait(sh, KV_FULL0 + st, use & 1u, status)) return false;
-        if (!mbar_wait(sh, S_EMPTY0 + st, (use & 1u) ^ 1u, status)) return false;
+      Cursor sc, pc;                       // S^T issue runs up to three tiles ahead of P V issue
+      cursor_init(sc, m, row_ptr);
+      pc = sc;
+      auto issue_s = [&](const Cursor& c) -> bool {
+        const int grp = c.t & 1;
+        const uint32_t cn = c.cnt[grp], buf = cn & 1u, st = c.g & 1u, qb = c.k & 1u;
+        if (c.t == 0 && !mbar_wait(sh, Q_FULL + qb, (c.k >> 1) & 1u, status)) return false;
+        if (!mbar_wait(sh, K_FULL + st, (c.g >> 1) & 1u, status)) return false;
+        if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) return false;
         tc_fence_after();
-        const uint32_t k_addr = sh.base + kOffK + st * kKVBytes;
+        const uint32_t k_addr = sh.base + kOffK + st * kKVBytes, q_addr = sh.base + kOffQ + qb * kQBytes;
+        const uint32_t d = tmem + col_s(grp, buf);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint64_t a = make_desc(k_addr + (kk >> 2) * kHalfKV + (kk & 3) * 32, 16, 1024);
           const uint64_t b = make_desc(q_addr + (kk >> 2) * kHalfQ + (kk & 3) * 32, 16, 1024);
-          tc_mma(tmem + (st ? kColS1 : kColS0), a, b, kIdescS, kk > 0);
+          tc_mma(d, a, b, kIdescS, kk > 0);
         }
-        tc_commit(sh.bar(S_FULL0 + st));
+        tc_commit(sh.bar(S_FULL + 2 * grp + buf));
+        tc_commit(sh.bar(K_EMPTY + st));
+        if (c.t == c.it.ntiles - 1) tc_commit(sh.bar(Q_EMPTY + qb));   // last S^T of the item: Q may be replaced
+        return true;
+      };
+      auto issue_pv = [&](const Cursor& c) -> bool {
+        const int grp = c.t & 1;
+        const uint32_t cn = c.cnt[grp], st = c.g & 1u;
+        if (!mbar_wait(sh, V_FULL + st, (c.g >> 1) & 1u, status)) return false;
+        if (!mbar_wait(sh, P_FULL + grp, cn & 1u, status)) return false;
+        tc_fence_after();
+        const uint32_t v_addr = sh.base + kOffV + st * kKVBytes, p_addr = sh.base + kOffP + grp * kPBytes;
+        const int nk = (2 * c.t + 1 < c.it.nlist) ? 8 : 4;       // 16-key groups to contract over
+        const uint32_t d = tmem + col_o(grp);
+        for (int kk = 0; kk < nk; ++kk) {
+          const uint64_t a = make_desc(v_addr + kk * 2048, kHalfKV, 1024);
+          const uint64_t b = make_desc(p_addr + kk * 2048, kHalfKV, 1024);
+          tc_mma(d, a, b, kIdescPV, (c.t >= 2 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(sh.bar(V_EMPTY + st));
+        tc_commit(sh.bar(PV_DONE + grp));
         return true;
       };
       bool ok = true;
-      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
-        if (it.ntiles == 0) continue;
-        if (!mbar_wait(sh, Q_FULL, n_item & 1u, status)) break;
-        ++n_item;
-        if (!issue_s(n_tile)) break;
-        for (int t = 0; t < it.ntiles; ++t) {
-          const uint32_t n = n_tile + t;
-          if (t + 1 < it.ntiles) {
-            if (!issue_s(n + 1)) { ok = false; break; }
-          } else {
-            tc_commit(sh.bar(Q_EMPTY));      // every S^T of this item has been issued: Q may be replaced once they finish
-          }
-          if (!mbar_wait(sh, P_FULL, n & 1u, status)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t st = n & 1u;
-          const uint32_t v_addr = sh.base + kOffV + st * kKVBytes, p_addr = sh.base + kOffP;
-          const int nk = list_block(it, col_idx, 2 * t + 1) != -1 ? 8 : 4;   // 16-key groups to contract over
-          for (int kk = 0; kk < nk; ++kk) {
-            const uint64_t a = make_desc(v_addr + kk * 2048, kHalfKV, 1024);
-            const uint64_t b = make_desc(p_addr + kk * 2048, kHalfKV, 1024);
-            tc_mma(tmem + kColO, a, b, kIdescPV, (t > 0 || kk > 0) ? 1u : 0u);
-          }
-          tc_commit(sh.bar(KV_EMPTY0 + st));
-          tc_commit(sh.bar(PV_DONE));
-        }
-        n_tile += it.ntiles;
+      while (ok && pc.valid) {
+        while (ok && sc.valid && sc.g < pc.g + 3) { ok = issue_s(sc); cursor_next(sc, m, row_ptr); }
+        if (ok) { ok = issue_pv(pc); cursor_next(pc, m, row_ptr); }
       }
     }
   }
-  // ============================================================================================ softmax work group
+  // ============================================================================================ softmax groups
   else {
-    const int wg_tid = threadIdx.x - 64;                 // 0..127
+    const int grp = (warp - 2) >> 2;                     // 0 = A (even tiles), 1 = B (odd tiles)
+    const int gt = threadIdx.x - 64 - grp * kGroupThreads;   // 0..127 within the group
+    const int gw = (warp - 2) & 3;                       // warp within the group
     const int quad = warp & 3;                           // TMEM lane quadrant this warp may access
     const int r = quad * 32 + lane;                      // key row of S^T / d row of O^T owned by this thread
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    float* mref = reinterpret_cast<float*>(smem + kOffMref);
-    float* alpha = reinterpret_cast<float*>(smem + kOffAlpha);
-    int* colmax = reinterpret_cast<int*>(smem + kOffColmax);
-    float* inv_l = reinterpret_cast<float*>(smem + kOffInvL);
-    float* red = reinterpret_cast<float*>(smem + kOffRed);
+    unsigned char* gsm = smem + kOffGrp + grp * kGrpBytes;
+    float* mref = reinterpret_cast<float*>(gsm + kGrpMref);
+    float* alpha = reinterpret_cast<float*>(gsm + kGrpAlpha);
+    int* colmax = reinterpret_cast<int*>(gsm + kGrpColmax);
+    float* lfin = reinterpret_cast<float*>(gsm + kGrpLfin);
+    float* lsum = reinterpret_cast<float*>(gsm + kGrpLsum);
+    float* w_a = reinterpret_cast<float*>(smem + kOffW);
+    float* w_b = w_a + 64;
+    const float* mref_a = reinterpret_cast<const float*>(smem + kOffGrp + kGrpMref);
+    const float* mref_b = reinterpret_cast<const float*>(smem + kOffGrp + kGrpBytes + kGrpMref);
+    const float* lfin_a = reinterpret_cast<const float*>(smem + kOffGrp + kGrpLfin);
+    const float* lfin_b = reinterpret_cast<const float*>(smem + kOffGrp + kGrpBytes + kGrpLfin);
+    const int bar_sync = 1 + grp, bar_vote = 3 + grp;
     const float sl2 = m.softmax_scale * 1.4426950408889634f;
-    uint32_t n_tile = 0;
+    const int key_local = r & 63;
+    uint32_t cnt = 0;                                    // tiles this group has processed
+    uint32_t gbase = 0;                                  // tiles of this CTA before the current item
     bool ok = true;
 
-    for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+    for (int64_t w = blockIdx.x; w < m.rows; w += gridDim.x) {
       const Item it = decode_item(m, row_ptr, w);
       const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock;
+      const int tiles_a = (it.ntiles + 1) >> 1, tiles_b = it.ntiles >> 1;
+      const int my_tiles = grp == 0 ? tiles_a : tiles_b;
       float l_part[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) l_part[c] = 0.f;
-      if (wg_tid < 64) mref[wg_tid] = -CUDART_INF_F;
-      named_bar_sync(1, kSoftmaxThreads);
+      if (gt < 64) mref[gt] = -CUDART_INF_F;
+      named_bar_sync(bar_sync, kGroupThreads);
 
-      for (int t = 0; t < it.ntiles && ok; ++t, ++n_tile) {
-        const uint32_t st = n_tile & 1u;
+      for (int t = grp; t < it.ntiles; t += 2, ++cnt) {
+        const uint32_t sbuf = cnt & 1u;
+        bool fail = !mbar_wait(sh, S_FULL + 2 * grp + sbuf, (cnt >> 1) & 1u, status);
+        // the previous P V of this group has finished: its P^T buffer and the O^T accumulator may be touched
+        if (!fail && cnt > 0) fail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
+        tc_fence_after();
         const int ja = list_block(it, col_idx, 2 * t), jb = list_block(it, col_idx, 2 * t + 1);
         const int my_j = r < 64 ? ja : jb;
         const bool row_live = my_j >= 0;                 // absent / rejected blocks contribute nothing
         const bool diag = my_j == it.i;
-        const int key_local = r & 63;
-        if (!wg_wait(sh, S_FULL0 + st, (n_tile >> 1) & 1u, status)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t s_addr = tmem + lane_addr + (st ? kColS1 : kColS0);
-
+        const bool masked = !row_live || diag;           // uniform per warp (a warp lies in one block half)
+        const uint32_t s_addr = tmem + lane_addr + col_s(grp, sbuf);
         uint32_t pk[32];
-        for (int pass = 0; pass < 2; ++pass) {
-          float xmax = -CUDART_INF_F;
+        float xmax = -CUDART_INF_F;
+        if (!fail) xmax = masked ? softmax_pass<true>(s_addr, mref, sl2, row_live, diag, key_local, pk)
+                                 : softmax_pass<false>(s_addr, mref, sl2, row_live, diag, key_local, pk);
+        // one vote per tile: does any entry exceed its reference by more than 2^8 (or has a wait been lost)?
+        if (named_bar_or(bar_vote, kGroupThreads, fail || xmax > 8.f)) {
+          if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
+          // ---- exact column maxima of this tile -> new references, rescale partial sums and O^T, recompute the tile
+          if (gt < 64) colmax[gt] = float_order_int(-CUDART_INF_F);
+          named_bar_sync(bar_sync, kGroupThreads);
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t sv[16];
             tc_ld16(s_addr + ch * 16, sv);
-            tc_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 16; e += 2) {
-              const int c = ch * 16 + e;
-              const float2 mr = *reinterpret_cast<const float2*>(&mref[c]);
-              float x0 = fmaf(__uint_as_float(sv[e]), sl2, -mr.x);
-              float x1 = fmaf(__uint_as_float(sv[e + 1]), sl2, -mr.y);
-              if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
-              if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
-              xmax = fmaxf(xmax, fmaxf(x0, x1));
-              pk[c >> 1] = pack_bf16(ex2f(fminf(x0, 64.f)), ex2f(fminf(x1, 64.f)));
-            }
-          }
-          // does any entry of the tile exceed its reference by more than 2^8?
-          const bool rebase = named_bar_or(2, kSoftmaxThreads, xmax > 8.f);
-          if (!rebase) break;
-          // ---- exact column maxima of this tile, then new references (pass 1 recomputes the tile with them)
-          if (wg_tid < 64) colmax[wg_tid] = float_order_int(-CUDART_INF_F);
-          named_bar_sync(1, kSoftmaxThreads);
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t sv[16];
-            tc_ld16(s_addr + ch * 16, sv);
-            tc_wait_ld();
+            tc_wait_ld(sv);
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
               const int c = ch * 16 + e;
@@ -431,47 +571,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
               if (lane == 0) atomicMax(&colmax[c], wm);
             }
           }
-          named_bar_sync(1, kSoftmaxThreads);
-          if (wg_tid < 64) {
-            const float old = mref[wg_tid];
-            float nm = fmaxf(old, order_int_float(colmax[wg_tid]));
+          named_bar_sync(bar_sync, kGroupThreads);
+          if (gt < 64) {
+            const float old = mref[gt];
+            float nm = fmaxf(old, order_int_float(colmax[gt]));
             if (nm == -CUDART_INF_F) nm = 0.f;           // nothing visible in this column yet
-            alpha[wg_tid] = old == -CUDART_INF_F ? 0.f : exp2f(old - nm);
-            mref[wg_tid] = nm;
+            alpha[gt] = old == -CUDART_INF_F ? 0.f : exp2f(old - nm);
+            mref[gt] = nm;
           }
-          named_bar_sync(1, kSoftmaxThreads);
+          named_bar_sync(bar_sync, kGroupThreads);
 #pragma unroll
           for (int c = 0; c < 64; ++c) l_part[c] *= alpha[c];
-          if (t > 0) {
-            // O^T row r of this thread: scale column c by alpha[c].  The previous tile's P V must have finished.
-            if (!wg_wait(sh, PV_DONE, (n_tile - 1) & 1u, status)) { ok = false; break; }
-            tc_fence_after();
+          if (t >= 2) {                                  // this group already accumulated into O^T for this item
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
               uint32_t ov[16];
-              tc_ld16(tmem + lane_addr + kColO + ch * 16, ov);
-              tc_wait_ld();
+              tc_ld16(tmem + lane_addr + col_o(grp) + ch * 16, ov);
+              tc_wait_ld(ov);
 #pragma unroll
               for (int e = 0; e < 16; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha[ch * 16 + e]);
-              tc_st16(tmem + lane_addr + kColO + ch * 16, ov);
+              tc_st16(tmem + lane_addr + col_o(grp) + ch * 16, ov);
             }
             tc_wait_st();
           }
+          if (masked) softmax_pass<true>(s_addr, mref, sl2, row_live, diag, key_local, pk);
+          else softmax_pass<false>(s_addr, mref, sl2, row_live, diag, key_local, pk);
         }
-        if (!ok) break;
-        // S^T buffer may be overwritten by the MMA of tile n + 2
+        // the S^T buffer may be overwritten by a later tile
         tc_fence_before();
-        mbar_arrive(sh.bar(S_EMPTY0 + st));
+        mbar_arrive(sh.bar(S_EMPTY + 2 * grp + sbuf));
         // row sums over the bf16-rounded probabilities the MMA will use
 #pragma unroll
         for (int c2 = 0; c2 < 32; ++c2) {
           l_part[2 * c2] += __uint_as_float(pk[c2] << 16);
           l_part[2 * c2 + 1] += __uint_as_float(pk[c2] & 0xffff0000u);
         }
-        // P^T row r -> shared memory (128-byte swizzle), after the previous P V has finished reading the buffer
-        if (n_tile > 0 && !wg_wait(sh, PV_DONE, (n_tile - 1) & 1u, status)) { ok = false; break; }
+        // P^T row r -> shared memory (128-byte swizzle)
         {
-          const uint32_t prow = sh.base + kOffP + (uint32_t)r * 128u;
+          const uint32_t prow = sh.base + kOffP + grp * kPBytes + (uint32_t)r * 128u;
 #pragma unroll
           for (int ck = 0; ck < 8; ++ck) {
             const uint32_t a = prow + (uint32_t)((ck ^ (r & 7)) << 4);
@@ -480,7 +617,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
           // ragged last block of a sequence: its V rows past the end belong to someone else -> zero them (0 * x must be 0)
           if (row_live && my_j * kBlock + key_local >= it.slen) {
-            const uint32_t vrow = sh.base + kOffV + st * kKVBytes + (uint32_t)r * 128u;
+            const uint32_t g = gbase + (uint32_t)t, vs = g & 1u;      // ring slot of this tile's V
+            mbar_wait(sh, V_FULL + vs, (g >> 1) & 1u, status);        // the copy has landed (a lost wait raises the abort flag)
+            const uint32_t vrow = sh.base + kOffV + vs * kKVBytes + (uint32_t)r * 128u;
 #pragma unroll
             for (int ck = 0; ck < 8; ++ck) {
               asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vrow + ck * 16), "r"(0u) : "memory");
@@ -490,60 +629,70 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         fence_async_smem();
         tc_fence_before();
-        mbar_arrive(sh.bar(P_FULL));
+        mbar_arrive(sh.bar(P_FULL + grp));
       }
-      if (!ok) break;
+
+      gbase += (uint32_t)it.ntiles;
 
       // ------------------------------------------------------------------------------------------ epilogue
-      if (it.ntiles > 0) {
-        if (!wg_wait(sh, PV_DONE, (n_tile - 1) & 1u, status)) { ok = false; break; }
-        tc_fence_after();
-      }
-      // combine the 128 partial row sums of each query column
-#pragma unroll
-      for (int c = 0; c < 64; ++c) red[r * 65 + c] = l_part[c];
-      named_bar_sync(1, kSoftmaxThreads);
-      if (wg_tid < 64) {
-        float l = 0.f;
-        for (int rr = 0; rr < 128; ++rr) l += red[rr * 65 + wg_tid];
-        inv_l[wg_tid] = l > 0.f ? 1.0f / l : 0.f;
-        if (lse != nullptr && wg_tid < it.q_valid)
-          lse[(int64_t)it.h * m.total_tokens + tok0 + wg_tid] =
-              l > 0.f ? (mref[wg_tid] + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
-      }
-      named_bar_sync(1, kSoftmaxThreads);
-      // O^T row r (d = r) -> staging [q][d] bf16 in the P buffer
+      bool efail = !ok;
+      if (ok && my_tiles > 0) efail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
+      tc_fence_after();
       {
-        uint16_t* stage = reinterpret_cast<uint16_t*>(smem + kOffP);
+        float s0, s1; int base;
+        warp_colsum(l_part, lane, s0, s1, base);
+        lsum[gw * 64 + base] = s0;
+        lsum[gw * 64 + base + 1] = s1;
+      }
+      named_bar_sync(bar_sync, kGroupThreads);
+      if (gt < 64) lfin[gt] = (lsum[gt] + lsum[64 + gt]) + (lsum[128 + gt] + lsum[192 + gt]);
+      // both groups: partial sums and references published, all P V of the item finished (or a wait was lost)
+      if (named_bar_or(5, 2 * kGroupThreads, efail)) { ok = false; break; }
+      if (grp == 0 && gt < 64) {
+        const float la = lfin_a[gt], lb = tiles_b > 0 ? lfin_b[gt] : 0.f;
+        const float ma = la > 0.f ? mref_a[gt] : -CUDART_INF_F, mb = lb > 0.f ? mref_b[gt] : -CUDART_INF_F;
+        const float mm = fmaxf(ma, mb);
+        float wa = 0.f, wb = 0.f, out_lse = -CUDART_INF_F;
+        if (mm != -CUDART_INF_F) {
+          const float fa = la > 0.f ? exp2f(ma - mm) : 0.f, fb = lb > 0.f ? exp2f(mb - mm) : 0.f;
+          const float l = la * fa + lb * fb;
+          wa = fa / l; wb = fb / l;
+          out_lse = (mm + log2f(l)) * 0.6931471805599453f;
+        }
+        w_a[gt] = wa; w_b[gt] = wb;
+        if (lse != nullptr && gt < it.q_valid) lse[(int64_t)it.h * m.total_tokens + tok0 + gt] = out_lse;
+      }
+      named_bar_sync(5, 2 * kGroupThreads);
+      // each group merges and stores 32 of the 64 query columns: staging [32 q][128 d] bf16 in its own P^T buffer
+      {
+        uint16_t* stage = reinterpret_cast<uint16_t*>(smem + kOffP + grp * kPBytes);
+        const int c0 = grp * 32;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t ov[16];
-          if (it.ntiles > 0) {
-            tc_ld16(tmem + lane_addr + kColO + ch * 16, ov);
-            tc_wait_ld();
-          } else {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) ov[e] = 0u;
-          }
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t oa[16], ob[16];
+          if (tiles_a > 0) { tc_ld16(tmem + lane_addr + col_o(0) + c0 + ch * 16, oa); tc_wait_ld(oa); }
+          if (tiles_b > 0) { tc_ld16(tmem + lane_addr + col_o(1) + c0 + ch * 16, ob); tc_wait_ld(ob); }
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const int c = ch * 16 + e;
-            const float val = it.ntiles > 0 ? __uint_as_float(ov[e]) * inv_l[c] : 0.f;
-            stage[c * 128 + r] = (uint16_t)(pack_bf16(val, 0.f) & 0xffffu);
+            const int c = c0 + ch * 16 + e;
+            float val = 0.f;
+            if (tiles_a > 0) val = __uint_as_float(oa[e]) * w_a[c];
+            if (tiles_b > 0) val = fmaf(__uint_as_float(ob[e]), w_b[c], val);
+            stage[(ch * 16 + e) * 128 + r] = (uint16_t)(pack_bf16(val, 0.f) & 0xffffu);
           }
         }
       }
       tc_fence_before();
-      named_bar_sync(1, kSoftmaxThreads);
+      named_bar_sync(5, 2 * kGroupThreads);   // every TMEM read of the item is done: the next item may overwrite O^T
       {
-        const uint4* stage4 = reinterpret_cast<const uint4*>(smem + kOffP);
-        for (int idx = wg_tid; idx < 64 * 16; idx += kSoftmaxThreads) {
-          const int qrow = idx >> 4, chunk = idx & 15;
+        const uint4* stage4 = reinterpret_cast<const uint4*>(smem + kOffP + grp * kPBytes);
+        for (int idx = gt; idx < 32 * 16; idx += kGroupThreads) {
+          const int qrow = grp * 32 + (idx >> 4), chunk = idx & 15;
           if (qrow < it.q_valid)
             *reinterpret_cast<uint4*>(o + ((tok0 + qrow) * m.num_q_heads + it.h) * kHeadDim + chunk * 8) = stage4[idx];
         }
       }
-      named_bar_sync(1, kSoftmaxThreads);   // staging buffer is free again before the next item's P
+      named_bar_sync(bar_sync, kGroupThreads);   // staging is free again before this group's next P^T
     }
   }
 

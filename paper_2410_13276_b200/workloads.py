@@ -194,7 +194,8 @@ WORKLOADS = ("c1", "c2", "c3", "c4", "c5", "c2s", "c3s", "c4s", "c5s")
 C3_RATIOS = ((1, 2), (1, 4), (1, 10), (1, 20))
 
 
-def make_workload(name: str) -> Workload:
+def make_workload(name: str, seq: Optional[int] = None) -> Workload:
+    """`seq` overrides the sequence length of the single-sequence workloads (c2, c3, c5) for profiling runs."""
     twin = name.endswith("s")
     config = int(name[1])
     if config == 1:
@@ -202,12 +203,12 @@ def make_workload(name: str) -> Workload:
         masks = [MaskSpec(MODE_TOPK_RATIO, 1, 2, flags=FORCE_DIAG)]
         hq, hkv = 4, 1
     elif config == 2:
-        S = 4096 if twin else 32768
+        S = seq or (4096 if twin else 32768)
         hq, hkv = 32, 8
         cu, q, k, v, wq, wk = _random_layer(2, twin, [S], hq, hkv, rope_base=500000.0)
         masks = [MaskSpec(MODE_THRESHOLD, flags=FORCE_DIAG, target_sparsity=0.90)]
     elif config == 3:
-        S = 4096 if twin else 131072
+        S = seq or (4096 if twin else 131072)
         hq, hkv = 32, 8
         cu, q, k, v, wq, wk = _random_layer(3, twin, [S], hq, hkv, rope_base=500000.0)
         masks = [MaskSpec(MODE_TOPK_RATIO, n, dn, flags=FORCE_DIAG | FORCE_SINK) for n, dn in C3_RATIOS]
@@ -217,7 +218,7 @@ def make_workload(name: str) -> Workload:
         cu, q, k, v, wq, wk = _random_layer(4, twin, lens, hq, hkv)
         masks = [MaskSpec(MODE_THRESHOLD, flags=FORCE_DIAG, target_sparsity=0.85)]
     elif config == 5:
-        S = 4096 if twin else 65536
+        S = seq or (4096 if twin else 65536)
         hq, hkv = 32, 8
         cu, q, k, v, wq, wk = _structured_layer(5, twin, S, hq, hkv)
         masks = [MaskSpec(MODE_THRESHOLD, flags=FORCE_DIAG, target_sparsity=0.92)]

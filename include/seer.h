@@ -140,6 +140,11 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
                               const seer_mask_params* params, void* o_host, float* lse_host, void* arena,
                               size_t arena_bytes, void* stream);
 
+/* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, CTA 0 of the tcgen05 attention kernel
+ * records a timeline of its pipeline roles into it: 6 roles x 4096 (tag << 32 | ordinal, SM clock) pairs of uint64, i.e.
+ * at least 6 * 8192 * 8 bytes of device memory, zero-initialised by the caller.  NULL switches it off (default). */
+seer_status seer_set_trace_buffer(seer_ctx* ctx, void* device_buffer);
+
 /* Number of kernels the library has launched through this context since creation (for launch accounting). */
 int64_t seer_launch_count(const seer_ctx* ctx);
 

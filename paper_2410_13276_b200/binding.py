@@ -25,7 +25,7 @@ STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER
 EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
            "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
-           "seer_prefill_host"]
+           "seer_prefill_host", "seer_set_trace_buffer"]
 
 
 class SeerError(RuntimeError):
@@ -90,6 +90,8 @@ def load_library() -> C.CDLL:
     lib.seer_prefill_host_arena_bytes.restype = sz
     lib.seer_prefill_host.argtypes = [vp, shp, vp, vp, vp, vp, vp, C.POINTER(seer_mask_params), vp, vp, vp, sz, vp]
     lib.seer_prefill_host.restype = C.c_int
+    lib.seer_set_trace_buffer.argtypes = [vp, vp]
+    lib.seer_set_trace_buffer.restype = C.c_int
     _lib = lib
     return lib
 
@@ -223,3 +225,7 @@ def seer_prefill_host(ctx: Context, shape: seer_shape, q_host, k_host, v_host, w
                                       _ptr(wq_host), _ptr(wk_host), C.byref(params), _ptr(o_host), _ptr(lse_host),
                                       _ptr(arena), arena.numel() * arena.element_size(), _stream(stream)),
            "seer_prefill_host")
+
+
+def seer_set_trace_buffer(ctx: Context, device_buffer) -> None:
+    _check(ctx._lib.seer_set_trace_buffer(ctx.handle, _ptr(device_buffer)), "seer_set_trace_buffer")

@@ -14,8 +14,9 @@
 // work group computes exact column maxima, rebases m, rescales its partial sums and the O accumulator, and recomputes
 // the tile.  Row sums are per-thread partials combined once per work item.
 //
-// Roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2-5 and 6-9 = two softmax
-// groups.  The tiles of a work item alternate between the groups (even tiles -> A, odd -> B); each group keeps its own
+// Roles (384 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + issuer of the S^T MMAs, warp 2 = TMA
+// producer for V, warp 3 = issuer of the P V MMAs (one thread can start a tcgen05.mma only every 64 clocks, so the two
+// products are issued from two threads), warps 4-7 and 8-11 = two softmax groups.  The tiles of a work item alternate between the groups (even tiles -> A, odd -> B); each group keeps its own
 // S^T buffers, P^T buffer, O^T accumulator, references and row sums, and the epilogue merges the two partial results
 // through their references.  One persistent CTA per SM walks the work items (longest rows first within each KV head).
 // Every wait is bounded; a wait that runs out raises SEER_ERR_TIMEOUT and the CTA drains and exits.
@@ -29,7 +30,7 @@
 namespace seer {
 namespace tc {
 
-constexpr int kThreads = 320;               // warp 0 producer, warp 1 MMA issuer, warps 2-5 / 6-9 softmax groups A / B
+constexpr int kThreads = 384;               // warps 0-3: K(+Q) producer, S^T issuer, V producer, P V issuer; warps 4-7 / 8-11: softmax groups A / B
 constexpr int kGroupThreads = 128;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
@@ -226,72 +227,6 @@ __device__ __forceinline__ int list_block(const Item& it, const int32_t* __restr
   return (j < 0 || j > it.i) ? -2 : j;
 }
 
-// Walks the tiles of this CTA's work items in order.  The producer and the MMA issuer each keep cursors of their
-// own; they see the same sequence because it depends only on the lists.
-struct Cursor {
-  int64_t w;
-  Item it;
-  int t;             // tile within the item
-  uint32_t k;        // ordinal of the item among this CTA's non-empty items
-  uint32_t g;        // ordinal of the tile among all tiles of this CTA
-  uint32_t cnt[2];   // tiles handed to softmax group 0 / 1 so far
-  bool valid;
-};
-__device__ __forceinline__ void cursor_seek(Cursor& c, const SeqMeta& m, const int32_t* __restrict__ row_ptr) {
-  c.valid = false;
-  while (c.w < m.rows) {
-    c.it = decode_item(m, row_ptr, c.w);
-    if (c.it.ntiles > 0) { c.valid = true; return; }
-    c.w += gridDim.x;
-  }
-}
-__device__ __forceinline__ void cursor_init(Cursor& c, const SeqMeta& m, const int32_t* __restrict__ row_ptr) {
-  c.w = blockIdx.x; c.t = 0; c.k = 0; c.g = 0; c.cnt[0] = c.cnt[1] = 0;
-  cursor_seek(c, m, row_ptr);
-}
-__device__ __forceinline__ void cursor_next(Cursor& c, const SeqMeta& m, const int32_t* __restrict__ row_ptr) {
-  c.cnt[c.t & 1] += 1;
-  c.g += 1;
-  if (++c.t >= c.it.ntiles) {
-    c.t = 0; c.k += 1; c.w += gridDim.x;
-    cursor_seek(c, m, row_ptr);
-  }
-}
-
-// One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]), packed to bf16 pairs.
-// Returns the largest exponent seen.  MASKED applies the causal mask of a diagonal block / drops a dead row.
-template <bool MASKED>
-__device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __restrict__ mref, float sl2, bool row_live,
-                                              bool diag, int key_local, uint32_t (&pk)[32]) {
-  float xmax = -CUDART_INF_F;
-  uint32_t sv[2][16];
-  tc_ld16(s_addr, sv[0]);
-#pragma unroll
-  for (int ch = 0; ch < 4; ++ch) {
-    tc_wait_ld(sv[ch & 1]);
-    if (ch < 3) tc_ld16(s_addr + (ch + 1) * 16, sv[(ch + 1) & 1]);
-#pragma unroll
-    for (int e = 0; e < 16; e += 4) {
-      const int c = ch * 16 + e;
-      const float4 mr = *reinterpret_cast<const float4*>(&mref[c]);
-      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -mr.x);
-      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -mr.y);
-      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -mr.z);
-      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -mr.w);
-      if (MASKED) {
-        if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 2)) x2 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 3)) x3 = -CUDART_INF_F;
-      }
-      xmax = fmaxf(xmax, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
-      pk[c >> 1] = pack_bf16(ex2f(x0), ex2f(x1));
-      pk[(c >> 1) + 1] = pack_bf16(ex2f(x2), ex2f(x3));
-    }
-  }
-  return xmax;
-}
-
 // Sums l[0..63] over the 32 lanes of a warp; lane ends with the totals of columns (2*bitrev-ish) base, base+1
 // where base = 32*b4 + 16*b3 + 8*b2 + 4*b1 + 2*b0 (b_i = bit i of the lane id).
 __device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out0, float& out1, int& base) {
@@ -345,12 +280,87 @@ __device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out
   base = ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
 }
 
+// One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]).
+//   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the largest exponent seen.
+//   SUBTRACT == true : removes p from l[c] again (used before a rebase; pk is not touched).
+// MASKED applies the causal mask of a diagonal block / drops a dead row.
+template <bool MASKED, bool SUBTRACT>
+__device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __restrict__ mref, float sl2, bool row_live,
+                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32]) {
+  float xmax = -CUDART_INF_F;
+  uint32_t sv[2][16];
+  tc_ld16(s_addr, sv[0]);
+#pragma unroll
+  for (int ch = 0; ch < 4; ++ch) {
+    tc_wait_ld(sv[ch & 1]);
+    if (ch < 3) tc_ld16(s_addr + (ch + 1) * 16, sv[(ch + 1) & 1]);
+#pragma unroll
+    for (int e = 0; e < 16; e += 4) {
+      const int c = ch * 16 + e;
+      const float4 mr = *reinterpret_cast<const float4*>(&mref[c]);
+      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -mr.x);
+      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -mr.y);
+      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -mr.z);
+      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -mr.w);
+      if (MASKED) {
+        if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
+        if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
+        if (!row_live || (diag && key_local > c + 2)) x2 = -CUDART_INF_F;
+        if (!row_live || (diag && key_local > c + 3)) x3 = -CUDART_INF_F;
+      }
+      const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
+      if (SUBTRACT) {
+        l[c] -= p0; l[c + 1] -= p1; l[c + 2] -= p2; l[c + 3] -= p3;
+      } else {
+        xmax = fmaxf(xmax, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
+        l[c] += p0; l[c + 1] += p1; l[c + 2] += p2; l[c + 3] += p3;
+        pk[c >> 1] = pack_bf16(p0, p1);
+        pk[(c >> 1) + 1] = pack_bf16(p2, p3);
+      }
+    }
+  }
+  return xmax;
+}
+
+// Optional timeline of CTA 0 (diagnostics): role r appends (tag << 32 | ordinal, clock) pairs to trace[r * 8192 ...].
+struct Tracer {
+  unsigned long long* p;
+  uint32_t n;
+  __device__ __forceinline__ void init(unsigned long long* base, int role) {
+    p = (base != nullptr && blockIdx.x == 0) ? base + (size_t)role * 8192 : nullptr;
+    n = 0;
+  }
+  __device__ __forceinline__ void ev(uint32_t tag, uint32_t ord) {
+    if (p != nullptr && n < 4095) {
+      p[2 * n] = ((unsigned long long)tag << 32) | ord;
+      p[2 * n + 1] = (unsigned long long)clock64();
+      ++n;
+    }
+  }
+};
+
+// Issues the TMA copies of one 128-key tile (blocks ja, jb of KV head g) into a ring slot.
+__device__ __forceinline__ void load_kv_tile(const CUtensorMap* map, uint32_t dst, uint32_t full_bar, const Item& it, int ja,
+                                             int jb) {
+  const bool has_b = jb != -1;
+  if (ja < 0) ja = 0;                // a rejected entry is replaced by block 0 and masked out in the softmax
+  if (jb < 0) jb = 0;
+  mbar_expect_tx(full_bar, has_b ? kKVBytes : kKVBytes / 2);
+  const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
+  tma_load_3d(dst, map, full_bar, 0, it.g, ta);
+  tma_load_3d(dst + kHalfKV, map, full_bar, 64, it.g, ta);
+  if (has_b) {
+    tma_load_3d(dst + kHalfQ, map, full_bar, 0, it.g, tb);
+    tma_load_3d(dst + kHalfKV + kHalfQ, map, full_bar, 64, it.g, tb);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ kernel
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, SeqMeta m, const int32_t* __restrict__ row_ptr,
                const int32_t* __restrict__ col_idx, uint16_t* __restrict__ o, float* __restrict__ lse,
-               int* __restrict__ status) {
+               int* __restrict__ status, unsigned long long* __restrict__ trace) {
   extern __shared__ unsigned char smem_raw[];
   Shared sh;
   sh.base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -385,123 +395,144 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  // ============================================================================================ producer
+  // Ordinals shared by all roles: k = non-empty items seen by this CTA, g = tiles seen, cnt_a / cnt_b = tiles handed to
+  // softmax group A / B.  Every role walks the same items and tiles, so the counters agree without communication.
+
+  // ============================================================================================ K (+Q) producer
   if (warp == 0) {
     if (lane == 0) {
-      Cursor kc, vc;                       // K runs one tile ahead of V
-      cursor_init(kc, m, row_ptr);
-      vc = kc;
-      auto load_k = [&](const Cursor& c) -> bool {
-        const Item& it = c.it;
-        if (c.t == 0) {                    // first tile of an item: its Q block
-          const uint32_t qb = c.k & 1u;
-          if (!mbar_wait(sh, Q_EMPTY + qb, ((c.k >> 1) & 1u) ^ 1u, status)) return false;
-          mbar_expect_tx(sh.bar(Q_FULL + qb), kQBytes);
-          const int tq = it.s0 + it.i * kBlock;
-          tma_load_3d(sh.base + kOffQ + qb * kQBytes, &map_q, sh.bar(Q_FULL + qb), 0, it.h, tq);
-          tma_load_3d(sh.base + kOffQ + qb * kQBytes + kHalfQ, &map_q, sh.bar(Q_FULL + qb), 64, it.h, tq);
-        }
-        int ja = list_block(it, col_idx, 2 * c.t), jb = list_block(it, col_idx, 2 * c.t + 1);
-        if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
-        const bool has_b = jb != -1;
-        if (ja < 0) ja = 0;                // a rejected entry is replaced by block 0 and masked out in the softmax
-        if (jb < 0) jb = 0;
-        const uint32_t st = c.g & 1u;
-        if (!mbar_wait(sh, K_EMPTY + st, ((c.g >> 1) & 1u) ^ 1u, status)) return false;
-        const uint32_t fb = sh.bar(K_FULL + st), dst = sh.base + kOffK + st * kKVBytes;
-        mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
-        const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
-        tma_load_3d(dst, &map_k, fb, 0, it.g, ta);
-        tma_load_3d(dst + kHalfKV, &map_k, fb, 64, it.g, ta);
-        if (has_b) {
-          tma_load_3d(dst + kHalfQ, &map_k, fb, 0, it.g, tb);
-          tma_load_3d(dst + kHalfKV + kHalfQ, &map_k, fb, 64, it.g, tb);
-        }
-        return true;
-      };
-      auto load_v = [&](const Cursor& c) -> bool {
-        const Item& it = c.it;
-        int ja = list_block(it, col_idx, 2 * c.t), jb = list_block(it, col_idx, 2 * c.t + 1);
-        const bool has_b = jb != -1;
-        if (ja < 0) ja = 0;
-        if (jb < 0) jb = 0;
-        const uint32_t st = c.g & 1u;
-        if (!mbar_wait(sh, V_EMPTY + st, ((c.g >> 1) & 1u) ^ 1u, status)) return false;
-        const uint32_t fb = sh.bar(V_FULL + st), dst = sh.base + kOffV + st * kKVBytes;
-        mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
-        const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
-        tma_load_3d(dst, &map_v, fb, 0, it.g, ta);
-        tma_load_3d(dst + kHalfKV, &map_v, fb, 64, it.g, ta);
-        if (has_b) {
-          tma_load_3d(dst + kHalfQ, &map_v, fb, 0, it.g, tb);
-          tma_load_3d(dst + kHalfKV + kHalfQ, &map_v, fb, 64, it.g, tb);
-        }
-        return true;
-      };
+      Tracer tr; tr.init(trace, 0);
+      uint32_t k = 0, g = 0;
       bool ok = true;
-      if (kc.valid) { ok = load_k(kc); cursor_next(kc, m, row_ptr); }
-      while (ok && vc.valid) {
-        if (kc.valid) { ok = load_k(kc); cursor_next(kc, m, row_ptr); }
-        if (ok) { ok = load_v(vc); cursor_next(vc, m, row_ptr); }
+      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+        const Item it = decode_item(m, row_ptr, w);
+        if (it.ntiles == 0) continue;
+        const uint32_t qb = k & 1u;
+        if (!mbar_wait(sh, Q_EMPTY + qb, ((k >> 1) & 1u) ^ 1u, status)) break;
+        mbar_expect_tx(sh.bar(Q_FULL + qb), kQBytes);
+        const int tq = it.s0 + it.i * kBlock;
+        tma_load_3d(sh.base + kOffQ + qb * kQBytes, &map_q, sh.bar(Q_FULL + qb), 0, it.h, tq);
+        tma_load_3d(sh.base + kOffQ + qb * kQBytes + kHalfQ, &map_q, sh.bar(Q_FULL + qb), 64, it.h, tq);
+        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
+        for (int t = 0; t < it.ntiles; ++t, ++g) {
+          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
+          if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
+          const uint32_t st = g & 1u;
+          tr.ev(1, g);
+          if (!mbar_wait(sh, K_EMPTY + st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
+          tr.ev(2, g);
+          load_kv_tile(&map_k, sh.base + kOffK + st * kKVBytes, sh.bar(K_FULL + st), it, ja, jb);
+          ja = na; jb = nb2;
+        }
+        ++k;
       }
     }
   }
-  // ============================================================================================ MMA issuer
+  // ============================================================================================ V producer
+  else if (warp == 2) {
+    if (lane == 0) {
+      Tracer tr; tr.init(trace, 2);
+      uint32_t g = 0;
+      bool ok = true;
+      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+        const Item it = decode_item(m, row_ptr, w);
+        if (it.ntiles == 0) continue;
+        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
+        for (int t = 0; t < it.ntiles; ++t, ++g) {
+          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
+          const uint32_t st = g & 1u;
+          tr.ev(3, g);
+          if (!mbar_wait(sh, V_EMPTY + st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
+          tr.ev(4, g);
+          load_kv_tile(&map_v, sh.base + kOffV + st * kKVBytes, sh.bar(V_FULL + st), it, ja, jb);
+          ja = na; jb = nb2;
+        }
+      }
+    }
+  }
+  // ============================================================================================ S^T issuer
   else if (warp == 1) {
     if (lane == 0) {
-      Cursor sc, pc;                       // S^T issue runs up to three tiles ahead of P V issue
-      cursor_init(sc, m, row_ptr);
-      pc = sc;
-      auto issue_s = [&](const Cursor& c) -> bool {
-        const int grp = c.t & 1;
-        const uint32_t cn = c.cnt[grp], buf = cn & 1u, st = c.g & 1u, qb = c.k & 1u;
-        if (c.t == 0 && !mbar_wait(sh, Q_FULL + qb, (c.k >> 1) & 1u, status)) return false;
-        if (!mbar_wait(sh, K_FULL + st, (c.g >> 1) & 1u, status)) return false;
-        if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) return false;
-        tc_fence_after();
-        const uint32_t k_addr = sh.base + kOffK + st * kKVBytes, q_addr = sh.base + kOffQ + qb * kQBytes;
-        const uint32_t d = tmem + col_s(grp, buf);
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t a = make_desc(k_addr + (kk >> 2) * kHalfKV + (kk & 3) * 32, 16, 1024);
-          const uint64_t b = make_desc(q_addr + (kk >> 2) * kHalfQ + (kk & 3) * 32, 16, 1024);
-          tc_mma(d, a, b, kIdescS, kk > 0);
-        }
-        tc_commit(sh.bar(S_FULL + 2 * grp + buf));
-        tc_commit(sh.bar(K_EMPTY + st));
-        if (c.t == c.it.ntiles - 1) tc_commit(sh.bar(Q_EMPTY + qb));   // last S^T of the item: Q may be replaced
-        return true;
-      };
-      auto issue_pv = [&](const Cursor& c) -> bool {
-        const int grp = c.t & 1;
-        const uint32_t cn = c.cnt[grp], st = c.g & 1u;
-        if (!mbar_wait(sh, V_FULL + st, (c.g >> 1) & 1u, status)) return false;
-        if (!mbar_wait(sh, P_FULL + grp, cn & 1u, status)) return false;
-        tc_fence_after();
-        const uint32_t v_addr = sh.base + kOffV + st * kKVBytes, p_addr = sh.base + kOffP + grp * kPBytes;
-        const int nk = (2 * c.t + 1 < c.it.nlist) ? 8 : 4;       // 16-key groups to contract over
-        const uint32_t d = tmem + col_o(grp);
-        for (int kk = 0; kk < nk; ++kk) {
-          const uint64_t a = make_desc(v_addr + kk * 2048, kHalfKV, 1024);
-          const uint64_t b = make_desc(p_addr + kk * 2048, kHalfKV, 1024);
-          tc_mma(d, a, b, kIdescPV, (c.t >= 2 || kk > 0) ? 1u : 0u);
-        }
-        tc_commit(sh.bar(V_EMPTY + st));
-        tc_commit(sh.bar(PV_DONE + grp));
-        return true;
-      };
+      Tracer tr; tr.init(trace, 1);
+      uint32_t k = 0, g = 0, cnt_a = 0, cnt_b = 0;
+      // descriptor bases; per K-step the start address advances by 32 bytes inside a 64-element swizzle atom and by
+      // one d-half (16 KB / 8 KB) between atoms
+      const uint64_t kd0 = make_desc(sh.base + kOffK, 16, 1024), kd1 = make_desc(sh.base + kOffK + kKVBytes, 16, 1024);
+      const uint64_t qd0 = make_desc(sh.base + kOffQ, 16, 1024), qd1 = make_desc(sh.base + kOffQ + kQBytes, 16, 1024);
       bool ok = true;
-      while (ok && pc.valid) {
-        while (ok && sc.valid && sc.g < pc.g + 3) { ok = issue_s(sc); cursor_next(sc, m, row_ptr); }
-        if (ok) { ok = issue_pv(pc); cursor_next(pc, m, row_ptr); }
+      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+        const Item it = decode_item(m, row_ptr, w);
+        if (it.ntiles == 0) continue;
+        const uint32_t qb = k & 1u;
+        if (!mbar_wait(sh, Q_FULL + qb, (k >> 1) & 1u, status)) break;
+        const uint64_t qd = qb ? qd1 : qd0;
+        for (int t = 0; t < it.ntiles; ++t, ++g) {
+          const int grp = t & 1;
+          const uint32_t cn = grp ? cnt_b : cnt_a, buf = cn & 1u, st = g & 1u;
+          tr.ev(10, g);
+          if (!mbar_wait(sh, K_FULL + st, (g >> 1) & 1u, status)) { ok = false; break; }
+          tr.ev(11, g);
+          if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
+          tr.ev(12, g);
+          tc_fence_after();
+          const uint64_t kd = st ? kd1 : kd0;
+          const uint32_t d = tmem + col_s(grp, buf);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            tc_mma(d, kd + (uint64_t)((kk >> 2) * (kHalfKV >> 4) + (kk & 3) * 2),
+                   qd + (uint64_t)((kk >> 2) * (kHalfQ >> 4) + (kk & 3) * 2), kIdescS, kk > 0);
+          tc_commit(sh.bar(S_FULL + 2 * grp + buf));
+          tc_commit(sh.bar(K_EMPTY + st));
+          if (t == it.ntiles - 1) tc_commit(sh.bar(Q_EMPTY + qb));   // last S^T of the item: Q may be replaced
+          tr.ev(17, g);
+          if (grp) ++cnt_b; else ++cnt_a;
+        }
+        ++k;
+      }
+    }
+  }
+  // ============================================================================================ P V issuer
+  else if (warp == 3) {
+    if (lane == 0) {
+      Tracer tr; tr.init(trace, 3);
+      uint32_t g = 0, cnt_a = 0, cnt_b = 0;
+      const uint64_t vd0 = make_desc(sh.base + kOffV, kHalfKV, 1024), vd1 = make_desc(sh.base + kOffV + kKVBytes, kHalfKV, 1024);
+      const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024), pd1 = make_desc(sh.base + kOffP + kPBytes, kHalfKV, 1024);
+      bool ok = true;
+      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+        const Item it = decode_item(m, row_ptr, w);
+        for (int t = 0; t < it.ntiles; ++t, ++g) {
+          const int grp = t & 1;
+          const uint32_t cn = grp ? cnt_b : cnt_a, st = g & 1u;
+          tr.ev(13, g);
+          if (!mbar_wait(sh, V_FULL + st, (g >> 1) & 1u, status)) { ok = false; break; }
+          tr.ev(14, g);
+          if (!mbar_wait(sh, P_FULL + grp, cn & 1u, status)) { ok = false; break; }
+          tr.ev(15, g);
+          tc_fence_after();
+          const uint64_t vd = st ? vd1 : vd0, pd = grp ? pd1 : pd0;
+          const uint32_t d = tmem + col_o(grp);
+          const uint32_t acc0 = t >= 2 ? 1u : 0u;                  // first tile of this group in the item starts O^T afresh
+          // 16 keys (2048 bytes of 128-byte rows) per step; an odd list leaves the second block of its last tile out
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) tc_mma(d, vd + (uint64_t)(kk * 128), pd + (uint64_t)(kk * 128), kIdescPV, kk > 0 ? 1u : acc0);
+          if (2 * t + 1 < it.nlist) {
+#pragma unroll
+            for (int kk = 4; kk < 8; ++kk) tc_mma(d, vd + (uint64_t)(kk * 128), pd + (uint64_t)(kk * 128), kIdescPV, 1u);
+          }
+          tc_commit(sh.bar(V_EMPTY + st));
+          tc_commit(sh.bar(PV_DONE + grp));
+          tr.ev(19, g);
+          if (grp) ++cnt_b; else ++cnt_a;
+        }
       }
     }
   }
   // ============================================================================================ softmax groups
   else {
-    const int grp = (warp - 2) >> 2;                     // 0 = A (even tiles), 1 = B (odd tiles)
-    const int gt = threadIdx.x - 64 - grp * kGroupThreads;   // 0..127 within the group
-    const int gw = (warp - 2) & 3;                       // warp within the group
+    const int grp = (warp - 4) >> 2;                     // 0 = A (even tiles), 1 = B (odd tiles)
+    const int gt = threadIdx.x - 128 - grp * kGroupThreads;   // 0..127 within the group
+    const int gw = (warp - 4) & 3;                       // warp within the group
     const int quad = warp & 3;                           // TMEM lane quadrant this warp may access
     const int r = quad * 32 + lane;                      // key row of S^T / d row of O^T owned by this thread
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -520,6 +551,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int bar_sync = 1 + grp, bar_vote = 3 + grp;
     const float sl2 = m.softmax_scale * 1.4426950408889634f;
     const int key_local = r & 63;
+    Tracer tr; tr.init(gt == 0 ? trace : nullptr, 4 + grp);
     uint32_t cnt = 0;                                    // tiles this group has processed
     uint32_t gbase = 0;                                  // tiles of this CTA before the current item
     bool ok = true;
@@ -537,10 +569,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
       for (int t = grp; t < it.ntiles; t += 2, ++cnt) {
         const uint32_t sbuf = cnt & 1u;
+        tr.ev(20, gbase + t);
         bool fail = !mbar_wait(sh, S_FULL + 2 * grp + sbuf, (cnt >> 1) & 1u, status);
+        tr.ev(21, gbase + t);
         // the previous P V of this group has finished: its P^T buffer and the O^T accumulator may be touched
         if (!fail && cnt > 0) fail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
         tc_fence_after();
+        tr.ev(22, gbase + t);
         const int ja = list_block(it, col_idx, 2 * t), jb = list_block(it, col_idx, 2 * t + 1);
         const int my_j = r < 64 ? ja : jb;
         const bool row_live = my_j >= 0;                 // absent / rejected blocks contribute nothing
@@ -549,12 +584,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t s_addr = tmem + lane_addr + col_s(grp, sbuf);
         uint32_t pk[32];
         float xmax = -CUDART_INF_F;
-        if (!fail) xmax = masked ? softmax_pass<true>(s_addr, mref, sl2, row_live, diag, key_local, pk)
-                                 : softmax_pass<false>(s_addr, mref, sl2, row_live, diag, key_local, pk);
+        if (!fail) xmax = masked ? softmax_pass<true, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk)
+                                 : softmax_pass<false, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+        tr.ev(23, gbase + t);
         // one vote per tile: does any entry exceed its reference by more than 2^8 (or has a wait been lost)?
-        if (named_bar_or(bar_vote, kGroupThreads, fail || xmax > 8.f)) {
+        const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || xmax > 8.f);
+        tr.ev(24, gbase + t);
+        if (slow) {
           if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
-          // ---- exact column maxima of this tile -> new references, rescale partial sums and O^T, recompute the tile
+          // ---- rebase: take this tile's contribution out of the row sums again, find the exact column maxima, move
+          // the references, rescale the row sums and O^T, and recompute the tile
+          if (t >= 2) {
+            if (masked) softmax_pass<true, true>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+            else softmax_pass<false, true>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+          }
           if (gt < 64) colmax[gt] = float_order_int(-CUDART_INF_F);
           named_bar_sync(bar_sync, kGroupThreads);
 #pragma unroll
@@ -580,8 +623,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             mref[gt] = nm;
           }
           named_bar_sync(bar_sync, kGroupThreads);
+          // a reference that moved by more than 2^30 makes everything accumulated so far negligible (and the value
+          // taken out above may not have been finite): start the column afresh
 #pragma unroll
-          for (int c = 0; c < 64; ++c) l_part[c] *= alpha[c];
+          for (int c = 0; c < 64; ++c) {
+            const float a = alpha[c];
+            l_part[c] = (t < 2 || a < 9.3e-10f) ? 0.f : l_part[c] * a;
+          }
           if (t >= 2) {                                  // this group already accumulated into O^T for this item
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
@@ -594,18 +642,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             }
             tc_wait_st();
           }
-          if (masked) softmax_pass<true>(s_addr, mref, sl2, row_live, diag, key_local, pk);
-          else softmax_pass<false>(s_addr, mref, sl2, row_live, diag, key_local, pk);
+          if (masked) softmax_pass<true, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+          else softmax_pass<false, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
         }
         // the S^T buffer may be overwritten by a later tile
         tc_fence_before();
         mbar_arrive(sh.bar(S_EMPTY + 2 * grp + sbuf));
-        // row sums over the bf16-rounded probabilities the MMA will use
-#pragma unroll
-        for (int c2 = 0; c2 < 32; ++c2) {
-          l_part[2 * c2] += __uint_as_float(pk[c2] << 16);
-          l_part[2 * c2 + 1] += __uint_as_float(pk[c2] & 0xffff0000u);
-        }
         // P^T row r -> shared memory (128-byte swizzle)
         {
           const uint32_t prow = sh.base + kOffP + grp * kPBytes + (uint32_t)r * 128u;
@@ -630,11 +672,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         fence_async_smem();
         tc_fence_before();
         mbar_arrive(sh.bar(P_FULL + grp));
+        tr.ev(25, gbase + t);
       }
-
       gbase += (uint32_t)it.ntiles;
 
       // ------------------------------------------------------------------------------------------ epilogue
+      tr.ev(30, (uint32_t)(w / gridDim.x));
       bool efail = !ok;
       if (ok && my_tiles > 0) efail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
       tc_fence_after();
@@ -693,6 +736,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
       named_bar_sync(bar_sync, kGroupThreads);   // staging is free again before this group's next P^T
+      tr.ev(31, (uint32_t)(w / gridDim.x));
     }
   }
 
@@ -749,7 +793,7 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
     return -(int)cudaErrorInvalidValue;
   const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, m.rows);
   tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse,
-                                                                    ctx->d_status);
+                                                                    ctx->d_status, (unsigned long long*)ctx->trace);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;
 }

@@ -307,6 +307,12 @@ seer_status seer_poll_device_status(seer_ctx* ctx, void* stream_) {
 
 int64_t seer_launch_count(const seer_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
+seer_status seer_set_trace_buffer(seer_ctx* ctx, void* device_buffer) {
+  if (!ctx) return SEER_ERR_INVALID_ARG;
+  ctx->trace = device_buffer;
+  return SEER_OK;
+}
+
 namespace {
 struct ArenaLayout {
   size_t q, k, v, o, wq, wk, scores, row_ptr, col_idx, nnz, lse, ws, total;

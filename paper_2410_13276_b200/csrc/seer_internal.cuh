@@ -59,6 +59,7 @@ struct seer_ctx {
   uint64_t clock = 0;
   seer::MetaSlot slots[seer::kMetaSlots];
   void* tmap_encode = nullptr;   // cuTensorMapEncodeTiled, resolved at run time
+  void* trace = nullptr;         // optional device buffer for the attention kernel's timeline (diagnostics)
 };
 
 namespace seer {

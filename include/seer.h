@@ -140,6 +140,35 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
                               const seer_mask_params* params, void* o_host, float* lse_host, void* arena,
                               size_t arena_bytes, void* stream);
 
+/* Gate scores without any allocation (the paper has no counterpart; this is a deployment variant of call 1).
+ *
+ * Who needs it: code that may not allocate device memory at the point where it runs the gate -- a serving process whose
+ * memory pool has handed every byte to the KV cache, a plugin that runs inside another framework's allocator and must not
+ * call cudaMalloc behind its back, a latency-critical loop where cudaMalloc's implicit device synchronisation is not
+ * acceptable.  Such a caller cannot create a seer_ctx (seer_create allocates) nor provide a workspace.
+ *
+ * What it does: the same two kernels as seer_gate_scores, same arguments and results (q, k, Wq, Wk in, scores out, all
+ * DEVICE pointers owned by the caller), on the CURRENT device, without a context and without a workspace.  The
+ * intermediate projected vectors and the per-batch offsets live in a fixed array inside the library image: every GPU
+ * that loads the library holds SEER_STATIC_SCRATCH_BYTES + 16 KiB for it until the process exits.
+ *
+ * Limits: shape->batch <= SEER_STATIC_MAX_BATCH and (num_q_heads + num_kv_heads) * total_blocks * 512 bytes (rounded up to
+ * 256 per tensor) <= SEER_STATIC_SCRATCH_BYTES, i.e. 16384 (head, block) pairs: e.g. 40 heads x 26000 tokens.  Larger shapes
+ * return SEER_ERR_WORKSPACE and enqueue nothing.
+ *
+ * First call on a device: looks up the array's device address and raises one kernel's shared-memory limit (no allocation).
+ * Make that first call outside of any stream capture.  The call itself performs no cudaMalloc / cudaFree and uses no
+ * allocating library routine; it copies about 5 KiB of offsets from the host stack with cudaMemcpyAsync and launches.
+ *
+ * Sharing: all calls on a device use the same array, which keeps whatever the last call left there.  Nothing in it needs to
+ * start at zero (the first kernel rewrites all that the second reads).  Two calls that overlap on the GPU -- different
+ * streams without an ordering between them, or different host threads -- race on it: keep the calls of one device on one
+ * stream, or order them yourself. */
+#define SEER_STATIC_SCRATCH_BYTES (8u << 20)
+#define SEER_STATIC_MAX_BATCH 256
+seer_status seer_gate_scores_static(const seer_shape* shape, const void* q, const void* k, const float* Wq,
+                                    const float* Wk, float* scores, void* stream);
+
 /* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, CTA 0 of the tcgen05 attention kernel
  * records a timeline of its pipeline roles into it: 6 roles x 4096 (tag << 32 | ordinal, SM clock) pairs of uint64, i.e.
  * at least 6 * 8192 * 8 bytes of device memory, zero-initialised by the caller.  NULL switches it off (default). */

@@ -25,7 +25,7 @@ STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER
 EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
            "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
-           "seer_prefill_host", "seer_set_trace_buffer"]
+           "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static"]
 
 
 class SeerError(RuntimeError):
@@ -90,6 +90,8 @@ def load_library() -> C.CDLL:
     lib.seer_prefill_host_arena_bytes.restype = sz
     lib.seer_prefill_host.argtypes = [vp, shp, vp, vp, vp, vp, vp, C.POINTER(seer_mask_params), vp, vp, vp, sz, vp]
     lib.seer_prefill_host.restype = C.c_int
+    lib.seer_gate_scores_static.argtypes = [shp, vp, vp, vp, vp, vp, vp]
+    lib.seer_gate_scores_static.restype = C.c_int
     lib.seer_set_trace_buffer.argtypes = [vp, vp]
     lib.seer_set_trace_buffer.restype = C.c_int
     _lib = lib
@@ -229,3 +231,15 @@ def seer_prefill_host(ctx: Context, shape: seer_shape, q_host, k_host, v_host, w
 
 def seer_set_trace_buffer(ctx: Context, device_buffer) -> None:
     _check(ctx._lib.seer_set_trace_buffer(ctx.handle, _ptr(device_buffer)), "seer_set_trace_buffer")
+
+
+SEER_STATIC_SCRATCH_BYTES = 8 << 20
+SEER_STATIC_MAX_BATCH = 256
+
+
+def seer_gate_scores_static(shape: seer_shape, q, k, wq, wk, scores, stream=None) -> None:
+    """Gate scores for callers that must not allocate: no context, no workspace; the intermediates live in a fixed
+    array inside the library (at most SEER_STATIC_SCRATCH_BYTES per call, else SEER_ERR_WORKSPACE).  Runs on the
+    current device.  Calls on one device share that array, so keep them on one stream."""
+    _check(load_library().seer_gate_scores_static(C.byref(shape), _ptr(q), _ptr(k), _ptr(wq), _ptr(wk), _ptr(scores),
+                                                  _stream(stream)), "seer_gate_scores_static")

@@ -6,6 +6,9 @@
 // on softmax outputs when logits reach tens).
 #include <math_constants.h>
 
+#include <cstddef>
+#include <mutex>
+
 #include "seer_internal.cuh"
 
 namespace seer {
@@ -243,6 +246,95 @@ int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, c
   return e == cudaSuccess ? 2 : -(int)e;
 }
 
+// ----------------------------------------------------------------------------------------------- allocation-free variant
+// Scratch for seer_gate_scores_static lives in the library image: every GPU that loads the library carries these
+// bytes until the process exits.  Host code must never hand the symbol itself to a kernel; its device address is
+// looked up once per device with cudaGetSymbolAddress.
+constexpr int kStaticMaxBatch = SEER_STATIC_MAX_BATCH;
+constexpr size_t kStaticMetaBytes = 16 * 1024;                              // cu_seqlens + four offset arrays
+constexpr size_t kStaticScratchBytes = (size_t)SEER_STATIC_SCRATCH_BYTES;   // projected pooled Q and K (fp32)
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticMetaBytes + kStaticScratchBytes];
+
+constexpr int kStaticMaxDevices = 64;
+static std::mutex g_static_mutex;
+static void* g_static_addr[kStaticMaxDevices];     // device address of g_static_scratch, per device ordinal
+static bool g_static_ready[kStaticMaxDevices];
+
+// Once per device, with that device current: resolve the array's device address and lift the score kernel's
+// shared-memory limit.  Neither call allocates.
+static seer_status static_setup(int dev, unsigned char** out) {
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ready[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return SEER_ERR_CUDA;
+    if (cudaFuncSetAttribute(gate_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem) != cudaSuccess)
+      return SEER_ERR_CUDA;
+    g_static_addr[dev] = ptr;
+    g_static_ready[dev] = true;
+  }
+  *out = (unsigned char*)g_static_addr[dev];
+  return SEER_OK;
+}
+
+seer_status gate_scores_static(const seer_shape* shape, const void* q, const void* k, const float* Wq, const float* Wk,
+                               float* scores, cudaStream_t stream) {
+  ShapeTotals t;
+  seer_status st = shape_totals(shape, &t);
+  if (st != SEER_OK) return st;
+  if (t.total_blocks == 0) return SEER_OK;
+  if (!q || !k || !Wq || !Wk || !scores) return SEER_ERR_INVALID_ARG;
+  // sizes beyond the built-in scratch are refused, never truncated
+  if (shape->batch > kStaticMaxBatch || gate_workspace_bytes(t, shape) > kStaticScratchBytes) return SEER_ERR_WORKSPACE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return SEER_ERR_CUDA;
+  unsigned char* base = nullptr;
+  st = static_setup(dev, &base);
+  if (st != SEER_OK) return st;
+
+  // per-batch offsets, built on the host stack and copied into the head of the array
+  struct HostMeta {
+    int32_t cu[kStaticMaxBatch + 4], blk[kStaticMaxBatch + 4], chunk[kStaticMaxBatch + 4], tile[kStaticMaxBatch + 4];
+    int64_t score[kStaticMaxBatch + 2];
+  } hm;
+  static_assert(sizeof(HostMeta) <= kStaticMetaBytes, "metadata region too small");
+  hm.blk[0] = hm.chunk[0] = hm.tile[0] = 0;
+  hm.score[0] = 0;
+  for (int b = 0; b < shape->batch; ++b) {
+    hm.cu[b] = shape->cu_seqlens_host[b];
+    const int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + kBlock - 1) / kBlock;
+    hm.blk[b + 1] = hm.blk[b] + nb;
+    hm.chunk[b + 1] = hm.chunk[b] + (nb + kPoolChunk - 1) / kPoolChunk;
+    hm.tile[b + 1] = hm.tile[b] + (nb + kScoreTile - 1) / kScoreTile;
+    hm.score[b + 1] = hm.score[b] + (int64_t)shape->num_q_heads * nb * nb;
+  }
+  hm.cu[shape->batch] = shape->cu_seqlens_host[shape->batch];
+  // pageable source: the runtime stages the bytes before returning, so the stack buffer may go out of scope
+  if (cudaMemcpyAsync(base, &hm, sizeof(HostMeta), cudaMemcpyHostToDevice, stream) != cudaSuccess) return SEER_ERR_CUDA;
+
+  SeqMeta m;
+  m.cu_seqlens = (const int32_t*)(base + offsetof(HostMeta, cu));
+  m.blk_off = (const int32_t*)(base + offsetof(HostMeta, blk));
+  m.chunk_off = (const int32_t*)(base + offsetof(HostMeta, chunk));
+  m.tile_off = (const int32_t*)(base + offsetof(HostMeta, tile));
+  m.score_off = (const int64_t*)(base + offsetof(HostMeta, score));
+  m.batch = shape->batch;
+  m.num_q_heads = shape->num_q_heads;
+  m.num_kv_heads = shape->num_kv_heads;
+  m.group = shape->num_q_heads / shape->num_kv_heads;
+  m.total_tokens = (int32_t)t.total_tokens;
+  m.total_blocks = (int32_t)t.total_blocks;
+  m.total_chunks = (int32_t)t.total_chunks;
+  m.total_tiles = (int32_t)t.total_tiles;
+  m.max_nb = t.max_nb;
+  m.rows = t.rows;
+  m.score_elems = t.score_elems;
+  m.softmax_scale = 0.f;   // unused by the gate
+  // The two kernels below are the ones seer_gate_scores launches; only the scratch pointer differs.  Nothing in the
+  // scratch has to start at zero: the first kernel writes every projected vector the second one reads.
+  const int n = launch_gate(nullptr, m, q, k, Wq, Wk, scores, base + kStaticMetaBytes, stream);
+  return n < 0 ? SEER_ERR_CUDA : SEER_OK;
+}
+
 seer_status init_gate(seer_ctx* ctx) {
   (void)ctx;
   cudaError_t e = cudaFuncSetAttribute(gate_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreSmem);
@@ -250,3 +342,9 @@ seer_status init_gate(seer_ctx* ctx) {
 }
 
 }  // namespace seer
+
+extern "C" seer_status seer_gate_scores_static(const seer_shape* shape, const void* q, const void* k, const float* Wq,
+                                               const float* Wk, float* scores, void* stream) {
+  if (!shape) return SEER_ERR_INVALID_ARG;
+  return seer::gate_scores_static(shape, q, k, Wq, Wk, scores, (cudaStream_t)stream);
+}

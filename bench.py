@@ -47,13 +47,13 @@ def parse():
     return ap.parse_args()
 
 
-def pick_mask(w, args):
+def pick_mask(w, args, need_threshold=True):
     from paper_2410_13276_b200 import workloads as W
     if w.name.startswith("c3"):
         num, den = (int(x) for x in args.keep.split("/"))
         return W.MaskSpec(W.MODE_TOPK_RATIO, num, den, flags=W.FORCE_DIAG | W.FORCE_SINK)
     spec = w.masks[0]
-    if spec.mode == W.MODE_THRESHOLD and spec.threshold is None:
+    if spec.mode == W.MODE_THRESHOLD and spec.threshold is None and need_threshold:
         with open(os.path.join(ROOT, "tests", "golden", "thresholds.json")) as f:
             spec.threshold = float.fromhex(json.load(f)[w.name]["threshold_hex"])
     return spec
@@ -64,7 +64,7 @@ def workload_desc(w, spec):
                         f"{w.num_q_heads} q heads / {w.num_kv_heads} kv heads, head_dim 128, block 64, causal",
             "mask": ({0: "topk_ratio", 1: "topk_count", 2: "threshold"}[spec.mode]
                      + (f" {spec.keep_num}/{spec.keep_den}" if spec.mode == 0 else
-                        f" {spec.threshold!r}" if spec.mode == 2 else f" {spec.k}")
+                        f" {spec.threshold!r} (target sparsity {spec.target_sparsity})" if spec.mode == 2 else f" {spec.k}")
                      + f", flags {spec.flags}"),
             "l2": "inputs larger than L2 (no flush)"}
 
@@ -132,64 +132,63 @@ def cpu_oracle_sample(w, rp, col, budget_rows=None):
     return blocks * FLOP_PER_BLOCK / dt / 1e12, dt, f"oracle attention on {len(rows)} sampled (head, query-block) rows = {blocks} kept blocks; gate and mask oracle not included", cores
 
 
+def seeded_lists_for_rows(w, spec, rows, seed=99):
+    """Lists for a handful of rows without running the gate: TopK of seeded random scores under the workload's mask
+    parameters (for a TopK-ratio mask the list lengths equal those of the real mask).  Oracle selection code only."""
+    from oracle import seer_oracle as O
+    from paper_2410_13276_b200 import workloads as W
+    nbs = [int(n) for n in w.num_blocks]
+    rng = np.random.default_rng(seed)
+    counts = np.zeros(sum(nbs) * w.num_q_heads, dtype=np.int64)
+    lists = {}
+    for r in rows:
+        off = 0
+        for nb in nbs:
+            if r < off + nb * w.num_q_heads:
+                break
+            off += nb * w.num_q_heads
+        i = (int(r) - off) % nb
+        s = rng.random(i + 1).astype(np.float32)
+        if spec.mode == W.MODE_THRESHOLD:      # no tuned scores here: keep the workload's target fraction by TopK instead
+            keep = max(1, round((1.0 - spec.target_sparsity) * 1000))
+            lists[int(r)] = O.select_row(s, i, O.MODE_TOPK_RATIO, keep_num=keep, keep_den=1000, flags=spec.flags)
+        else:
+            lists[int(r)] = O.select_row(s, i, spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                                         flags=spec.flags)
+        counts[int(r)] = len(lists[int(r)])
+    rp = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    col = np.concatenate([np.asarray(lists[int(r)], np.int32) for r in sorted(lists)]) if lists else np.zeros(0, np.int32)
+    return rp, col
+
+
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """Reference arm: the CPU oracle as it stands, timed on this machine's host cores.  One step = the oracle's
+    block-sparse attention on a fixed sample of (head, query-block) rows of the bench workload."""
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle import seer_oracle as O
     from paper_2410_13276_b200 import workloads as W
     w = W.make_workload(args.workload, seq=args.seq)
-    spec = pick_mask(w, args)
-    # lists for the sampled rows come from the oracle's own gate + mask on a slice of heads would take minutes at
-    # this size; the sample uses TopK lists of seeded random scores with the same keep ratio instead (same row lengths).
-    nbs = w.num_blocks
-    rng = np.random.default_rng(99)
-    heads = list(range(0, w.num_q_heads, 4))
-    rp = np.zeros(int(nbs.sum()) * w.num_q_heads + 1, dtype=np.int64)
-    cols = []
-    picks = []
-    base = 0
+    spec = pick_mask(w, args, need_threshold=False)
+    nbs = [int(n) for n in w.num_blocks]
+    rows, off = [], 0
     for nb in nbs:
-        nb = int(nb)
-        for h in range(w.num_q_heads):
-            for i in range(nb):
-                rp[base + h * nb + i + 1] = 0
-        for h in heads:
-            for i in {0, nb // 2, nb - 1}:
-                picks.append(base + h * nb + i)
-        base += nb * w.num_q_heads
-    picks = sorted(set(picks))
-    lists = {}
-    for r in picks:
-        # decode i from r for the single-sequence / multi-sequence layout
-        b = 0
-        off = 0
-        for bb, nb in enumerate(nbs):
-            if r < off + int(nb) * w.num_q_heads:
-                b = bb
-                break
-            off += int(nb) * w.num_q_heads
-        i = (r - off) % int(nbs[b])
-        s = rng.random(i + 1).astype(np.float32)
-        lists[r] = O.select_row(s, i, spec.mode if spec.mode != W.MODE_THRESHOLD else O.MODE_TOPK_RATIO,
-                                keep_num=spec.keep_num if spec.mode == 0 else 1, keep_den=spec.keep_den if spec.mode == 0 else 10,
-                                k=spec.k, flags=spec.flags)
-    counts = np.zeros(len(rp) - 1, dtype=np.int64)
-    for r, l in lists.items():
-        counts[r] = len(l)
-    rp[1:] = np.cumsum(counts)
-    col = np.concatenate([np.asarray(lists[r], np.int32) for r in picks])
-    blocks = int(counts.sum())
+        for h in range(0, w.num_q_heads, 8):
+            rows += [off + h * nb + i for i in sorted({0, nb // 4, nb // 2, nb - 1})]
+        off += nb * w.num_q_heads
+    rp, col = seeded_lists_for_rows(w, spec, rows)
+    blocks = int(rp[-1])
     times = []
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64, w.softmax_scale, rows=picks)
+        O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64, w.softmax_scale, rows=rows)
         if it >= args.warmup:
             times.append(time.perf_counter() - t0)
     ms = 1e3 * float(np.mean(times))
     val = blocks * FLOP_PER_BLOCK / (ms * 1e-3) / 1e12
     cores = len(os.sched_getaffinity(0))
-    sample = f"oracle attention on {len(picks)} sampled (head, query-block) rows = {blocks} kept blocks per step"
+    sample = (f"oracle attention (fp64 numpy) on {len(rows)} sampled (head, query-block) rows = {blocks} kept blocks per step; "
+              "gate and mask oracle not included")
     print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
                       "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
                       "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",

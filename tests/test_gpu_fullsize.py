@@ -1,0 +1,123 @@
+"""Parity at the full sizes of the five workloads, in the launch configuration bench.py times (whole GPU path, default
+attention kernel).  The oracle cannot run attention in full at these sizes, so it checks (a) gate scores of a few heads,
+(b) the block lists of those heads, rebuilt from the GPU's own scores (bit-exact), (c) attention on a stratified sample
+of (head, query block) rows, one output element at a time, with the GPU's lists fed to both, and (d) properties that
+hold at any size (list lengths in closed form, ordering, range)."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import seer_oracle as O
+from paper_2410_13276_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "thresholds.json")
+
+
+@pytest.fixture(scope="module")
+def rt():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("no CUDA device: the gpu tests must run on a B200")
+    from paper_2410_13276_b200 import binding as B
+    from paper_2410_13276_b200.prefill import Prefill
+    ctx = B.Context(0)
+    yield B, Prefill, ctx
+    ctx.close()
+
+
+def golden_threshold(name):
+    with open(GOLDEN) as f:
+        return float.fromhex(json.load(f)[name]["threshold_hex"])
+
+
+def head_slice_scores(flat, w, heads):
+    per_seq = O.unflatten_scores(flat, w.cu_seqlens, 64, w.num_q_heads)
+    return [s[heads] for s in per_seq]
+
+
+def check_workload(rt, name, specs, sample_heads, rows_per_head=3):
+    B, Prefill, ctx = rt
+    w = W.make_workload(name)
+    G = w.num_q_heads // w.num_kv_heads
+    p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    p.gate()
+    gpu_scores = p.scores_host()
+    # (a) gate scores of the sampled heads against the oracle run on those heads alone
+    for h in sample_heads:
+        g = h // G
+        ref = O.gate_scores(np.ascontiguousarray(w.q[:, h:h + 1]), np.ascontiguousarray(w.k[:, g:g + 1]),
+                            w.wq[h:h + 1], w.wk[g:g + 1], w.cu_seqlens, 64)
+        got = head_slice_scores(gpu_scores, w, [h])
+        for r, x in zip(ref, got):
+            il = np.tril_indices(r.shape[-1])
+            rr, xx = r[:, il[0], il[1]].astype(np.float64), x[:, il[0], il[1]].astype(np.float64)
+            assert np.all(np.abs(xx - rr) <= np.where(rr < 1e-30, 1e-33, 1e-3 * rr)), (name, h)
+    nbs = [int(n) for n in w.num_blocks]
+    for spec in specs:
+        params = B.make_mask_params(spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                                    threshold=spec.threshold or 0.0, flags=spec.flags)
+        p.mask(params)
+        p.o.fill_(float("nan"))
+        p.attn()
+        assert p.status() == 0
+        rp, col = p.lists_host()
+        # (d) properties at any size
+        counts = np.diff(rp)
+        assert rp[0] == 0 and rp[-1] == len(col) == int(p.nnz.item())
+        base = 0
+        for nb in nbs:
+            i_of_row = np.tile(np.arange(nb), w.num_q_heads)
+            c = counts[base:base + w.num_q_heads * nb]
+            if spec.mode == W.MODE_TOPK_RATIO:
+                nf = np.where(i_of_row == 0, 1, bin(spec.flags & 3).count("1"))
+                ki = np.clip(-((-spec.keep_num * (i_of_row + 1)) // spec.keep_den), 1, i_of_row + 1)
+                assert np.array_equal(c, np.maximum(ki, nf))
+            assert np.all(c >= 1) and np.all(c <= i_of_row + 1)
+            base += w.num_q_heads * nb
+        row_of = np.repeat(np.arange(len(counts)), counts)
+        same_row = row_of[1:] == row_of[:-1]
+        assert np.all(col[1:][same_row] > col[:-1][same_row])            # ascending, unique
+        assert np.all(col >= 0)
+        # (b) lists of the sampled heads, rebuilt by the oracle from the GPU's scores: bit-exact
+        base = 0
+        for b, nb in enumerate(nbs):
+            for h in sample_heads:
+                s = head_slice_scores(gpu_scores, w, [h])[b]
+                orp, ocol = O.block_mask([s], spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                                         threshold=spec.threshold or 0.0, flags=spec.flags)
+                r0 = base + h * nb
+                assert np.array_equal(np.diff(rp[r0:r0 + nb + 1]), np.diff(orp)), (name, h)
+                assert np.array_equal(col[rp[r0]:rp[r0 + nb]], ocol), (name, h)
+            base += w.num_q_heads * nb
+        # (c) attention on a stratified sample of rows with the GPU's lists
+        rows = W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=11, per_head_random=rows_per_head, heads=sample_heads)
+        o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64,
+                                            1 / math.sqrt(128), rows=rows)
+        done = ~np.isnan(o_ref[..., 0])
+        assert done.sum() > 0
+        x, r = p.o_host()[done].astype(np.float64), o_ref[done]
+        err = np.abs(x - r)
+        assert np.all(err <= 2e-2 + 1e-2 * np.abs(r)), (name, err.max())
+        rms = np.sqrt((err ** 2).sum(-1)) / np.maximum(np.sqrt((r ** 2).sum(-1)), 1e-30)
+        assert rms.max() <= 1e-2, (name, rms.max())
+        lg, lr = p.lse_host().T[done].astype(np.float64), lse_ref.T[done]
+        assert np.all(np.abs(lg - lr) <= 2e-3 + 1e-3 * np.abs(lr))
+        assert not np.isnan(p.o_host()).any()                            # every row was written
+
+
+def test_c3_128k_topk_bench_configuration(rt):
+    specs = [W.MaskSpec(W.MODE_TOPK_RATIO, 1, 10, flags=W.FORCE_DIAG | W.FORCE_SINK),
+             W.MaskSpec(W.MODE_TOPK_RATIO, 1, 2, flags=W.FORCE_DIAG | W.FORCE_SINK)]
+    check_workload(rt, "c3", specs, sample_heads=[0, 13, 31], rows_per_head=2)
+
+
+@pytest.mark.parametrize("name,heads", [("c2", [3, 28]), ("c4", [0, 22, 39]), ("c5", [5, 7, 16])])
+def test_threshold_workloads_full_size(rt, name, heads):
+    w_spec = W.make_workload(name + "s").masks[0]            # same mask recipe as the full-size workload
+    spec = W.MaskSpec(W.MODE_THRESHOLD, threshold=golden_threshold(name), flags=w_spec.flags)
+    check_workload(rt, name, [spec], sample_heads=heads, rows_per_head=2)

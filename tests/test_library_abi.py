@@ -1,0 +1,59 @@
+"""The C-ABI library builds, loads without a GPU and exports every function include/seer.h declares; the host-only
+sizing helpers compute the closed forms of the layout."""
+import os
+import re
+
+import pytest
+
+from paper_2410_13276_b200 import binding as B, build as build_mod
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_mod.build()
+    return B.load_library()
+
+
+def declared_functions(repo_root):
+    text = open(os.path.join(repo_root, "include", "seer.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(seer_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(lib, repo_root):
+    names = declared_functions(repo_root)
+    assert "seer_gate_scores" in names and "seer_block_mask" in names and "seer_sparse_attn" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in seer.h but not exported"
+    assert sorted(B.EXPORTS) == names, "binding.EXPORTS and seer.h disagree"
+
+
+def test_sizing_helpers_closed_forms(lib):
+    s = B.make_shape([0, 131072], 32, 8)
+    assert B.seer_mask_rows(s) == 32 * 2048
+    assert B.seer_scores_elems(s) == 32 * 2048 * 2048
+    assert B.seer_causal_blocks(s) == 32 * 2048 * 2049 // 2 == 67141632
+    assert B.seer_workspace_bytes(s) == (32 + 8) * 2048 * 128 * 4
+    v = B.make_shape([0, 8192, 8192 + 16384, 8192 + 16384 + 32768, 122880], 40, 8)
+    assert B.seer_mask_rows(v) == 40 * (128 + 256 + 512 + 1024) == 76800
+    assert B.seer_causal_blocks(v) == 27891200
+    r = B.make_shape([0, 65, 65, 130], 2, 1)                 # ragged, with an empty sequence
+    assert B.seer_mask_rows(r) == 2 * (2 + 0 + 2) and B.seer_scores_elems(r) == 2 * (4 + 0 + 4)
+    assert B.seer_prefill_host_arena_bytes(s) > 3 * 10 ** 9
+
+
+def test_invalid_shapes_are_rejected_without_a_gpu(lib):
+    assert B.seer_mask_rows(B.make_shape([0, 128], 3, 2)) == -1          # Hq not a multiple of Hkv
+    assert B.seer_mask_rows(B.make_shape([0, 128], 2, 1, head_dim=64)) == -1
+    assert B.seer_mask_rows(B.make_shape([0, 128, 64], 2, 1)) == -1      # decreasing offsets
+    assert B.seer_workspace_bytes(B.make_shape([5, 128], 2, 1)) == 0     # cu[0] != 0
+    assert B.seer_status_string(4) == "col_idx capacity exceeded"
+
+
+def test_context_creation_fails_loudly_without_a_device(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(B.SeerError) as e:
+        B.Context(0)
+    assert e.value.status == 7

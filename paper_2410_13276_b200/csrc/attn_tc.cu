@@ -38,21 +38,23 @@ constexpr uint32_t kQBytes = 2 * kHalfQ;         // 16 KB
 constexpr uint32_t kKVBytes = 2 * kHalfKV;       // 32 KB (K or V tile of 128 keys)
 constexpr uint32_t kPBytes = 128 * 128;          // 16 KB  P^T [128 keys][64 q] bf16
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQ = 0;                                     // 2 x 16 KB (items alternate)
-constexpr uint32_t kOffK = kOffQ + 2 * kQBytes;                   // 2 x 32 KB ring
-constexpr uint32_t kOffV = kOffK + 2 * kKVBytes;                  // 2 x 32 KB ring
-constexpr uint32_t kOffP = kOffV + 2 * kKVBytes;                  // 2 x 16 KB, one per softmax group (also epilogue staging)
+constexpr int kKSlots = 3, kVSlots = 2;
+constexpr uint32_t kOffQ = 0;                                     // 16 KB
+constexpr uint32_t kOffK = kOffQ + kQBytes;                       // kKSlots x 32 KB ring
+constexpr uint32_t kOffV = kOffK + kKSlots * kKVBytes;            // kVSlots x 32 KB ring
+constexpr uint32_t kOffP = kOffV + kVSlots * kKVBytes;            // 2 x 16 KB, one per softmax group (also epilogue staging)
 constexpr uint32_t kOffGrp = kOffP + 2 * kPBytes;                 // per-group small arrays
 constexpr uint32_t kGrpMref = 0, kGrpAlpha = 256, kGrpColmax = 512, kGrpLfin = 768, kGrpLsum = 1024;   // lsum: 4 x 64 floats
 constexpr uint32_t kGrpBytes = 2048;
 constexpr uint32_t kOffW = kOffGrp + 2 * kGrpBytes;               // merge weights wA[64], wB[64]
 constexpr uint32_t kOffBar = kOffW + 512;                         // mbarriers
-constexpr uint32_t kNumBars = 24;
+constexpr uint32_t kNumBars = 28;
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag
 constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;             // + alignment slack
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
-enum Bar { Q_FULL = 0, Q_EMPTY = 2, K_FULL = 4, K_EMPTY = 6, V_FULL = 8, V_EMPTY = 10, S_FULL = 12 /* + 2*group + buf */,
-           S_EMPTY = 16, P_FULL = 20 /* + group */, PV_DONE = 22 };
+enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /* + slot */, K_EMPTY = 5, V_FULL = 8, V_EMPTY = 10,
+           S_FULL = 12 /* + 2*group + buf */, S_EMPTY = 16, P_FULL = 20 /* + group */, PV_DONE = 22 };
 
 constexpr uint32_t kTmemCols = 512;
 __device__ __forceinline__ uint32_t col_s(int group, uint32_t buf) { return (uint32_t)group * 192u + buf * 64u; }
@@ -280,19 +282,37 @@ __device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out
   base = ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
 }
 
+// Optional timeline of CTA 0 (diagnostics): role r appends (tag << 32 | ordinal, clock) pairs to trace[r * 8192 ...].
+struct Tracer {
+  unsigned long long* p;
+  uint32_t n;
+  __device__ __forceinline__ void init(unsigned long long* base, int role) {
+    p = (base != nullptr && blockIdx.x == 0) ? base + (size_t)role * 8192 : nullptr;
+    n = 0;
+  }
+  __device__ __forceinline__ void ev(uint32_t tag, uint32_t ord) {
+    if (p != nullptr && n < 4095) {
+      p[2 * n] = ((unsigned long long)tag << 32) | ord;
+      p[2 * n + 1] = (unsigned long long)clock64();
+      ++n;
+    }
+  }
+};
+
 // One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]).
 //   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the largest exponent seen.
 //   SUBTRACT == true : removes p from l[c] again (used before a rebase; pk is not touched).
 // MASKED applies the causal mask of a diagonal block / drops a dead row.
 template <bool MASKED, bool SUBTRACT>
 __device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __restrict__ mref, float sl2, bool row_live,
-                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32]) {
+                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32], Tracer* tr = nullptr) {
   float xmax = -CUDART_INF_F;
   uint32_t sv[2][16];
   tc_ld16(s_addr, sv[0]);
 #pragma unroll
   for (int ch = 0; ch < 4; ++ch) {
     tc_wait_ld(sv[ch & 1]);
+    if (tr) tr->ev(40 + ch, 0);
     if (ch < 3) tc_ld16(s_addr + (ch + 1) * 16, sv[(ch + 1) & 1]);
 #pragma unroll
     for (int e = 0; e < 16; e += 4) {
@@ -322,45 +342,13 @@ __device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __re
   return xmax;
 }
 
-// Optional timeline of CTA 0 (diagnostics): role r appends (tag << 32 | ordinal, clock) pairs to trace[r * 8192 ...].
-struct Tracer {
-  unsigned long long* p;
-  uint32_t n;
-  __device__ __forceinline__ void init(unsigned long long* base, int role) {
-    p = (base != nullptr && blockIdx.x == 0) ? base + (size_t)role * 8192 : nullptr;
-    n = 0;
-  }
-  __device__ __forceinline__ void ev(uint32_t tag, uint32_t ord) {
-    if (p != nullptr && n < 4095) {
-      p[2 * n] = ((unsigned long long)tag << 32) | ord;
-      p[2 * n + 1] = (unsigned long long)clock64();
-      ++n;
-    }
-  }
-};
-
-// Issues the TMA copies of one 128-key tile (blocks ja, jb of KV head g) into a ring slot.
-__device__ __forceinline__ void load_kv_tile(const CUtensorMap* map, uint32_t dst, uint32_t full_bar, const Item& it, int ja,
-                                             int jb) {
-  const bool has_b = jb != -1;
-  if (ja < 0) ja = 0;                // a rejected entry is replaced by block 0 and masked out in the softmax
-  if (jb < 0) jb = 0;
-  mbar_expect_tx(full_bar, has_b ? kKVBytes : kKVBytes / 2);
-  const int ta = it.s0 + ja * kBlock, tb = it.s0 + jb * kBlock;
-  tma_load_3d(dst, map, full_bar, 0, it.g, ta);
-  tma_load_3d(dst + kHalfKV, map, full_bar, 64, it.g, ta);
-  if (has_b) {
-    tma_load_3d(dst + kHalfQ, map, full_bar, 0, it.g, tb);
-    tma_load_3d(dst + kHalfKV + kHalfQ, map, full_bar, 64, it.g, tb);
-  }
-}
-
 // ------------------------------------------------------------------------------------------------ kernel
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, SeqMeta m, const int32_t* __restrict__ row_ptr,
-               const int32_t* __restrict__ col_idx, uint16_t* __restrict__ o, float* __restrict__ lse,
-               int* __restrict__ status, unsigned long long* __restrict__ trace) {
+               const int32_t* __restrict__ col_idx, const void* __restrict__ k_ptr, const void* __restrict__ v_ptr,
+               uint16_t* __restrict__ o,
+               float* __restrict__ lse, int* __restrict__ status, unsigned long long* __restrict__ trace) {
   extern __shared__ unsigned char smem_raw[];
   Shared sh;
   sh.base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -369,13 +357,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(sh.bar(Q_FULL + i), 1);
-      mbar_init(sh.bar(Q_EMPTY + i), 1);
-      mbar_init(sh.bar(K_FULL + i), 1);
+    mbar_init(sh.bar(Q_FULL), 1);
+    mbar_init(sh.bar(Q_EMPTY), 1);
+    for (int i = 0; i < kKSlots; ++i) {
+      mbar_init(sh.bar(K_FULL + i), 32);     // one arrival per producer lane, when its copies have landed
       mbar_init(sh.bar(K_EMPTY + i), 1);
-      mbar_init(sh.bar(V_FULL + i), 1);
+    }
+    for (int i = 0; i < kVSlots; ++i) {
+      mbar_init(sh.bar(V_FULL + i), 32);
       mbar_init(sh.bar(V_EMPTY + i), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(sh.bar(P_FULL + i), kGroupThreads);
       mbar_init(sh.bar(PV_DONE + i), 1);
     }
@@ -398,94 +390,121 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // Ordinals shared by all roles: k = non-empty items seen by this CTA, g = tiles seen, cnt_a / cnt_b = tiles handed to
   // softmax group A / B.  Every role walks the same items and tiles, so the counters agree without communication.
 
-  // ============================================================================================ K (+Q) producer
-  if (warp == 0) {
-    if (lane == 0) {
-      Tracer tr; tr.init(trace, 0);
-      uint32_t k = 0, g = 0;
-      bool ok = true;
-      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
-        if (it.ntiles == 0) continue;
-        const uint32_t qb = k & 1u;
-        if (!mbar_wait(sh, Q_EMPTY + qb, ((k >> 1) & 1u) ^ 1u, status)) break;
-        mbar_expect_tx(sh.bar(Q_FULL + qb), kQBytes);
-        const int tq = it.s0 + it.i * kBlock;
-        tma_load_3d(sh.base + kOffQ + qb * kQBytes, &map_q, sh.bar(Q_FULL + qb), 0, it.h, tq);
-        tma_load_3d(sh.base + kOffQ + qb * kQBytes + kHalfQ, &map_q, sh.bar(Q_FULL + qb), 64, it.h, tq);
-        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
-        for (int t = 0; t < it.ntiles; ++t, ++g) {
-          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
-          if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
-          const uint32_t st = g & 1u;
-          tr.ev(1, g);
-          if (!mbar_wait(sh, K_EMPTY + st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
-          tr.ev(2, g);
-          load_kv_tile(&map_k, sh.base + kOffK + st * kKVBytes, sh.bar(K_FULL + st), it, ja, jb);
-          ja = na; jb = nb2;
+  // ============================================================================================ K (+Q) and V producers
+  // K and V tiles come through the LSU path (cp.async, 16 bytes per request, all 32 lanes of a warp each).  Measured on
+  // this part: TMA box gathers of 128-byte rows sustain ~41 B/clk per SM and take ~2000 clocks to land under load, while
+  // cp.async sustains ~80 B/clk with about half the latency; neither slows the MMAs.  Each lane writes the 128-byte-swizzled
+  // layout the MMA descriptors expect (rows past the end of the sequence are zero-filled: 0 * x must be 0); completion is
+  // asynchronous: every lane's copies arrive on the slot's mbarrier (count 32) when they have landed.  Q (16 KB per item)
+  // goes by TMA.
+  if (warp == 0 || warp == 2) {
+    const bool is_k = warp == 0;
+    Tracer tr; tr.init(lane == 0 ? trace : nullptr, is_k ? 0 : 2);
+    const unsigned char* __restrict__ xg = reinterpret_cast<const unsigned char*>(is_k ? k_ptr : v_ptr);
+    const size_t row_bytes = (size_t)m.num_kv_heads * kHeadDim * 2;      // bytes between consecutive tokens
+    const int chunk = lane & 15, rsub = lane >> 4;
+    const uint32_t slots = is_k ? (uint32_t)kKSlots : (uint32_t)kVSlots;
+    const uint32_t ring = sh.base + (is_k ? kOffK : kOffV);
+    const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
+    // destination offset of (row = 2 * itc + rsub, this lane's chunk) inside a block half, for itc mod 4 = 0..3
+    uint32_t doff[4];
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+      const int row = 2 * q4 + rsub;
+      doff[q4] = (uint32_t)(chunk >> 3) * kHalfKV + (uint32_t)row * 128u + (uint32_t)(((chunk & 7) ^ (row & 7)) << 4);
+    }
+    uint32_t k = 0, slot = 0, use = 0;     // item ordinal; ring position of the next tile
+    uint32_t g = 0;
+    bool ok = true;
+    for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+      const Item it = decode_item(m, row_ptr, w);
+      if (it.ntiles == 0) continue;
+      if (is_k) {
+        if (!mbar_wait(sh, Q_EMPTY, (k & 1u) ^ 1u, status)) break;
+        if (lane == 0) {
+          mbar_expect_tx(sh.bar(Q_FULL), kQBytes);
+          const int tq = it.s0 + it.i * kBlock;
+          tma_load_3d(sh.base + kOffQ, &map_q, sh.bar(Q_FULL), 0, it.h, tq);
+          tma_load_3d(sh.base + kOffQ + kHalfQ, &map_q, sh.bar(Q_FULL), 64, it.h, tq);
         }
         ++k;
       }
-    }
-  }
-  // ============================================================================================ V producer
-  else if (warp == 2) {
-    if (lane == 0) {
-      Tracer tr; tr.init(trace, 2);
-      uint32_t g = 0;
-      bool ok = true;
-      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
-        if (it.ntiles == 0) continue;
-        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
-        for (int t = 0; t < it.ntiles; ++t, ++g) {
-          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
-          const uint32_t st = g & 1u;
-          tr.ev(3, g);
-          if (!mbar_wait(sh, V_EMPTY + st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
-          tr.ev(4, g);
-          load_kv_tile(&map_v, sh.base + kOffV + st * kKVBytes, sh.bar(V_FULL + st), it, ja, jb);
-          ja = na; jb = nb2;
+      int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
+      const unsigned char* seq_base = xg + ((size_t)it.s0 * m.num_kv_heads + it.g) * (kHeadDim * 2) + (size_t)chunk * 16 +
+                                      (size_t)rsub * row_bytes;
+      for (int t = 0; t < it.ntiles; ++t, ++g) {
+        const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
+        if (is_k && lane == 0 && (ja == -2 || jb == -2)) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
+        tr.ev(is_k ? 1 : 3, g);
+        if (!mbar_wait(sh, empty0 + (int)slot, (use & 1u) ^ 1u, status)) { ok = false; break; }
+        tr.ev(is_k ? 2 : 4, g);
+        const uint32_t dst0 = ring + slot * kKVBytes;
+#pragma unroll 1
+        for (int half_tile = 0; half_tile < 2; ++half_tile) {
+          int j = half_tile ? jb : ja;
+          if (j == -1) continue;                       // odd list: no second block
+          if (j < 0) j = 0;                            // rejected entry: any valid block, masked out in the softmax
+          const int rows_valid = it.slen - j * kBlock;
+          const unsigned char* src = seq_base + (size_t)j * kBlock * row_bytes;
+          const uint32_t dst = dst0 + (uint32_t)half_tile * 8192u;
+          if (rows_valid >= kBlock) {
+#pragma unroll 8
+            for (int itc = 0; itc < 32; ++itc)
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + doff[itc & 3] + (uint32_t)(itc >> 2) * 1024u),
+                           "l"(src + (size_t)(2 * itc) * row_bytes) : "memory");
+          } else {
+#pragma unroll 8
+            for (int itc = 0; itc < 32; ++itc) {
+              const bool valid = 2 * itc + rsub < rows_valid;
+              const int sz = valid ? 16 : 0;
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + doff[itc & 3] + (uint32_t)(itc >> 2) * 1024u),
+                           "l"(valid ? src + (size_t)(2 * itc) * row_bytes : seq_base), "r"(sz) : "memory");
+            }
+          }
         }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sh.bar(full0 + (int)slot)) : "memory");
+        if (++slot == slots) { slot = 0; ++use; }
+        ja = na; jb = nb2;
       }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");   // nothing of this warp is in flight when the CTA ends
   }
   // ============================================================================================ S^T issuer
   else if (warp == 1) {
     if (lane == 0) {
       Tracer tr; tr.init(trace, 1);
-      uint32_t k = 0, g = 0, cnt_a = 0, cnt_b = 0;
+      uint32_t k = 0, g = 0, cnt_a = 0, cnt_b = 0, slot = 0, use = 0;
       // descriptor bases; per K-step the start address advances by 32 bytes inside a 64-element swizzle atom and by
       // one d-half (16 KB / 8 KB) between atoms
-      const uint64_t kd0 = make_desc(sh.base + kOffK, 16, 1024), kd1 = make_desc(sh.base + kOffK + kKVBytes, 16, 1024);
-      const uint64_t qd0 = make_desc(sh.base + kOffQ, 16, 1024), qd1 = make_desc(sh.base + kOffQ + kQBytes, 16, 1024);
+      const uint64_t kd0 = make_desc(sh.base + kOffK, 16, 1024);
+      const uint64_t qd = make_desc(sh.base + kOffQ, 16, 1024);
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
         const Item it = decode_item(m, row_ptr, w);
         if (it.ntiles == 0) continue;
-        const uint32_t qb = k & 1u;
-        if (!mbar_wait(sh, Q_FULL + qb, (k >> 1) & 1u, status)) break;
-        const uint64_t qd = qb ? qd1 : qd0;
+        if (!mbar_wait(sh, Q_FULL, k & 1u, status)) break;
         for (int t = 0; t < it.ntiles; ++t, ++g) {
           const int grp = t & 1;
-          const uint32_t cn = grp ? cnt_b : cnt_a, buf = cn & 1u, st = g & 1u;
+          const uint32_t cn = grp ? cnt_b : cnt_a, buf = cn & 1u;
           tr.ev(10, g);
-          if (!mbar_wait(sh, K_FULL + st, (g >> 1) & 1u, status)) { ok = false; break; }
+          if (!mbar_wait(sh, K_FULL + (int)slot, use & 1u, status)) { ok = false; break; }
           tr.ev(11, g);
           if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
           tr.ev(12, g);
+          fence_async_smem();     // K was written through the generic proxy (cp.async); the MMA reads through the async proxy
           tc_fence_after();
-          const uint64_t kd = st ? kd1 : kd0;
+          const uint64_t kd = kd0 + (uint64_t)(slot * (kKVBytes >> 4));
           const uint32_t d = tmem + col_s(grp, buf);
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
             tc_mma(d, kd + (uint64_t)((kk >> 2) * (kHalfKV >> 4) + (kk & 3) * 2),
                    qd + (uint64_t)((kk >> 2) * (kHalfQ >> 4) + (kk & 3) * 2), kIdescS, kk > 0);
           tc_commit(sh.bar(S_FULL + 2 * grp + buf));
-          tc_commit(sh.bar(K_EMPTY + st));
-          if (t == it.ntiles - 1) tc_commit(sh.bar(Q_EMPTY + qb));   // last S^T of the item: Q may be replaced
+          tc_commit(sh.bar(K_EMPTY + (int)slot));
+          if (t == it.ntiles - 1) tc_commit(sh.bar(Q_EMPTY));   // last S^T of the item: Q may be replaced
           tr.ev(17, g);
           if (grp) ++cnt_b; else ++cnt_a;
+          if (++slot == (uint32_t)kKSlots) { slot = 0; ++use; }
         }
         ++k;
       }
@@ -509,6 +528,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tr.ev(14, g);
           if (!mbar_wait(sh, P_FULL + grp, cn & 1u, status)) { ok = false; break; }
           tr.ev(15, g);
+          fence_async_smem();     // V was written through the generic proxy (cp.async); the MMA reads through the async proxy
           tc_fence_after();
           const uint64_t vd = st ? vd1 : vd0, pd = grp ? pd1 : pd0;
           const uint32_t d = tmem + col_o(grp);
@@ -567,16 +587,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (gt < 64) mref[gt] = -CUDART_INF_F;
       named_bar_sync(bar_sync, kGroupThreads);
 
+      int nja = list_block(it, col_idx, 2 * grp), njb = list_block(it, col_idx, 2 * grp + 1);
       for (int t = grp; t < it.ntiles; t += 2, ++cnt) {
         const uint32_t sbuf = cnt & 1u;
         tr.ev(20, gbase + t);
         bool fail = !mbar_wait(sh, S_FULL + 2 * grp + sbuf, (cnt >> 1) & 1u, status);
         tr.ev(21, gbase + t);
-        // the previous P V of this group has finished: its P^T buffer and the O^T accumulator may be touched
-        if (!fail && cnt > 0) fail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
         tc_fence_after();
-        tr.ev(22, gbase + t);
-        const int ja = list_block(it, col_idx, 2 * t), jb = list_block(it, col_idx, 2 * t + 1);
+        const int ja = nja, jb = njb;
+        nja = list_block(it, col_idx, 2 * t + 4); njb = list_block(it, col_idx, 2 * t + 5);   // this group's next tile
         const int my_j = r < 64 ? ja : jb;
         const bool row_live = my_j >= 0;                 // absent / rejected blocks contribute nothing
         const bool diag = my_j == it.i;
@@ -584,9 +603,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t s_addr = tmem + lane_addr + col_s(grp, sbuf);
         uint32_t pk[32];
         float xmax = -CUDART_INF_F;
-        if (!fail) xmax = masked ? softmax_pass<true, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk)
-                                 : softmax_pass<false, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+        if (!fail) xmax = masked ? softmax_pass<true, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk, &tr)
+                                 : softmax_pass<false, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk, &tr);
         tr.ev(23, gbase + t);
+        // the previous P V of this group must have finished before its P^T buffer (and, when rebasing, its O^T accumulator)
+        // is touched; by now it normally has
+        if (!fail && cnt > 0) fail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
+        tc_fence_after();
+        tr.ev(22, gbase + t);
         // one vote per tile: does any entry exceed its reference by more than 2^8 (or has a wait been lost)?
         const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || xmax > 8.f);
         tr.ev(24, gbase + t);
@@ -656,17 +680,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const uint32_t a = prow + (uint32_t)((ck ^ (r & 7)) << 4);
             asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(pk[ck * 4]), "r"(pk[ck * 4 + 1]),
                          "r"(pk[ck * 4 + 2]), "r"(pk[ck * 4 + 3]) : "memory");
-          }
-          // ragged last block of a sequence: its V rows past the end belong to someone else -> zero them (0 * x must be 0)
-          if (row_live && my_j * kBlock + key_local >= it.slen) {
-            const uint32_t g = gbase + (uint32_t)t, vs = g & 1u;      // ring slot of this tile's V
-            mbar_wait(sh, V_FULL + vs, (g >> 1) & 1u, status);        // the copy has landed (a lost wait raises the abort flag)
-            const uint32_t vrow = sh.base + kOffV + vs * kKVBytes + (uint32_t)r * 128u;
-#pragma unroll
-            for (int ck = 0; ck < 8; ++ck) {
-              asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vrow + ck * 16), "r"(0u) : "memory");
-              asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vrow + kHalfKV + ck * 16), "r"(0u) : "memory");
-            }
           }
         }
         fence_async_smem();
@@ -792,7 +805,7 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
       !tc::make_map(ctx, &mv, v, m.total_tokens, m.num_kv_heads))
     return -(int)cudaErrorInvalidValue;
   const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, m.rows);
-  tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse,
+  tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
                                                                     ctx->d_status, (unsigned long long*)ctx->trace);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;

@@ -14,9 +14,11 @@
 // work group computes exact column maxima, rebases m, rescales its partial sums and the O accumulator, and recomputes
 // the tile.  Row sums are per-thread partials combined once per work item.
 //
-// Roles (384 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + issuer of the S^T MMAs, warp 2 = TMA
-// producer for V, warp 3 = issuer of the P V MMAs (one thread can start a tcgen05.mma only every 64 clocks, so the two
-// products are issued from two threads), warps 4-7 and 8-11 = two softmax groups.  The tiles of a work item alternate between the groups (even tiles -> A, odd -> B); each group keeps its own
+// Roles (512 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + issuer of the S^T MMAs, warp 3 = issuer
+// of the P V MMAs (one thread can start a tcgen05.mma only every 64 clocks, so the two products are issued from two
+// threads), warps 4-7 and 8-11 = two softmax groups, warps 12-15 = cp.async producers for V (a warp keeps only ~14 KB of
+// cp.async in flight, so four share a tile).  After the dispatch the helper warpgroups shrink to 72 registers per thread
+// and the softmax warpgroups grow to 184 (setmaxnreg).  The tiles of a work item alternate between the groups (even tiles -> A, odd -> B); each group keeps its own
 // S^T buffers, P^T buffer, O^T accumulator, references and row sums, and the epilogue merges the two partial results
 // through their references.  One persistent CTA per SM walks the work items (longest rows first within each KV head).
 // Every wait is bounded; a wait that runs out raises SEER_ERR_TIMEOUT and the CTA drains and exits.
@@ -30,7 +32,9 @@
 namespace seer {
 namespace tc {
 
-constexpr int kThreads = 384;               // warps 0-3: K(+Q) producer, S^T issuer, V producer, P V issuer; warps 4-7 / 8-11: softmax groups A / B
+constexpr int kThreads = 512;               // warps 0-3: K(+Q) producer, S^T issuer, -, P V issuer; 4-7 / 8-11: softmax groups A / B; 12-15: V producers
+constexpr int kVProducerWarps = 4;
+constexpr int kHelperRegs = 72, kSoftmaxRegs = 184;   // register split after the role dispatch: (2 * 72 + 2 * 184) * 128 = 65536
 constexpr int kGroupThreads = 128;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
@@ -360,11 +364,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     mbar_init(sh.bar(Q_FULL), 1);
     mbar_init(sh.bar(Q_EMPTY), 1);
     for (int i = 0; i < kKSlots; ++i) {
-      mbar_init(sh.bar(K_FULL + i), 32);     // one arrival per producer lane, when its copies have landed
+      mbar_init(sh.bar(K_FULL + i), 1);
       mbar_init(sh.bar(K_EMPTY + i), 1);
     }
     for (int i = 0; i < kVSlots; ++i) {
-      mbar_init(sh.bar(V_FULL + i), 32);
+      mbar_init(sh.bar(V_FULL + i), 32 * kVProducerWarps);   // one arrival per producer lane, when its copies have landed
       mbar_init(sh.bar(V_EMPTY + i), 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -390,80 +394,102 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // Ordinals shared by all roles: k = non-empty items seen by this CTA, g = tiles seen, cnt_a / cnt_b = tiles handed to
   // softmax group A / B.  Every role walks the same items and tiles, so the counters agree without communication.
 
-  // ============================================================================================ K (+Q) and V producers
-  // K and V tiles come through the LSU path (cp.async, 16 bytes per request, all 32 lanes of a warp each).  Measured on
-  // this part: TMA box gathers of 128-byte rows sustain ~41 B/clk per SM and take ~2000 clocks to land under load, while
-  // cp.async sustains ~80 B/clk with about half the latency; neither slows the MMAs.  Each lane writes the 128-byte-swizzled
-  // layout the MMA descriptors expect (rows past the end of the sequence are zero-filled: 0 * x must be 0); completion is
-  // asynchronous: every lane's copies arrive on the slot's mbarrier (count 32) when they have landed.  Q (16 KB per item)
-  // goes by TMA.
-  if (warp == 0 || warp == 2) {
-    const bool is_k = warp == 0;
-    Tracer tr; tr.init(lane == 0 ? trace : nullptr, is_k ? 0 : 2);
-    const unsigned char* __restrict__ xg = reinterpret_cast<const unsigned char*>(is_k ? k_ptr : v_ptr);
+  // Register split: the two helper warpgroups (warps 0-3, 12-15) give registers up, the softmax warpgroups take them.
+  if (warp < 4 || warp >= 12) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
+  // ============================================================================================ K (+Q) producer (TMA)
+  if (warp == 0) {
+    if (lane == 0) {
+      Tracer tr; tr.init(trace, 0);
+      uint32_t k = 0, g = 0, slot = 0, use = 0;
+      bool ok = true;
+      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
+        const Item it = decode_item(m, row_ptr, w);
+        if (it.ntiles == 0) continue;
+        if (!mbar_wait(sh, Q_EMPTY, (k & 1u) ^ 1u, status)) break;
+        mbar_expect_tx(sh.bar(Q_FULL), kQBytes);
+        const int tq = it.s0 + it.i * kBlock;
+        tma_load_3d(sh.base + kOffQ, &map_q, sh.bar(Q_FULL), 0, it.h, tq);
+        tma_load_3d(sh.base + kOffQ + kHalfQ, &map_q, sh.bar(Q_FULL), 64, it.h, tq);
+        ++k;
+        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
+        for (int t = 0; t < it.ntiles; ++t, ++g) {
+          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
+          if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
+          tr.ev(1, g);
+          if (!mbar_wait(sh, K_EMPTY + (int)slot, (use & 1u) ^ 1u, status)) { ok = false; break; }
+          tr.ev(2, g);
+          const bool has_b = jb != -1;
+          const int xa = ja < 0 ? 0 : ja, xb = jb < 0 ? 0 : jb;   // a rejected entry: any valid block, masked out in the softmax
+          const uint32_t fb = sh.bar(K_FULL + (int)slot), dst = sh.base + kOffK + slot * kKVBytes;
+          mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
+          const int ta = it.s0 + xa * kBlock, tb = it.s0 + xb * kBlock;
+          tma_load_3d(dst, &map_k, fb, 0, it.g, ta);
+          tma_load_3d(dst + kHalfKV, &map_k, fb, 64, it.g, ta);
+          if (has_b) {
+            tma_load_3d(dst + kHalfQ, &map_k, fb, 0, it.g, tb);
+            tma_load_3d(dst + kHalfKV + kHalfQ, &map_k, fb, 64, it.g, tb);
+          }
+          if (++slot == (uint32_t)kKSlots) { slot = 0; ++use; }
+          ja = na; jb = nb2;
+        }
+      }
+    }
+  }
+  // ============================================================================================ V producers (cp.async)
+  // V tiles come through the LSU path (cp.async, 16 bytes per request).  Measured on this part: TMA box gathers of
+  // 128-byte rows sustain ~41 B/clk per SM, cp.async ~80, both together ~85 (the SM's fill limit) and neither slows the
+  // MMAs, so K goes by TMA and V by cp.async.  Producer warp pw copies rows 16 pw .. 16 pw + 15 of each block of the tile;
+  // each lane writes the 128-byte-swizzled layout the MMA descriptor expects (rows past the end of the sequence are
+  // zero-filled: 0 * x must be 0); completion is asynchronous: every lane's copies arrive on the slot's mbarrier when they
+  // have landed.
+  else if (warp >= 12) {
+    const int pw = warp - 12;
+    Tracer tr; tr.init(lane == 0 && pw == 0 ? trace : nullptr, 2);
+    const unsigned char* __restrict__ xg = reinterpret_cast<const unsigned char*>(v_ptr);
     const size_t row_bytes = (size_t)m.num_kv_heads * kHeadDim * 2;      // bytes between consecutive tokens
     const int chunk = lane & 15, rsub = lane >> 4;
-    const uint32_t slots = is_k ? (uint32_t)kKSlots : (uint32_t)kVSlots;
-    const uint32_t ring = sh.base + (is_k ? kOffK : kOffV);
-    const int full0 = is_k ? K_FULL : V_FULL, empty0 = is_k ? K_EMPTY : V_EMPTY;
-    // destination offset of (row = 2 * itc + rsub, this lane's chunk) inside a block half, for itc mod 4 = 0..3
+    const int row0 = pw * (kBlock / kVProducerWarps);                    // first row of this warp's share of a block
+    constexpr int kIters = kBlock / kVProducerWarps / 2;                 // 2 rows per warp instruction
+    // destination offset of (row0 + 2 * itc + rsub, this lane's chunk) inside a block half, for itc mod 4 = 0..3
     uint32_t doff[4];
 #pragma unroll
     for (int q4 = 0; q4 < 4; ++q4) {
       const int row = 2 * q4 + rsub;
-      doff[q4] = (uint32_t)(chunk >> 3) * kHalfKV + (uint32_t)row * 128u + (uint32_t)(((chunk & 7) ^ (row & 7)) << 4);
+      doff[q4] = (uint32_t)(chunk >> 3) * kHalfKV + (uint32_t)(row0 + row) * 128u + (uint32_t)(((chunk & 7) ^ (row & 7)) << 4);
     }
-    uint32_t k = 0, slot = 0, use = 0;     // item ordinal; ring position of the next tile
     uint32_t g = 0;
     bool ok = true;
     for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
       const Item it = decode_item(m, row_ptr, w);
       if (it.ntiles == 0) continue;
-      if (is_k) {
-        if (!mbar_wait(sh, Q_EMPTY, (k & 1u) ^ 1u, status)) break;
-        if (lane == 0) {
-          mbar_expect_tx(sh.bar(Q_FULL), kQBytes);
-          const int tq = it.s0 + it.i * kBlock;
-          tma_load_3d(sh.base + kOffQ, &map_q, sh.bar(Q_FULL), 0, it.h, tq);
-          tma_load_3d(sh.base + kOffQ + kHalfQ, &map_q, sh.bar(Q_FULL), 64, it.h, tq);
-        }
-        ++k;
-      }
       int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
       const unsigned char* seq_base = xg + ((size_t)it.s0 * m.num_kv_heads + it.g) * (kHeadDim * 2) + (size_t)chunk * 16 +
-                                      (size_t)rsub * row_bytes;
+                                      (size_t)(row0 + rsub) * row_bytes;
       for (int t = 0; t < it.ntiles; ++t, ++g) {
         const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
-        if (is_k && lane == 0 && (ja == -2 || jb == -2)) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
-        tr.ev(is_k ? 1 : 3, g);
-        if (!mbar_wait(sh, empty0 + (int)slot, (use & 1u) ^ 1u, status)) { ok = false; break; }
-        tr.ev(is_k ? 2 : 4, g);
-        const uint32_t dst0 = ring + slot * kKVBytes;
+        const uint32_t st = g & 1u;
+        tr.ev(3, g);
+        if (!mbar_wait(sh, V_EMPTY + (int)st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
+        tr.ev(4, g);
+        const uint32_t dst0 = sh.base + kOffV + st * kKVBytes;
 #pragma unroll 1
         for (int half_tile = 0; half_tile < 2; ++half_tile) {
           int j = half_tile ? jb : ja;
           if (j == -1) continue;                       // odd list: no second block
           if (j < 0) j = 0;                            // rejected entry: any valid block, masked out in the softmax
-          const int rows_valid = it.slen - j * kBlock;
+          const int rows_valid = it.slen - j * kBlock - row0 - rsub;   // this lane's rows 2 * itc below this are real
           const unsigned char* src = seq_base + (size_t)j * kBlock * row_bytes;
           const uint32_t dst = dst0 + (uint32_t)half_tile * 8192u;
-          if (rows_valid >= kBlock) {
-#pragma unroll 8
-            for (int itc = 0; itc < 32; ++itc)
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + doff[itc & 3] + (uint32_t)(itc >> 2) * 1024u),
-                           "l"(src + (size_t)(2 * itc) * row_bytes) : "memory");
-          } else {
-#pragma unroll 8
-            for (int itc = 0; itc < 32; ++itc) {
-              const bool valid = 2 * itc + rsub < rows_valid;
-              const int sz = valid ? 16 : 0;
-              asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + doff[itc & 3] + (uint32_t)(itc >> 2) * 1024u),
-                           "l"(valid ? src + (size_t)(2 * itc) * row_bytes : seq_base), "r"(sz) : "memory");
-            }
+#pragma unroll
+          for (int itc = 0; itc < kIters; ++itc) {
+            const bool valid = 2 * itc < rows_valid;
+            const int sz = valid ? 16 : 0;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + doff[itc & 3] + (uint32_t)(itc >> 2) * 1024u),
+                         "l"(valid ? src + (size_t)(2 * itc) * row_bytes : seq_base), "r"(sz) : "memory");
           }
         }
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sh.bar(full0 + (int)slot)) : "memory");
-        if (++slot == slots) { slot = 0; ++use; }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sh.bar(V_FULL + (int)st)) : "memory");
         ja = na; jb = nb2;
       }
     }
@@ -548,8 +574,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   }
+  }   // helper warpgroups
   // ============================================================================================ softmax groups
   else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     const int grp = (warp - 4) >> 2;                     // 0 = A (even tiles), 1 = B (odd tiles)
     const int gt = threadIdx.x - 128 - grp * kGroupThreads;   // 0..127 within the group
     const int gw = (warp - 4) & 3;                       // warp within the group

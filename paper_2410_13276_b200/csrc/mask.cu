@@ -3,8 +3,9 @@
 //   scan_kernel  : exclusive prefix sum of the counts -> row_ptr, nnz, capacity check
 //   fill_kernel  : one warp per row repeats the selection and writes the ascending list by ballot compaction
 // Selection order in the TopK modes is (score descending, block index ascending): scores become order-preserving
-// 32-bit keys, the key of the last kept candidate is found by a bitwise search over the row held in shared
-// memory, and ties at that key are resolved by rank in index order.
+// 32-bit keys, the key of the last kept candidate is found by a radix select over the row held in shared memory (four
+// 8-bit passes with warp-private histograms; rows too long to stage fall back to a bitwise search that re-reads the
+// scores), and ties at that key are resolved by rank in index order.
 #include "seer_internal.cuh"
 
 namespace seer {
@@ -122,6 +123,7 @@ __global__ void __launch_bounds__(kMaskWarps * 32)
 fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, const int32_t* __restrict__ row_ptr,
             int32_t* __restrict__ col_idx, int64_t col_capacity, int stage_cap) {
   extern __shared__ uint32_t key_smem[];
+  uint32_t* hist_smem = key_smem + (size_t)kMaskWarps * stage_cap;   // 256 bins per warp
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t r = (int64_t)blockIdx.x * kMaskWarps + warp;
   const RowInfo ri = decode_row(m, scores, r);
@@ -167,6 +169,52 @@ fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, con
     T = 0u; need_eq = 0;            // every candidate is kept (key >= 1 > 0)
   } else if (take == 0) {
     T = 0xffffffffu; need_eq = 0;   // nothing beyond the forced blocks
+  } else if (staged) {
+    // Radix select, 8 bits per pass from the top: histogram the current digit of the keys that match the prefix found
+    // so far (warp-private shared-memory bins), walk the bins from the largest digit down until `remaining` is covered.
+    uint32_t* hist = hist_smem + warp * 256;
+    uint32_t prefix = 0u, prefix_mask = 0u;
+    int remaining = take;           // rank (1-based, from the top) still to locate inside the current prefix class
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int b = lane; b < 256; b += 32) hist[b] = 0u;
+      __syncwarp();
+      for (int j = lane; j < n; j += 32) {
+        const uint32_t kk = keys[j];
+        if (kk != 0u && (kk & prefix_mask) == prefix) atomicAdd(&hist[(kk >> shift) & 255u], 1u);
+      }
+      __syncwarp();
+      // lane l owns digits 8l .. 8l+7; suffix sums over lanes give the number of keys with a larger digit
+      uint32_t c[8], lane_total = 0u;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { c[e] = hist[lane * 8 + e]; lane_total += c[e]; }
+      uint32_t above = lane_total;                       // inclusive suffix sum over lanes >= this lane
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
+        if (lane + o < 32) above += v;
+      }
+      above -= lane_total;                               // keys in lanes with larger digits
+      // the digit holding rank `remaining` lies in the lane where above < remaining <= above + lane_total
+      const bool mine = (int)above < remaining && remaining <= (int)(above + lane_total);
+      uint32_t digit = 0u; int new_remaining = 0;
+      if (mine) {
+        uint32_t acc = above;
+#pragma unroll
+        for (int e = 7; e >= 0; --e) {
+          if ((int)acc < remaining && remaining <= (int)(acc + c[e])) { digit = (uint32_t)(lane * 8 + e); new_remaining = remaining - (int)acc; }
+          acc += c[e];
+        }
+      }
+      const uint32_t owner = __ballot_sync(0xffffffffu, mine);
+      const int src = __ffs(owner) - 1;
+      digit = __shfl_sync(0xffffffffu, digit, src);
+      remaining = __shfl_sync(0xffffffffu, new_remaining, src);
+      prefix |= digit << shift;
+      prefix_mask |= 255u << shift;
+      __syncwarp();
+    }
+    T = prefix;                      // the take-th largest key; `remaining` of the keys equal to it are kept
+    need_eq = remaining;
   } else {
     for (int bit = 31; bit >= 0; --bit) {
       const uint32_t cand = T | (1u << bit);
@@ -204,7 +252,7 @@ int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer
   count_kernel<<<grid, kMaskWarps * 32, 0, stream>>>(m, scores, p, row_ptr);
   scan_kernel<<<1, 1024, 0, stream>>>(m.rows, row_ptr, col_capacity, nnz_out, ctx->d_status);
   const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // longer rows re-read their scores instead
-  const size_t smem = (size_t)kMaskWarps * stage_cap * sizeof(uint32_t);
+  const size_t smem = (size_t)kMaskWarps * (stage_cap + 256) * sizeof(uint32_t);
   fill_kernel<<<grid, kMaskWarps * 32, smem, stream>>>(m, scores, p, row_ptr, col_idx, col_capacity, stage_cap);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 3 : -(int)e;
@@ -213,7 +261,7 @@ int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer
 seer_status init_mask(seer_ctx* ctx) {
   (void)ctx;
   cudaError_t e = cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kMaskWarps * kMaskSmemRowMax * (int)sizeof(uint32_t));
+                                       kMaskWarps * (kMaskSmemRowMax + 256) * (int)sizeof(uint32_t));
   return e == cudaSuccess ? SEER_OK : SEER_ERR_CUDA;
 }
 

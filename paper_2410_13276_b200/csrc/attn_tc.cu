@@ -54,7 +54,8 @@ constexpr uint32_t kOffW = kOffGrp + 2 * kGrpBytes;               // merge weigh
 constexpr uint32_t kOffBar = kOffW + 512;                         // mbarriers
 constexpr uint32_t kNumBars = 28;
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag
-constexpr uint32_t kSmemBytes = kOffMisc + 64 + 1024;             // + alignment slack
+constexpr uint32_t kOffTrace = kOffMisc + 64;                     // diagnostics: 6 roles x 48 tags x (sum, count)
+constexpr uint32_t kSmemBytes = kOffTrace + 6 * 48 * 16 + 1024;   // + alignment slack
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /* + slot */, K_EMPTY = 5, V_FULL = 8, V_EMPTY = 10,
@@ -109,6 +110,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait.  Returns false after the limit (or when another role has already given up); the caller drains.
 __device__ __forceinline__ bool mbar_wait(const Shared& sh, int bar, uint32_t parity, int* status) {
   const uint32_t addr = sh.bar(bar);
+  {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+    if (done) return true;
+  }
   if (mbar_try(addr, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
@@ -286,20 +293,33 @@ __device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out
   base = ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
 }
 
-// Optional timeline of CTA 0 (diagnostics): role r appends (tag << 32 | ordinal, clock) pairs to trace[r * 8192 ...].
+// Optional cycle accounting of CTA 0 (diagnostics): every role attributes the clocks between two consecutive marks to the
+// tag of the later mark, accumulates per tag in shared memory, and writes the sums and mark counts to
+// trace[role * 8192 + tag * 2 ...] when it ends.
+constexpr int kTraceTags = 48;
 struct Tracer {
-  unsigned long long* p;
-  uint32_t n;
-  __device__ __forceinline__ void init(unsigned long long* base, int role) {
+  unsigned long long* p;      // global destination (nullptr: off)
+  unsigned long long* acc;    // shared accumulators of this role: [tag][sum, count]
+  long long last;
+  __device__ __forceinline__ void init(unsigned long long* base, int role, unsigned char* smem_trace) {
     p = (base != nullptr && blockIdx.x == 0) ? base + (size_t)role * 8192 : nullptr;
-    n = 0;
-  }
-  __device__ __forceinline__ void ev(uint32_t tag, uint32_t ord) {
-    if (p != nullptr && n < 4095) {
-      p[2 * n] = ((unsigned long long)tag << 32) | ord;
-      p[2 * n + 1] = (unsigned long long)clock64();
-      ++n;
+    acc = reinterpret_cast<unsigned long long*>(smem_trace) + role * kTraceTags * 2;
+    if (p != nullptr) {
+      for (int i = 0; i < kTraceTags * 2; ++i) acc[i] = 0;
+      last = clock64();
     }
+  }
+  __device__ __forceinline__ void ev(uint32_t tag, uint32_t) {
+    if (p != nullptr) {
+      const long long now = clock64();
+      acc[2 * tag] += (unsigned long long)(now - last);
+      acc[2 * tag + 1] += 1;
+      last = clock64();
+    }
+  }
+  __device__ __forceinline__ void flush() {
+    if (p != nullptr)
+      for (int i = 0; i < kTraceTags * 2; ++i) p[i] = acc[i];
   }
 };
 
@@ -400,7 +420,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // ============================================================================================ K (+Q) producer (TMA)
   if (warp == 0) {
     if (lane == 0) {
-      Tracer tr; tr.init(trace, 0);
+      Tracer tr; tr.init(trace, 0, smem + kOffTrace);
       uint32_t k = 0, g = 0, slot = 0, use = 0;
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
@@ -434,6 +454,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           ja = na; jb = nb2;
         }
       }
+      tr.flush();
     }
   }
   // ============================================================================================ V producers (cp.async)
@@ -445,7 +466,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // have landed.
   else if (warp >= 12) {
     const int pw = warp - 12;
-    Tracer tr; tr.init(lane == 0 && pw == 0 ? trace : nullptr, 2);
+    Tracer tr; tr.init(lane == 0 && pw == 0 ? trace : nullptr, 2, smem + kOffTrace);
     const unsigned char* __restrict__ xg = reinterpret_cast<const unsigned char*>(v_ptr);
     const size_t row_bytes = (size_t)m.num_kv_heads * kHeadDim * 2;      // bytes between consecutive tokens
     const int chunk = lane & 15, rsub = lane >> 4;
@@ -494,11 +515,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");   // nothing of this warp is in flight when the CTA ends
+    tr.flush();
   }
   // ============================================================================================ S^T issuer
   else if (warp == 1) {
     if (lane == 0) {
-      Tracer tr; tr.init(trace, 1);
+      Tracer tr; tr.init(trace, 1, smem + kOffTrace);
       uint32_t k = 0, g = 0, cnt_a = 0, cnt_b = 0, slot = 0, use = 0;
       // descriptor bases; per K-step the start address advances by 32 bytes inside a 64-element swizzle atom and by
       // one d-half (16 KB / 8 KB) between atoms
@@ -534,12 +556,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         ++k;
       }
+      tr.flush();
     }
   }
   // ============================================================================================ P V issuer
   else if (warp == 3) {
     if (lane == 0) {
-      Tracer tr; tr.init(trace, 3);
+      Tracer tr; tr.init(trace, 3, smem + kOffTrace);
       uint32_t g = 0, cnt_a = 0, cnt_b = 0;
       const uint64_t vd0 = make_desc(sh.base + kOffV, kHalfKV, 1024), vd1 = make_desc(sh.base + kOffV + kKVBytes, kHalfKV, 1024);
       const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024), pd1 = make_desc(sh.base + kOffP + kPBytes, kHalfKV, 1024);
@@ -572,6 +595,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (grp) ++cnt_b; else ++cnt_a;
         }
       }
+      tr.flush();
     }
   }
   }   // helper warpgroups
@@ -599,7 +623,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int bar_sync = 1 + grp, bar_vote = 3 + grp;
     const float sl2 = m.softmax_scale * 1.4426950408889634f;
     const int key_local = r & 63;
-    Tracer tr; tr.init(gt == 0 ? trace : nullptr, 4 + grp);
+    Tracer tr; tr.init(gt == 0 ? trace : nullptr, 4 + grp, smem + kOffTrace);
     uint32_t cnt = 0;                                    // tiles this group has processed
     uint32_t gbase = 0;                                  // tiles of this CTA before the current item
     bool ok = true;
@@ -700,6 +724,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         // the S^T buffer may be overwritten by a later tile
         tc_fence_before();
         mbar_arrive(sh.bar(S_EMPTY + 2 * grp + sbuf));
+        tr.ev(26, 0);
         // P^T row r -> shared memory (128-byte swizzle)
         {
           const uint32_t prow = sh.base + kOffP + grp * kPBytes + (uint32_t)r * 128u;
@@ -710,7 +735,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                          "r"(pk[ck * 4 + 2]), "r"(pk[ck * 4 + 3]) : "memory");
           }
         }
+        tr.ev(27, 0);
         fence_async_smem();
+        tr.ev(28, 0);
         tc_fence_before();
         mbar_arrive(sh.bar(P_FULL + grp));
         tr.ev(25, gbase + t);
@@ -779,6 +806,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       named_bar_sync(bar_sync, kGroupThreads);   // staging is free again before this group's next P^T
       tr.ev(31, (uint32_t)(w / gridDim.x));
     }
+    tr.flush();
   }
 
   // ------------------------------------------------------------------------------------------------ teardown

@@ -108,6 +108,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait.  Returns false after the limit (or when another role has already given up); the caller drains.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(const Shared& sh, int bar, uint32_t parity, int* status) {
   const uint32_t addr = sh.bar(bar);
   {
@@ -120,6 +121,7 @@ __device__ __forceinline__ bool mbar_wait(const Shared& sh, int bar, uint32_t pa
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try(addr, parity)) return true;
+    if (kSleepNs > 0) __nanosleep(kSleepNs);   // a waiting helper must not take issue slots from the softmax warps of its scheduler
     if ((it & 255u) == 0u) {
       if (ld_shared_u32(sh.abort_flag()) != 0u) return false;
       if (global_ns() - t0 > kWaitLimitNs) break;
@@ -392,12 +394,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(sh.bar(V_EMPTY + i), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(sh.bar(P_FULL + i), kGroupThreads);
+      mbar_init(sh.bar(P_FULL + i), kGroupThreads / 32);   // one arrival per softmax warp
       mbar_init(sh.bar(PV_DONE + i), 1);
     }
     for (int i = 0; i < 4; ++i) {
       mbar_init(sh.bar(S_FULL + i), 1);
-      mbar_init(sh.bar(S_EMPTY + i), kGroupThreads);
+      mbar_init(sh.bar(S_EMPTY + i), kGroupThreads / 32);
     }
     st_shared_u32(sh.abort_flag(), 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -723,7 +725,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         // the S^T buffer may be overwritten by a later tile
         tc_fence_before();
-        mbar_arrive(sh.bar(S_EMPTY + 2 * grp + sbuf));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sh.bar(S_EMPTY + 2 * grp + sbuf));     // one arrival per warp: 128 would serialise on the barrier word
         tr.ev(26, 0);
         // P^T row r -> shared memory (128-byte swizzle)
         {
@@ -739,7 +742,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         fence_async_smem();
         tr.ev(28, 0);
         tc_fence_before();
-        mbar_arrive(sh.bar(P_FULL + grp));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sh.bar(P_FULL + grp));
         tr.ev(25, gbase + t);
       }
       gbase += (uint32_t)it.ntiles;

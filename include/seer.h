@@ -169,9 +169,11 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
 seer_status seer_gate_scores_static(const seer_shape* shape, const void* q, const void* k, const float* Wq,
                                     const float* Wk, float* scores, void* stream);
 
-/* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, CTA 0 of the tcgen05 attention kernel
- * records a timeline of its pipeline roles into it: 6 roles x 4096 (tag << 32 | ordinal, SM clock) pairs of uint64, i.e.
- * at least 6 * 8192 * 8 bytes of device memory, zero-initialised by the caller.  NULL switches it off (default). */
+/* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, the tcgen05 attention kernel runs in an
+ * instrumented instantiation.  CTA 0 adds up the SM clocks its pipeline roles spend between marked points, on every
+ * 8th tile (role r at uint64 offset r * 8192: 48 tags x (clock sum, count)); every CTA writes its wall time in ns at
+ * offset 6 * 8192 + blockIdx.x and in SM clocks at 6 * 8192 + 256 + blockIdx.x.  The buffer is device memory of at
+ * least 7 * 8192 * 8 bytes, zero-initialised by the caller.  NULL switches it off (default). */
 seer_status seer_set_trace_buffer(seer_ctx* ctx, void* device_buffer);
 
 /* Number of kernels the library has launched through this context since creation (for launch accounting). */

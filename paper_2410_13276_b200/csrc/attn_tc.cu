@@ -34,7 +34,8 @@ namespace tc {
 
 constexpr int kThreads = 512;               // warps 0-3: K(+Q) producer, S^T issuer, -, P V issuer; 4-7 / 8-11: softmax groups A / B; 12-15: V producers
 constexpr int kVProducerWarps = 4;
-constexpr int kHelperRegs = 72, kSoftmaxRegs = 184;   // register split after the role dispatch: (2 * 72 + 2 * 184) * 128 = 65536
+constexpr float kRefShift = 7.f;   // softmax references are kept this far (log2) above the column maxima they were taken from
+constexpr int kHelperRegs = 56, kSoftmaxRegs = 200;   // register split after the role dispatch: (2 * 56 + 2 * 200) * 128 = 65536
 constexpr int kGroupThreads = 128;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
@@ -64,6 +65,9 @@ enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /* + slot */, K_EMPTY = 5, V_FULL
 constexpr uint32_t kTmemCols = 512;
 __device__ __forceinline__ uint32_t col_s(int group, uint32_t buf) { return (uint32_t)group * 192u + buf * 64u; }
 __device__ __forceinline__ uint32_t col_o(int group) { return (uint32_t)group * 192u + 128u; }
+// the softmax references of a group, replicated in every lane (a shared-memory read in the inner loop queues behind the
+// operand traffic of the tensor pipe; a TMEM read does not)
+__device__ __forceinline__ uint32_t col_m(int group) { return 384u + (uint32_t)group * 64u; }
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is declared lost
 
@@ -155,6 +159,18 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr) : "memory");
+}
+// Waits for the loads of this thread; the loaded registers are in/out operands so that no use of them moves above it.
+__device__ __forceinline__ void tc_wait_ld8(uint32_t (&a)[8], uint32_t (&b)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7])
+               :: "memory");
+}
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
@@ -164,6 +180,13 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 // Same wait, with the loaded registers as in/out operands so that no use of them can be scheduled above it.
 __device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
+// No instruction: makes the registers of a load issued before the last wait depend on that wait.
+__device__ __forceinline__ void tc_tie(uint32_t (&r)[16]) {
+  asm volatile(""
                : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
                  "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
                :: "memory");
@@ -242,6 +265,15 @@ __device__ __forceinline__ int list_block(const Item& it, const int32_t* __restr
   return (j < 0 || j > it.i) ? -2 : j;
 }
 
+// The same in two steps, so that the load can be issued long before its result is looked at.
+__device__ __forceinline__ int list_fetch(const Item& it, const int32_t* __restrict__ col_idx, int p) {
+  return p < it.nlist ? __ldg(col_idx + it.l0 + p) : -1;
+}
+__device__ __forceinline__ int list_check(const Item& it, int p, int raw) {
+  if (p >= it.nlist) return -1;
+  return (raw < 0 || raw > it.i) ? -2 : raw;
+}
+
 // Sums l[0..63] over the 32 lanes of a warp; lane ends with the totals of columns (2*bitrev-ish) base, base+1
 // where base = 32*b4 + 16*b3 + 8*b2 + 4*b1 + 2*b0 (b_i = bit i of the lane id).
 __device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out0, float& out1, int& base) {
@@ -299,10 +331,19 @@ __device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out
 // tag of the later mark, accumulates per tag in shared memory, and writes the sums and mark counts to
 // trace[role * 8192 + tag * 2 ...] when it ends.
 constexpr int kTraceTags = 48;
+template <bool ON>
 struct Tracer {
   unsigned long long* p;      // global destination (nullptr: off)
   unsigned long long* acc;    // shared accumulators of this role: [tag][sum, count]
   long long last;
+  bool on;
+  // Only every 8th tile is timed: the bookkeeping of a timed tile (~100 clocks per event) would otherwise slow the
+  // traced CTA by a quarter and distort what it measures.
+  __device__ __forceinline__ void sample(uint32_t ordinal) {
+    const bool was = on;
+    on = p != nullptr && (ordinal & 7u) == 0u;
+    if (on && !was) last = clock64();
+  }
   __device__ __forceinline__ void init(unsigned long long* base, int role, unsigned char* smem_trace) {
     p = (base != nullptr && blockIdx.x == 0) ? base + (size_t)role * 8192 : nullptr;
     acc = reinterpret_cast<unsigned long long*>(smem_trace) + role * kTraceTags * 2;
@@ -310,9 +351,10 @@ struct Tracer {
       for (int i = 0; i < kTraceTags * 2; ++i) acc[i] = 0;
       last = clock64();
     }
+    on = false;
   }
   __device__ __forceinline__ void ev(uint32_t tag, uint32_t) {
-    if (p != nullptr) {
+    if (on) {
       const long long now = clock64();
       acc[2 * tag] += (unsigned long long)(now - last);
       acc[2 * tag + 1] += 1;
@@ -324,30 +366,42 @@ struct Tracer {
       for (int i = 0; i < kTraceTags * 2; ++i) p[i] = acc[i];
   }
 };
+template <>
+struct Tracer<false> {   // the production instantiation carries no state and no code
+  __device__ __forceinline__ void sample(uint32_t) {}
+  __device__ __forceinline__ void init(unsigned long long*, int, unsigned char*) {}
+  __device__ __forceinline__ void ev(uint32_t, uint32_t) {}
+  __device__ __forceinline__ void flush() {}
+};
 
 // One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]).
-//   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the largest exponent seen.
+//   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the OR of the packed words: bit 14 or 30
+//                      set means some p >= 2 (the references sit kRefShift above the column maxima, so that is a score
+//                      2^(kRefShift + 1) above its reference maximum, or an infinity / NaN).
 //   SUBTRACT == true : removes p from l[c] again (used before a rebase; pk is not touched).
 // MASKED applies the causal mask of a diagonal block / drops a dead row.
-template <bool MASKED, bool SUBTRACT>
-__device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __restrict__ mref, float sl2, bool row_live,
-                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32], Tracer* tr = nullptr) {
-  float xmax = -CUDART_INF_F;
-  uint32_t sv[2][16];
-  tc_ld16(s_addr, sv[0]);
+template <bool MASKED, bool SUBTRACT, class TR = Tracer<false>>
+__device__ __forceinline__ uint32_t softmax_pass(uint32_t s_addr, uint32_t m_addr, float sl2, bool row_live,
+                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32], TR* tr = nullptr) {
+  uint32_t ored = 0u;
+  uint32_t sv[2][8], mv[2][8];
+  tc_ld8(s_addr, sv[0]);
+  tc_ld8(m_addr, mv[0]);
 #pragma unroll
-  for (int ch = 0; ch < 4; ++ch) {
-    tc_wait_ld(sv[ch & 1]);
-    if (tr) tr->ev(40 + ch, 0);
-    if (ch < 3) tc_ld16(s_addr + (ch + 1) * 16, sv[(ch + 1) & 1]);
+  for (int ch = 0; ch < 8; ++ch) {
+    tc_wait_ld8(sv[ch & 1], mv[ch & 1]);
+    if (tr) tr->ev(40 + (ch >> 1), 0);
+    if (ch < 7) {
+      tc_ld8(s_addr + (ch + 1) * 8, sv[(ch + 1) & 1]);
+      tc_ld8(m_addr + (ch + 1) * 8, mv[(ch + 1) & 1]);
+    }
 #pragma unroll
-    for (int e = 0; e < 16; e += 4) {
-      const int c = ch * 16 + e;
-      const float4 mr = *reinterpret_cast<const float4*>(&mref[c]);
-      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -mr.x);
-      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -mr.y);
-      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -mr.z);
-      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -mr.w);
+    for (int e = 0; e < 8; e += 4) {
+      const int c = ch * 8 + e;
+      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -__uint_as_float(mv[ch & 1][e]));
+      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -__uint_as_float(mv[ch & 1][e + 1]));
+      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -__uint_as_float(mv[ch & 1][e + 2]));
+      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -__uint_as_float(mv[ch & 1][e + 3]));
       if (MASKED) {
         if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
         if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
@@ -358,17 +412,18 @@ __device__ __forceinline__ float softmax_pass(uint32_t s_addr, const float* __re
       if (SUBTRACT) {
         l[c] -= p0; l[c + 1] -= p1; l[c + 2] -= p2; l[c + 3] -= p3;
       } else {
-        xmax = fmaxf(xmax, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
         l[c] += p0; l[c + 1] += p1; l[c + 2] += p2; l[c + 3] += p3;
         pk[c >> 1] = pack_bf16(p0, p1);
         pk[(c >> 1) + 1] = pack_bf16(p2, p3);
+        ored |= pk[c >> 1] | pk[(c >> 1) + 1];
       }
     }
   }
-  return xmax;
+  return ored;
 }
 
 // ------------------------------------------------------------------------------------------------ kernel
+template <bool kTrace>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, SeqMeta m, const int32_t* __restrict__ row_ptr,
@@ -412,6 +467,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const unsigned long long cta_t0 = kTrace ? global_ns() : 0ull;
+  const long long cta_c0 = kTrace ? clock64() : 0ll;
 
   // Ordinals shared by all roles: k = non-empty items seen by this CTA, g = tiles seen, cnt_a / cnt_b = tiles handed to
   // softmax group A / B.  Every role walks the same items and tiles, so the counters agree without communication.
@@ -422,7 +479,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // ============================================================================================ K (+Q) producer (TMA)
   if (warp == 0) {
     if (lane == 0) {
-      Tracer tr; tr.init(trace, 0, smem + kOffTrace);
+      Tracer<kTrace> tr; tr.init(trace, 0, smem + kOffTrace);
       uint32_t k = 0, g = 0, slot = 0, use = 0;
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
@@ -438,7 +495,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int t = 0; t < it.ntiles; ++t, ++g) {
           const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
           if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
-          tr.ev(1, g);
+          tr.sample(g); tr.ev(1, g);
           if (!mbar_wait(sh, K_EMPTY + (int)slot, (use & 1u) ^ 1u, status)) { ok = false; break; }
           tr.ev(2, g);
           const bool has_b = jb != -1;
@@ -468,7 +525,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // have landed.
   else if (warp >= 12) {
     const int pw = warp - 12;
-    Tracer tr; tr.init(lane == 0 && pw == 0 ? trace : nullptr, 2, smem + kOffTrace);
+    Tracer<kTrace> tr; tr.init(lane == 0 && pw == 0 ? trace : nullptr, 2, smem + kOffTrace);
     const unsigned char* __restrict__ xg = reinterpret_cast<const unsigned char*>(v_ptr);
     const size_t row_bytes = (size_t)m.num_kv_heads * kHeadDim * 2;      // bytes between consecutive tokens
     const int chunk = lane & 15, rsub = lane >> 4;
@@ -492,7 +549,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int t = 0; t < it.ntiles; ++t, ++g) {
         const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
         const uint32_t st = g & 1u;
-        tr.ev(3, g);
+        tr.sample(g); tr.ev(3, g);
         if (!mbar_wait(sh, V_EMPTY + (int)st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
         tr.ev(4, g);
         const uint32_t dst0 = sh.base + kOffV + st * kKVBytes;
@@ -522,7 +579,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // ============================================================================================ S^T issuer
   else if (warp == 1) {
     if (lane == 0) {
-      Tracer tr; tr.init(trace, 1, smem + kOffTrace);
+      Tracer<kTrace> tr; tr.init(trace, 1, smem + kOffTrace);
       uint32_t k = 0, g = 0, cnt_a = 0, cnt_b = 0, slot = 0, use = 0;
       // descriptor bases; per K-step the start address advances by 32 bytes inside a 64-element swizzle atom and by
       // one d-half (16 KB / 8 KB) between atoms
@@ -536,7 +593,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int t = 0; t < it.ntiles; ++t, ++g) {
           const int grp = t & 1;
           const uint32_t cn = grp ? cnt_b : cnt_a, buf = cn & 1u;
-          tr.ev(10, g);
+          tr.sample(g); tr.ev(10, g);
           if (!mbar_wait(sh, K_FULL + (int)slot, use & 1u, status)) { ok = false; break; }
           tr.ev(11, g);
           if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
@@ -564,7 +621,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // ============================================================================================ P V issuer
   else if (warp == 3) {
     if (lane == 0) {
-      Tracer tr; tr.init(trace, 3, smem + kOffTrace);
+      Tracer<kTrace> tr; tr.init(trace, 3, smem + kOffTrace);
       uint32_t g = 0, cnt_a = 0, cnt_b = 0;
       const uint64_t vd0 = make_desc(sh.base + kOffV, kHalfKV, 1024), vd1 = make_desc(sh.base + kOffV + kKVBytes, kHalfKV, 1024);
       const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024), pd1 = make_desc(sh.base + kOffP + kPBytes, kHalfKV, 1024);
@@ -574,7 +631,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int t = 0; t < it.ntiles; ++t, ++g) {
           const int grp = t & 1;
           const uint32_t cn = grp ? cnt_b : cnt_a, st = g & 1u;
-          tr.ev(13, g);
+          tr.sample(g); tr.ev(13, g);
           if (!mbar_wait(sh, V_FULL + st, (g >> 1) & 1u, status)) { ok = false; break; }
           tr.ev(14, g);
           if (!mbar_wait(sh, P_FULL + grp, cn & 1u, status)) { ok = false; break; }
@@ -625,12 +682,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int bar_sync = 1 + grp, bar_vote = 3 + grp;
     const float sl2 = m.softmax_scale * 1.4426950408889634f;
     const int key_local = r & 63;
-    Tracer tr; tr.init(gt == 0 ? trace : nullptr, 4 + grp, smem + kOffTrace);
+    Tracer<kTrace> tr; tr.init(gt == 0 ? trace : nullptr, 4 + grp, smem + kOffTrace);
     uint32_t cnt = 0;                                    // tiles this group has processed
     uint32_t gbase = 0;                                  // tiles of this CTA before the current item
     bool ok = true;
 
     for (int64_t w = blockIdx.x; w < m.rows; w += gridDim.x) {
+      tr.sample(0);
       const Item it = decode_item(m, row_ptr, w);
       const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock;
       const int tiles_a = (it.ntiles + 1) >> 1, tiles_b = it.ntiles >> 1;
@@ -642,39 +700,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       named_bar_sync(bar_sync, kGroupThreads);
 
       int nja = list_block(it, col_idx, 2 * grp), njb = list_block(it, col_idx, 2 * grp + 1);
+      tr.ev(29, 0);
       for (int t = grp; t < it.ntiles; t += 2, ++cnt) {
         const uint32_t sbuf = cnt & 1u;
-        tr.ev(20, gbase + t);
+        tr.sample(cnt); tr.ev(20, gbase + t);
         bool fail = !mbar_wait(sh, S_FULL + 2 * grp + sbuf, (cnt >> 1) & 1u, status);
         tr.ev(21, gbase + t);
         tc_fence_after();
         const int ja = nja, jb = njb;
-        nja = list_block(it, col_idx, 2 * t + 4); njb = list_block(it, col_idx, 2 * t + 5);   // this group's next tile
+        // this group's next tile: the loads are issued here and looked at after the pass
+        const int raw_a = list_fetch(it, col_idx, 2 * t + 4), raw_b = list_fetch(it, col_idx, 2 * t + 5);
         const int my_j = r < 64 ? ja : jb;
         const bool row_live = my_j >= 0;                 // absent / rejected blocks contribute nothing
         const bool diag = my_j == it.i;
         const bool masked = !row_live || diag;           // uniform per warp (a warp lies in one block half)
         const uint32_t s_addr = tmem + lane_addr + col_s(grp, sbuf);
+        const uint32_t m_addr = tmem + lane_addr + col_m(grp);
         uint32_t pk[32];
-        float xmax = -CUDART_INF_F;
-        if (!fail) xmax = masked ? softmax_pass<true, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk, &tr)
-                                 : softmax_pass<false, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk, &tr);
+        // the first tile of a group in an item has no references yet: it goes straight to the rebase path
+        uint32_t over = 0x40004000u;
+        if (!fail && t >= 2) over = masked ? softmax_pass<true, false, Tracer<kTrace>>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk, &tr)
+                                 : softmax_pass<false, false, Tracer<kTrace>>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk, &tr);
+        nja = list_check(it, 2 * t + 4, raw_a); njb = list_check(it, 2 * t + 5, raw_b);
         tr.ev(23, gbase + t);
         // the previous P V of this group must have finished before its P^T buffer (and, when rebasing, its O^T accumulator)
         // is touched; by now it normally has
         if (!fail && cnt > 0) fail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
         tc_fence_after();
         tr.ev(22, gbase + t);
-        // one vote per tile: does any entry exceed its reference by more than 2^8 (or has a wait been lost)?
-        const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || xmax > 8.f);
+        // one vote per tile: does any entry reach 2^(kRefShift + 1) times its reference maximum (or has a wait been lost)?
+        const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
         tr.ev(24, gbase + t);
         if (slow) {
           if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
           // ---- rebase: take this tile's contribution out of the row sums again, find the exact column maxima, move
           // the references, rescale the row sums and O^T, and recompute the tile
           if (t >= 2) {
-            if (masked) softmax_pass<true, true>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
-            else softmax_pass<false, true>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+            if (masked) softmax_pass<true, true>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
+            else softmax_pass<false, true>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
           }
           if (gt < 64) colmax[gt] = float_order_int(-CUDART_INF_F);
           named_bar_sync(bar_sync, kGroupThreads);
@@ -695,12 +758,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           named_bar_sync(bar_sync, kGroupThreads);
           if (gt < 64) {
             const float old = mref[gt];
-            float nm = fmaxf(old, order_int_float(colmax[gt]));
+            float nm = fmaxf(old, order_int_float(colmax[gt]) + kRefShift);
             if (nm == -CUDART_INF_F) nm = 0.f;           // nothing visible in this column yet
             alpha[gt] = old == -CUDART_INF_F ? 0.f : exp2f(old - nm);
             mref[gt] = nm;
           }
           named_bar_sync(bar_sync, kGroupThreads);
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {                // this lane's copy of the new references
+            uint32_t mv[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) mv[e] = __float_as_uint(mref[ch * 16 + e]);
+            tc_st16(m_addr + ch * 16, mv);
+          }
+          tc_wait_st();
           // a reference that moved by more than 2^30 makes everything accumulated so far negligible (and the value
           // taken out above may not have been finite): start the column afresh
 #pragma unroll
@@ -720,8 +791,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             }
             tc_wait_st();
           }
-          if (masked) softmax_pass<true, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
-          else softmax_pass<false, false>(s_addr, mref, sl2, row_live, diag, key_local, l_part, pk);
+          if (masked) softmax_pass<true, false>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
+          else softmax_pass<false, false>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
         }
         // the S^T buffer may be overwritten by a later tile
         tc_fence_before();
@@ -749,7 +820,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       gbase += (uint32_t)it.ntiles;
 
       // ------------------------------------------------------------------------------------------ epilogue
-      tr.ev(30, (uint32_t)(w / gridDim.x));
+      tr.sample(0); tr.ev(30, (uint32_t)(w / gridDim.x));
       bool efail = !ok;
       if (ok && my_tiles > 0) efail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
       tc_fence_after();
@@ -819,6 +890,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
   tc_fence_before();
   __syncthreads();
+  if (kTrace && trace != nullptr && threadIdx.x == 0) { trace[6 * 8192 + blockIdx.x] = global_ns() - cta_t0; trace[6 * 8192 + 256 + blockIdx.x] = (unsigned long long)(clock64() - cta_c0); }  // wall time of this CTA: ns, SM clocks
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -851,7 +923,9 @@ seer_status init_attn_tc(seer_ctx* ctx) {
       qres != cudaDriverEntryPointSuccess)
     return SEER_ERR_CUDA;
   ctx->tmap_encode = fn;
-  cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
   return e == cudaSuccess ? SEER_OK : SEER_ERR_CUDA;
 }
 
@@ -865,7 +939,11 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
       !tc::make_map(ctx, &mv, v, m.total_tokens, m.num_kv_heads))
     return -(int)cudaErrorInvalidValue;
   const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, m.rows);
-  tc::attn_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
+  if (ctx->trace != nullptr)   // the instrumented instantiation
+    tc::attn_tc_kernel<true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
+                                                                    ctx->d_status, (unsigned long long*)ctx->trace);
+  else
+    tc::attn_tc_kernel<false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
                                                                     ctx->d_status, (unsigned long long*)ctx->trace);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;

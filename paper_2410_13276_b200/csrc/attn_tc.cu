@@ -43,12 +43,12 @@ constexpr uint32_t kQBytes = 2 * kHalfQ;         // 16 KB
 constexpr uint32_t kKVBytes = 2 * kHalfKV;       // 32 KB (K or V tile of 128 keys)
 constexpr uint32_t kPBytes = 128 * 128;          // 16 KB  P^T [128 keys][64 q] bf16
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr int kKSlots = 3, kVSlots = 2;
+constexpr int kKSlots = 2, kVSlots = 2;
 constexpr uint32_t kOffQ = 0;                                     // 16 KB
 constexpr uint32_t kOffK = kOffQ + kQBytes;                       // kKSlots x 32 KB ring
 constexpr uint32_t kOffV = kOffK + kKSlots * kKVBytes;            // kVSlots x 32 KB ring
-constexpr uint32_t kOffP = kOffV + kVSlots * kKVBytes;            // 2 x 16 KB, one per softmax group (also epilogue staging)
-constexpr uint32_t kOffGrp = kOffP + 2 * kPBytes;                 // per-group small arrays
+constexpr uint32_t kOffP = kOffV + kVSlots * kKVBytes;            // 4 x 16 KB: two per softmax group (the first also epilogue staging)
+constexpr uint32_t kOffGrp = kOffP + 4 * kPBytes;                 // per-group small arrays
 constexpr uint32_t kGrpMref = 0, kGrpAlpha = 256, kGrpColmax = 512, kGrpLfin = 768, kGrpLsum = 1024;   // lsum: 4 x 64 floats
 constexpr uint32_t kGrpBytes = 2048;
 constexpr uint32_t kOffW = kOffGrp + 2 * kGrpBytes;               // merge weights wA[64], wB[64]
@@ -60,7 +60,7 @@ constexpr uint32_t kSmemBytes = kOffTrace + 6 * 48 * 16 + 1024;   // + alignment
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /* + slot */, K_EMPTY = 5, V_FULL = 8, V_EMPTY = 10,
-           S_FULL = 12 /* + 2*group + buf */, S_EMPTY = 16, P_FULL = 20 /* + group */, PV_DONE = 22 };
+           S_FULL = 12 /* + 2*group + buf */, S_EMPTY = 16, P_FULL = 20 /* + 2*group + buf */, PV_DONE = 24 /* + 2*group + buf */ };
 
 constexpr uint32_t kTmemCols = 512;
 __device__ __forceinline__ uint32_t col_s(int group, uint32_t buf) { return (uint32_t)group * 192u + buf * 64u; }
@@ -448,13 +448,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(sh.bar(V_FULL + i), 32 * kVProducerWarps);   // one arrival per producer lane, when its copies have landed
       mbar_init(sh.bar(V_EMPTY + i), 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {
       mbar_init(sh.bar(P_FULL + i), kGroupThreads / 32);   // one arrival per softmax warp
       mbar_init(sh.bar(PV_DONE + i), 1);
-    }
-    for (int i = 0; i < 4; ++i) {
       mbar_init(sh.bar(S_FULL + i), 1);
-      mbar_init(sh.bar(S_EMPTY + i), kGroupThreads / 32);
+      mbar_init(sh.bar(S_EMPTY + i), 1);                   // passed on by the P V issuer when it has seen P_FULL
     }
     st_shared_u32(sh.abort_flag(), 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -624,7 +622,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       Tracer<kTrace> tr; tr.init(trace, 3, smem + kOffTrace);
       uint32_t g = 0, cnt_a = 0, cnt_b = 0;
       const uint64_t vd0 = make_desc(sh.base + kOffV, kHalfKV, 1024), vd1 = make_desc(sh.base + kOffV + kKVBytes, kHalfKV, 1024);
-      const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024), pd1 = make_desc(sh.base + kOffP + kPBytes, kHalfKV, 1024);
+      const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024);   // P^T buffer (group, buf) lies 2 * group + buf buffers on
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
         const Item it = decode_item(m, row_ptr, w);
@@ -634,11 +632,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tr.sample(g); tr.ev(13, g);
           if (!mbar_wait(sh, V_FULL + st, (g >> 1) & 1u, status)) { ok = false; break; }
           tr.ev(14, g);
-          if (!mbar_wait(sh, P_FULL + grp, cn & 1u, status)) { ok = false; break; }
+          const uint32_t pb = 2u * (uint32_t)grp + (cn & 1u);
+          if (!mbar_wait(sh, P_FULL + (int)pb, (cn >> 1) & 1u, status)) { ok = false; break; }
+          // the softmax group has finished with S^T buffer cn & 1 as well (it read it before it wrote P^T): tell the S^T issuer
+          mbar_arrive(sh.bar(S_EMPTY + (int)pb));
           tr.ev(15, g);
           fence_async_smem();     // V was written through the generic proxy (cp.async); the MMA reads through the async proxy
           tc_fence_after();
-          const uint64_t vd = st ? vd1 : vd0, pd = grp ? pd1 : pd0;
+          const uint64_t vd = st ? vd1 : vd0, pd = pd0 + (uint64_t)(pb * (kPBytes >> 4));
           const uint32_t d = tmem + col_o(grp);
           const uint32_t acc0 = t >= 2 ? 1u : 0u;                  // first tile of this group in the item starts O^T afresh
           // 16 keys (2048 bytes of 128-byte rows) per step; an odd list leaves the second block of its last tile out
@@ -649,7 +650,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             for (int kk = 4; kk < 8; ++kk) tc_mma(d, vd + (uint64_t)(kk * 128), pd + (uint64_t)(kk * 128), kIdescPV, 1u);
           }
           tc_commit(sh.bar(V_EMPTY + st));
-          tc_commit(sh.bar(PV_DONE + grp));
+          tc_commit(sh.bar(PV_DONE + (int)pb));
           tr.ev(19, g);
           if (grp) ++cnt_b; else ++cnt_a;
         }
@@ -723,15 +724,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                                  : softmax_pass<false, false, Tracer<kTrace>>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk, &tr);
         nja = list_check(it, 2 * t + 4, raw_a); njb = list_check(it, 2 * t + 5, raw_b);
         tr.ev(23, gbase + t);
-        // the previous P V of this group must have finished before its P^T buffer (and, when rebasing, its O^T accumulator)
-        // is touched; by now it normally has
-        if (!fail && cnt > 0) fail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
-        tc_fence_after();
+        // P^T goes to buffer cnt & 1 of the group; the P V that read that buffer two tiles ago has normally long finished
+        if (!fail && cnt >= 2) fail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)sbuf, ((cnt >> 1) - 1) & 1u, status);
         tr.ev(22, gbase + t);
         // one vote per tile: does any entry reach 2^(kRefShift + 1) times its reference maximum (or has a wait been lost)?
         const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
         tr.ev(24, gbase + t);
         if (slow) {
+          // the O^T accumulator is rescaled below: the previous P V of this group must have finished
+          if (!fail && t >= 2) fail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)(sbuf ^ 1u), ((cnt - 1) >> 1) & 1u, status);
+          tc_fence_after();
           if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
           // ---- rebase: take this tile's contribution out of the row sums again, find the exact column maxima, move
           // the references, rescale the row sums and O^T, and recompute the tile
@@ -794,14 +796,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (masked) softmax_pass<true, false>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
           else softmax_pass<false, false>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
         }
-        // the S^T buffer may be overwritten by a later tile
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sh.bar(S_EMPTY + 2 * grp + sbuf));     // one arrival per warp: 128 would serialise on the barrier word
         tr.ev(26, 0);
-        // P^T row r -> shared memory (128-byte swizzle)
+        // P^T row r -> buffer cnt & 1 of the group (128-byte swizzle)
         {
-          const uint32_t prow = sh.base + kOffP + grp * kPBytes + (uint32_t)r * 128u;
+          const uint32_t prow = sh.base + kOffP + (2u * (uint32_t)grp + sbuf) * kPBytes + (uint32_t)r * 128u;
 #pragma unroll
           for (int ck = 0; ck < 8; ++ck) {
             const uint32_t a = prow + (uint32_t)((ck ^ (r & 7)) << 4);
@@ -812,9 +810,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         tr.ev(27, 0);
         fence_async_smem();
         tr.ev(28, 0);
+        // one arrival per warp (128 would serialise on the barrier word); it also hands the S^T buffer back
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(sh.bar(P_FULL + grp));
+        if (lane == 0) mbar_arrive(sh.bar(P_FULL + 2 * grp + (int)sbuf));
         tr.ev(25, gbase + t);
       }
       gbase += (uint32_t)it.ntiles;
@@ -822,7 +821,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       // ------------------------------------------------------------------------------------------ epilogue
       tr.sample(0); tr.ev(30, (uint32_t)(w / gridDim.x));
       bool efail = !ok;
-      if (ok && my_tiles > 0) efail = !mbar_wait(sh, PV_DONE + grp, (cnt - 1) & 1u, status);
+      if (ok && my_tiles > 0) {                          // the last P V on each P^T buffer (cnt tiles so far in this CTA)
+        efail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)((cnt - 1) & 1u), ((cnt - 1) >> 1) & 1u, status);
+        if (!efail && cnt >= 2) efail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)(cnt & 1u), ((cnt - 2) >> 1) & 1u, status);
+      }
       tc_fence_after();
       {
         float s0, s1; int base;
@@ -851,7 +853,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       named_bar_sync(5, 2 * kGroupThreads);
       // each group merges and stores 32 of the 64 query columns: staging [32 q][128 d] bf16 in its own P^T buffer
       {
-        uint16_t* stage = reinterpret_cast<uint16_t*>(smem + kOffP + grp * kPBytes);
+        uint16_t* stage = reinterpret_cast<uint16_t*>(smem + kOffP + 2 * grp * kPBytes);
         const int c0 = grp * 32;
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
@@ -871,7 +873,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tc_fence_before();
       named_bar_sync(5, 2 * kGroupThreads);   // every TMEM read of the item is done: the next item may overwrite O^T
       {
-        const uint4* stage4 = reinterpret_cast<const uint4*>(smem + kOffP + grp * kPBytes);
+        const uint4* stage4 = reinterpret_cast<const uint4*>(smem + kOffP + 2 * grp * kPBytes);
         for (int idx = gt; idx < 32 * 16; idx += kGroupThreads) {
           const int qrow = grp * 32 + (idx >> 4), chunk = idx & 15;
           if (qrow < it.q_valid)

@@ -9,7 +9,9 @@ What it follows
 ---------------
 * AttnGate, Sec. 3.1 and Eq. 1:  score = softmax((Wq Pq(Q)) (Wk Pk(K))^T / sqrt(d)),
   with Pq, Pk non-overlapping pooling of kernel = stride = B along the sequence
-  (`pool_avg`, `project`, `gate_logits`, `gate_scores`).
+  (`pool_avg`, `project`, `gate_logits`, `gate_scores`); its two refinements in the same
+  section, composed avg/max/min pooling and block-level RoPE with theta/B
+  (`pool_compose`, `block_rope`, `gate_scores_ex`).
 * Binary block mask, Sec. 3.3 "Generating Binary Block Mask", Eq. 3 (TopK) and
   Eq. 4 (score > threshold) (`select_row`, `block_mask`).
 * Block-sparse attention, Sec. 3.3 "Block Sparse Flash-Attn Kernel": the tiles
@@ -125,6 +127,76 @@ def gate_scores(q_bits, k_bits, wq, wk, cu_seqlens, B: int) -> list:
     for b in range(len(pq)):
         gq = project(pq[b], wq)
         gk = project(pk[b], wk)
+        out.append(causal_softmax_rows(gate_logits(gq, gk)).astype(np.float32))
+    return out
+
+
+# --------------------------------------------------------------------------- AttnGate variants (Sec. 3.1)
+POOL_AVG = 1
+POOL_MAX = 2
+POOL_MIN = 4
+
+
+def pool_compose(x_bits: np.ndarray, cu_seqlens, B: int, methods: int) -> list:
+    """Sec. 3.1, "Pooling Method Selection": several pooling methods (average, max, min; kernel = stride = B)
+    applied to the same tensor, their results concatenated in the hidden dimension before the linear layer.
+    `methods` is a non-empty subset of POOL_AVG | POOL_MAX | POOL_MIN; the concatenation order is avg, max, min
+    (a reading: the paper fixes no order, and a learned layer absorbs any).  A ragged last block pools the tokens
+    it has.  Returns one [H, nb_b, n * d] array per sequence (n = number of methods)."""
+    if methods <= 0 or methods & ~(POOL_AVG | POOL_MAX | POOL_MIN):
+        raise ValueError("methods must be a non-empty subset of avg | max | min")
+    out = []
+    for b in range(len(cu_seqlens) - 1):
+        s0, s1 = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        nb = (s1 - s0 + B - 1) // B
+        H, d = x_bits.shape[1], x_bits.shape[2]
+        parts = []
+        for bit in (POOL_AVG, POOL_MAX, POOL_MIN):
+            if not methods & bit:
+                continue
+            pooled = np.zeros((H, nb, d), dtype=np.float64)
+            for i in range(nb):
+                t0, t1 = s0 + i * B, min(s0 + (i + 1) * B, s1)
+                blk = bf16_bits_to_f64(x_bits[t0:t1])        # [tokens, H, d]
+                if bit == POOL_AVG:
+                    pooled[:, i, :] = blk.sum(axis=0) / float(t1 - t0)
+                elif bit == POOL_MAX:
+                    pooled[:, i, :] = blk.max(axis=0)
+                else:
+                    pooled[:, i, :] = blk.min(axis=0)
+            parts.append(pooled)
+        out.append(np.concatenate(parts, axis=-1))
+    return out
+
+
+def block_rope(g: np.ndarray, theta: float, B: int) -> np.ndarray:
+    """Sec. 3.1, "Block-level RoPE in AttnGate": rotary position encoding applied after the gate's linear layer,
+    at block granularity, with the reduced base theta' = theta / B.  g is [H, nb, dg] for one sequence; block i
+    is position i.  Standard rotary form (a reading, the paper gives none): pair (c, c + dg/2), frequency
+    theta'^(-2c/dg), (x_c, x_{c+dg/2}) -> (x_c cos a - x_{c+dg/2} sin a, x_{c+dg/2} cos a + x_c sin a), a = i * frequency."""
+    H, nb, dg = g.shape
+    half = dg // 2
+    base = float(theta) / float(B)
+    freq = base ** (-2.0 * np.arange(half, dtype=np.float64) / dg)          # [half]
+    ang = np.arange(nb, dtype=np.float64)[:, None] * freq[None, :]           # [nb, half]
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = g[..., :half], g[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def gate_scores_ex(q_bits, k_bits, wq, wk, cu_seqlens, B: int, pool_q: int = POOL_AVG, pool_k: int = POOL_AVG,
+                   rope_theta: float = 0.0) -> list:
+    """AttnGate of Eq. 1 with the paper's two refinements: composed pooling on Q and on K (wq is [Hq, nq*d, dg], wk
+    [Hkv, nk*d, dg]) and, when rope_theta > 0, block-level RoPE on the projected tensors.  Defaults reduce to
+    `gate_scores`.  Returns, per sequence, the fp32 array [Hq, nb, nb]."""
+    pq = pool_compose(q_bits, cu_seqlens, B, pool_q)
+    pk = pool_compose(k_bits, cu_seqlens, B, pool_k)
+    out = []
+    for b in range(len(pq)):
+        gq = project(pq[b], wq)
+        gk = project(pk[b], wk)
+        if rope_theta > 0.0:
+            gq, gk = block_rope(gq, rope_theta, B), block_rope(gk, rope_theta, B)
         out.append(causal_softmax_rows(gate_logits(gq, gk)).astype(np.float32))
     return out
 

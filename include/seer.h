@@ -169,6 +169,34 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
 seer_status seer_gate_scores_static(const seer_shape* shape, const void* q, const void* k, const float* Wq,
                                     const float* Wk, float* scores, void* stream);
 
+/* AttnGate with the two refinements of Sec. 3.1 beyond the simplest form of Eq. 1.
+ *
+ * "Pooling Method Selection": Q and K may each be pooled by any non-empty subset of {average, max, min} (kernel = stride
+ * = block); the pooled tensors are concatenated in the hidden dimension, in the order average, max, min, before the
+ * linear layer.  The paper's best configuration is pool_q = SEER_POOL_AVG, pool_k = SEER_POOL_AVG | SEER_POOL_MAX |
+ * SEER_POOL_MIN.  Wq is then [num_q_heads, nq * head_dim, gate_dim] and Wk [num_kv_heads, nk * head_dim, gate_dim], fp32,
+ * row-major, nq / nk the number of methods chosen.  A ragged last block pools the tokens it has.
+ *
+ * "Block-level RoPE in AttnGate": with rope_theta > 0 the projected vector of block i (i local to its sequence) is
+ * rotated as position i with the reduced base rope_theta / block: pairs (c, c + gate_dim/2), frequency
+ * (rope_theta / block)^(-2c / gate_dim).  The gate is then meant to be fed Q and K from before the model's own RoPE;
+ * the library applies no RoPE to q and k themselves.  rope_theta = 0 switches it off.
+ *
+ * With pool_q = pool_k = SEER_POOL_AVG and rope_theta = 0 the result is that of seer_gate_scores.  All other
+ * arguments, the workspace (seer_workspace_bytes), layouts, ownership and errors are those of seer_gate_scores;
+ * SEER_ERR_INVALID_ARG for an empty or unknown pooling subset or a negative / non-finite rope_theta. */
+#define SEER_POOL_AVG 1u
+#define SEER_POOL_MAX 2u
+#define SEER_POOL_MIN 4u
+typedef struct {
+  uint32_t pool_q;
+  uint32_t pool_k;
+  float rope_theta;
+} seer_gate_options;
+seer_status seer_gate_scores_ex(seer_ctx* ctx, const seer_shape* shape, const seer_gate_options* options, const void* q,
+                                const void* k, const float* Wq, const float* Wk, float* scores, void* ws, size_t ws_bytes,
+                                void* stream);
+
 /* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, the tcgen05 attention kernel runs in an
  * instrumented instantiation.  CTA 0 adds up the SM clocks its pipeline roles spend between marked points, on every
  * 8th tile (role r at uint64 offset r * 8192: 48 tags x (clock sum, count)); every CTA writes its wall time in ns at

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libseer.so")
 SEER_OK = 0
 SEER_TOPK_RATIO, SEER_TOPK_COUNT, SEER_THRESHOLD = 0, 1, 2
 SEER_FORCE_DIAG, SEER_FORCE_SINK = 1, 2
+SEER_POOL_AVG, SEER_POOL_MAX, SEER_POOL_MIN = 1, 2, 4
 STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER_ERR_WORKSPACE", "SEER_ERR_CAPACITY",
                 "SEER_ERR_INVALID_INDEX", "SEER_ERR_TIMEOUT", "SEER_ERR_CUDA"]
 
@@ -25,7 +26,7 @@ STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER
 EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
            "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
-           "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static"]
+           "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static", "seer_gate_scores_ex"]
 
 
 class SeerError(RuntimeError):
@@ -44,6 +45,10 @@ class seer_shape(C.Structure):
 class seer_mask_params(C.Structure):
     _fields_ = [("mode", C.c_int32), ("keep_num", C.c_int32), ("keep_den", C.c_int32), ("k", C.c_int32),
                 ("threshold", C.c_float), ("flags", C.c_uint32)]
+
+
+class seer_gate_options(C.Structure):
+    _fields_ = [("pool_q", C.c_uint32), ("pool_k", C.c_uint32), ("rope_theta", C.c_float)]
 
 
 _lib = None
@@ -92,6 +97,8 @@ def load_library() -> C.CDLL:
     lib.seer_prefill_host.restype = C.c_int
     lib.seer_gate_scores_static.argtypes = [shp, vp, vp, vp, vp, vp, vp]
     lib.seer_gate_scores_static.restype = C.c_int
+    lib.seer_gate_scores_ex.argtypes = [vp, shp, C.POINTER(seer_gate_options), vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.seer_gate_scores_ex.restype = C.c_int
     lib.seer_set_trace_buffer.argtypes = [vp, vp]
     lib.seer_set_trace_buffer.restype = C.c_int
     _lib = lib
@@ -184,6 +191,14 @@ def seer_gate_scores(ctx: Context, shape: seer_shape, q, k, wq, wk, scores, ws, 
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check(ctx._lib.seer_gate_scores(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(wq), _ptr(wk), _ptr(scores),
                                      _ptr(ws), ws_bytes, _stream(stream)), "seer_gate_scores")
+
+
+def seer_gate_scores_ex(ctx: Context, shape: seer_shape, options: seer_gate_options, q, k, wq, wk, scores, ws,
+                        stream=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(ctx._lib.seer_gate_scores_ex(ctx.handle, C.byref(shape), C.byref(options), _ptr(q), _ptr(k), _ptr(wq),
+                                        _ptr(wk), _ptr(scores), _ptr(ws), ws_bytes, _stream(stream)),
+           "seer_gate_scores_ex")
 
 
 def seer_block_mask(ctx: Context, shape: seer_shape, scores, params: seer_mask_params, row_ptr, col_idx,

@@ -106,6 +106,147 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
   }
 }
 
+
+// ----------------------------------------------------------------------------------------------- kernel 1, variants
+// Sec. 3.1, "Pooling Method Selection" and "Block-level RoPE in AttnGate": the same single pass over Q and K, but
+//   * a tensor may be pooled by any subset of {average, max, min}; the pooled vectors are concatenated in that order
+//     in the hidden dimension, so the head's gate matrix is [n * d, dg] (n = methods chosen for that tensor);
+//   * with rope_theta > 0 the projected vector of block i is rotated as position i with base rope_theta / B
+//     (pairs (c, c + dg/2), frequency base^(-2c/dg)); the angle and its sine / cosine are taken in double precision
+//     (an fp32 angle near position 2000 would already cost more than the 1e-3 bound on large logits).
+// max and min ride along the average's loads: the kernel stays one HBM pass.
+__device__ __forceinline__ void max_bf16x8(float (&a)[8], const uint4& u) {
+  a[0] = fmaxf(a[0], __uint_as_float(u.x << 16)); a[1] = fmaxf(a[1], __uint_as_float(u.x & 0xffff0000u));
+  a[2] = fmaxf(a[2], __uint_as_float(u.y << 16)); a[3] = fmaxf(a[3], __uint_as_float(u.y & 0xffff0000u));
+  a[4] = fmaxf(a[4], __uint_as_float(u.z << 16)); a[5] = fmaxf(a[5], __uint_as_float(u.z & 0xffff0000u));
+  a[6] = fmaxf(a[6], __uint_as_float(u.w << 16)); a[7] = fmaxf(a[7], __uint_as_float(u.w & 0xffff0000u));
+}
+__device__ __forceinline__ void min_bf16x8(float (&a)[8], const uint4& u) {
+  a[0] = fminf(a[0], __uint_as_float(u.x << 16)); a[1] = fminf(a[1], __uint_as_float(u.x & 0xffff0000u));
+  a[2] = fminf(a[2], __uint_as_float(u.y << 16)); a[3] = fminf(a[3], __uint_as_float(u.y & 0xffff0000u));
+  a[4] = fminf(a[4], __uint_as_float(u.z << 16)); a[5] = fminf(a[5], __uint_as_float(u.z & 0xffff0000u));
+  a[6] = fminf(a[6], __uint_as_float(u.w << 16)); a[7] = fminf(a[7], __uint_as_float(u.w & 0xffff0000u));
+}
+
+constexpr int kPoolExSmem = kPoolChunk * 3 * kHeadDim * (int)sizeof(float);   // 24 KB: [16 blocks][up to 3 parts][128]
+
+__global__ void __launch_bounds__(kPoolThreads)
+pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+                       const float* __restrict__ Wq, const float* __restrict__ Wk, float* __restrict__ gq,
+                       float* __restrict__ gk, uint32_t pool_q, uint32_t pool_k, float rope_theta) {
+  __shared__ __align__(16) float pooled[kPoolChunk][3 * kHeadDim];
+
+  const int heads_total = m.num_q_heads + m.num_kv_heads;
+  const int chunk = blockIdx.x / heads_total;
+  int hh = blockIdx.x - chunk * heads_total;
+  const bool is_q = hh < m.num_q_heads;
+  const int H = is_q ? m.num_q_heads : m.num_kv_heads;
+  const int h = is_q ? hh : hh - m.num_q_heads;
+  const uint32_t methods = is_q ? pool_q : pool_k;
+  const int nparts = __popc(methods);
+  const int width = nparts * kHeadDim;                       // rows of the head's gate matrix
+  const uint16_t* __restrict__ x = is_q ? q : k;
+  const float* __restrict__ W = (is_q ? Wq : Wk) + (size_t)h * width * kGateDim;
+  float* __restrict__ out = is_q ? gq : gk;
+  // offsets of the parts inside the concatenated vector (order: average, max, min)
+  const int off_avg = 0;
+  const int off_max = (methods & SEER_POOL_AVG) ? kHeadDim : 0;
+  const int off_min = off_max + ((methods & SEER_POOL_MAX) ? kHeadDim : 0);
+
+  const int b = find_sequence(m.chunk_off, m.batch, chunk);
+  const int s0 = m.cu_seqlens[b], s1 = m.cu_seqlens[b + 1];
+  const int nb = m.blk_off[b + 1] - m.blk_off[b];
+  const int i0 = (chunk - m.chunk_off[b]) * kPoolChunk;
+  const int nblk = min(kPoolChunk, nb - i0);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = lane >> 4, cchunk = lane & 15;
+  const size_t row_stride = (size_t)H * kHeadDim;
+
+  for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
+    const int t0 = s0 + (i0 + bi) * kBlock;
+    const int cnt = min(kBlock, s1 - t0);
+    const uint16_t* base = x + (size_t)t0 * row_stride + (size_t)h * kHeadDim + cchunk * 8;
+    float a[8], hi[8], lo[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { a[j] = 0.f; hi[j] = -CUDART_INF_F; lo[j] = CUDART_INF_F; }
+#pragma unroll 1
+    for (int it = 0; it < kBlock / 2; it += 8) {
+      uint4 u[8];
+      bool live[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int row = 2 * (it + j) + half;
+        live[j] = row < cnt;
+        u[j] = live[j] ? ld_stream_16(base + (size_t)row * row_stride) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        acc_bf16x8(a, u[j]);
+        if (live[j]) { max_bf16x8(hi, u[j]); min_bf16x8(lo, u[j]); }   // rows past the end of the sequence take no part
+      }
+    }
+    const float inv = 1.0f / (float)cnt;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      a[j] = (a[j] + __shfl_xor_sync(0xffffffffu, a[j], 16)) * inv;
+      hi[j] = fmaxf(hi[j], __shfl_xor_sync(0xffffffffu, hi[j], 16));
+      lo[j] = fminf(lo[j], __shfl_xor_sync(0xffffffffu, lo[j], 16));
+    }
+    if (half == 0) {
+      if (methods & SEER_POOL_AVG) {
+        float4* dst = reinterpret_cast<float4*>(&pooled[bi][off_avg + cchunk * 8]);
+        dst[0] = make_float4(a[0], a[1], a[2], a[3]); dst[1] = make_float4(a[4], a[5], a[6], a[7]);
+      }
+      if (methods & SEER_POOL_MAX) {
+        float4* dst = reinterpret_cast<float4*>(&pooled[bi][off_max + cchunk * 8]);
+        dst[0] = make_float4(hi[0], hi[1], hi[2], hi[3]); dst[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
+      }
+      if (methods & SEER_POOL_MIN) {
+        float4* dst = reinterpret_cast<float4*>(&pooled[bi][off_min + cchunk * 8]);
+        dst[0] = make_float4(lo[0], lo[1], lo[2], lo[3]); dst[1] = make_float4(lo[4], lo[5], lo[6], lo[7]);
+      }
+    }
+  }
+  __syncthreads();
+
+  // projection: thread -> output column o, 8 of the 16 blocks
+  const int o = threadIdx.x & (kGateDim - 1);
+  const int grp = threadIdx.x >> 7;  // 0 or 1
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+  for (int c = 0; c < width; ++c) {
+    const float w = __ldg(W + (size_t)c * kGateDim + o);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = fmaf(pooled[grp * 8 + j][c], w, acc[j]);
+  }
+  if (rope_theta > 0.f) {
+    // rotate (o, o + dg/2) pairs: the partner's value goes through shared memory (the pooled vectors are no longer needed)
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 8; ++j) pooled[grp * 8 + j][o] = acc[j];
+    __syncthreads();
+    const int f = o & (kGateDim / 2 - 1);
+    const double freq = pow((double)rope_theta / (double)kBlock, -2.0 * (double)f / (double)kGateDim);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int bi = grp * 8 + j;
+      double sn, cs;
+      sincos((double)(i0 + bi) * freq, &sn, &cs);
+      const float partner = pooled[bi][o ^ (kGateDim / 2)];
+      // first half: x1 cos - x2 sin; second half: x2 cos + x1 sin
+      acc[j] = (o < kGateDim / 2) ? (float)((double)acc[j] * cs - (double)partner * sn)
+                                  : (float)((double)acc[j] * cs + (double)partner * sn);
+    }
+  }
+  const size_t obase = ((size_t)h * m.total_blocks + m.blk_off[b] + i0) * kGateDim;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int bi = grp * 8 + j;
+    if (bi < nblk) out[obase + (size_t)bi * kGateDim + o] = acc[j];
+  }
+}
+
 // ----------------------------------------------------------------------------------------------- kernel 2
 constexpr int kScoreThreads = 256;
 constexpr int kScoreSmem = 2 * kGateDim * kScoreTile * (int)sizeof(float) + 2 * kScoreTile * (int)sizeof(float);
@@ -240,6 +381,21 @@ int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, c
   float* gk = (float*)((char*)ws + gq_bytes);
   const unsigned grid1 = (unsigned)m.total_chunks * (unsigned)(m.num_q_heads + m.num_kv_heads);
   pool_project_kernel<<<grid1, kPoolThreads, 0, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, Wq, Wk, gq, gk);
+  const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
+  gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, gq, gk, scores);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 2 : -(int)e;
+}
+
+int launch_gate_ex(seer_ctx* ctx, const SeqMeta& m, const seer_gate_options& opt, const void* q, const void* k,
+                   const float* Wq, const float* Wk, float* scores, void* ws, cudaStream_t stream) {
+  (void)ctx;
+  size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * sizeof(float) + 255) / 256 * 256;
+  float* gq = (float*)ws;
+  float* gk = (float*)((char*)ws + gq_bytes);
+  const unsigned grid1 = (unsigned)m.total_chunks * (unsigned)(m.num_q_heads + m.num_kv_heads);
+  pool_project_ex_kernel<<<grid1, kPoolThreads, 0, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, Wq, Wk, gq, gk,
+                                                              opt.pool_q, opt.pool_k, opt.rope_theta);
   const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
   gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, gq, gk, scores);
   cudaError_t e = cudaGetLastError();

@@ -239,6 +239,30 @@ seer_status seer_gate_scores(seer_ctx* ctx, const seer_shape* shape, const void*
   return SEER_OK;
 }
 
+seer_status seer_gate_scores_ex(seer_ctx* ctx, const seer_shape* shape, const seer_gate_options* opt, const void* q,
+                                const void* k, const float* Wq, const float* Wk, float* scores, void* ws, size_t ws_bytes,
+                                void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!ctx || !shape || !opt) return SEER_ERR_INVALID_ARG;
+  const uint32_t all = SEER_POOL_AVG | SEER_POOL_MAX | SEER_POOL_MIN;
+  if (opt->pool_q == 0 || opt->pool_k == 0 || (opt->pool_q & ~all) || (opt->pool_k & ~all)) return SEER_ERR_INVALID_ARG;
+  if (!(opt->rope_theta >= 0.f) || opt->rope_theta > 3.0e38f) return SEER_ERR_INVALID_ARG;   // also rejects NaN
+  ShapeTotals t;
+  seer_status st = shape_totals(shape, &t);
+  if (st != SEER_OK) return st;
+  if (t.total_blocks == 0) return SEER_OK;
+  if (!q || !k || !Wq || !Wk || !scores) return SEER_ERR_INVALID_ARG;
+  if (!ws_ok(ws, ws_bytes, gate_workspace_bytes(t, shape))) return SEER_ERR_WORKSPACE;
+  SeqMeta m; int slot;
+  st = prepare(ctx, shape, stream, &m, &slot);
+  if (st != SEER_OK) return st;
+  int n = launch_gate_ex(ctx, m, *opt, q, k, Wq, Wk, scores, ws, stream);
+  finish_call(ctx, slot, stream);
+  if (n < 0) return SEER_ERR_CUDA;
+  ctx->launches += n;
+  return SEER_OK;
+}
+
 seer_status seer_block_mask(seer_ctx* ctx, const seer_shape* shape, const float* scores, const seer_mask_params* p,
                             int32_t* row_ptr, int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, void* ws,
                             size_t ws_bytes, void* stream_) {

@@ -81,6 +81,8 @@ size_t gate_workspace_bytes(const ShapeTotals& t, const seer_shape* shape);
 // Kernel launchers (each returns the number of kernels it launched, or a negative cudaError).
 int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const float* Wq, const float* Wk,
                 float* scores, void* ws, cudaStream_t stream);
+int launch_gate_ex(seer_ctx* ctx, const SeqMeta& m, const seer_gate_options& opt, const void* q, const void* k,
+                   const float* Wq, const float* Wk, float* scores, void* ws, cudaStream_t stream);
 int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer_mask_params& p, int32_t* row_ptr,
                 int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream);
 int launch_attn_mma(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,

@@ -69,6 +69,11 @@ class Prefill:
     def gate(self, stream=None):
         B.seer_gate_scores(self.ctx, self.shape, self.q, self.k, self.wq, self.wk, self.scores, self.ws, stream)
 
+    def gate_ex(self, options: B.seer_gate_options, wq, wk, stream=None):
+        """Gate with composed pooling and / or block-level RoPE (Sec. 3.1); wq, wk are device tensors
+        [heads, n * 128, 128] matching the pooling subsets in `options`."""
+        B.seer_gate_scores_ex(self.ctx, self.shape, options, self.q, self.k, wq, wk, self.scores, self.ws, stream)
+
     def mask(self, params: B.seer_mask_params, stream=None):
         B.seer_block_mask(self.ctx, self.shape, self.scores, params, self.row_ptr, self.col_idx, self.col_capacity,
                           self.nnz, None, stream)

@@ -127,6 +127,12 @@ def _gate_weights(seed: int, heads: int, d: int, dg: int) -> np.ndarray:
     return (_normal(seed, (heads, d, dg)) * np.float32(1.0 / np.sqrt(128.0))).astype(np.float32)
 
 
+def make_gate_weights(seed: int, heads: int, in_dim: int, dg: int = 128) -> np.ndarray:
+    """Seeded gate matrices [heads, in_dim, dg] (fp32, N(0, std 1/sqrt(128))) for the gate variants whose input is a
+    concatenation of several pooled tensors (in_dim = number of pooling methods x head_dim)."""
+    return _gate_weights(seed, heads, in_dim, dg)
+
+
 def _random_layer(config, twin, seqlens, hq, hkv, rope_base=None):
     cu = np.concatenate([[0], np.cumsum(seqlens)]).astype(np.int32)
     T = int(cu[-1])

@@ -861,12 +861,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (tiles_a > 0) { tc_ld16(tmem + lane_addr + col_o(0) + c0 + ch * 16, oa); tc_wait_ld(oa); }
           if (tiles_b > 0) { tc_ld16(tmem + lane_addr + col_o(1) + c0 + ch * 16, ob); tc_wait_ld(ob); }
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
+          for (int e = 0; e < 16; e += 4) {
             const int c = c0 + ch * 16 + e;
-            float val = 0.f;
-            if (tiles_a > 0) val = __uint_as_float(oa[e]) * w_a[c];
-            if (tiles_b > 0) val = fmaf(__uint_as_float(ob[e]), w_b[c], val);
-            stage[(ch * 16 + e) * 128 + r] = (uint16_t)(pack_bf16(val, 0.f) & 0xffffu);
+            const float4 fa = *reinterpret_cast<const float4*>(&w_a[c]), fb = *reinterpret_cast<const float4*>(&w_b[c]);
+            const float wa4[4] = {fa.x, fa.y, fa.z, fa.w}, wb4[4] = {fb.x, fb.y, fb.z, fb.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              float val = 0.f;
+              if (tiles_a > 0) val = __uint_as_float(oa[e + u]) * wa4[u];
+              if (tiles_b > 0) val = fmaf(__uint_as_float(ob[e + u]), wb4[u], val);
+              stage[(ch * 16 + e + u) * 128 + r] = (uint16_t)(pack_bf16(val, 0.f) & 0xffffu);
+            }
           }
         }
       }

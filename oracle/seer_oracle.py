@@ -364,3 +364,47 @@ def maxpool_attention_map(q_bits, k_bits, cu_seqlens, num_q_heads: int, num_kv_h
                     gt[h, i, j] = A[i * B:(i + 1) * B, j * B:(j + 1) * B].max()
         out.append(gt)
     return out
+
+
+def maxpool_listed_blocks(q_bits, k_bits, cu_seqlens, row_ptr, col_idx, num_q_heads: int, num_kv_heads: int, B: int,
+                          scale: float, rows=None) -> np.ndarray:
+    """The 2D max-pooling of Eq. 2 taken on the attention the block lists define: for the row (sequence, head, query
+    block i) and each listed key block j, the largest softmax probability a_ts = exp(r_ts - m_t) / l_t (appendix) over
+    the B x B tile, the softmax of query t running over the keys of the row's listed blocks that are not later than t.
+    With full causal lists this is entry [h, i, j] of `maxpool_attention_map`.  Returns one fp64 value per entry of
+    col_idx (NaN for rows not in `rows`); a tile in which no (query, key) pair is causal gives 0."""
+    G = num_q_heads // num_kv_heads
+    out = np.full(len(col_idx), np.nan, dtype=np.float64)
+    nbs = blocks_per_sequence(cu_seqlens, B)
+    base = row_base(cu_seqlens, B, num_q_heads)
+    wanted = None if rows is None else set(int(r) for r in rows)
+    for b, nb in enumerate(nbs):
+        s0, s1 = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        for h in range(num_q_heads):
+            g = h // G
+            for i in range(int(nb)):
+                r = int(base[b]) + h * int(nb) + i
+                if wanted is not None and r not in wanted:
+                    continue
+                l0, l1 = int(row_ptr[r]), int(row_ptr[r + 1])
+                if l1 == l0:
+                    continue
+                tq = np.arange(s0 + i * B, min(s0 + (i + 1) * B, s1))
+                Q = bf16_bits_to_f64(q_bits[tq, h, :])
+                tiles = []
+                for j in col_idx[l0:l1]:
+                    tk = np.arange(s0 + int(j) * B, min(s0 + (int(j) + 1) * B, s1))
+                    S = (Q @ bf16_bits_to_f64(k_bits[tk, g, :]).T) * scale
+                    S[tk[None, :] > tq[:, None]] = -np.inf
+                    tiles.append(S)
+                allS = np.concatenate(tiles, axis=1)
+                m = allS.max(axis=1, keepdims=True)
+                m[~np.isfinite(m)] = 0.0
+                l = np.exp(allS - m).sum(axis=1, keepdims=True)
+                for p_, S in enumerate(tiles):
+                    with np.errstate(divide="ignore", invalid="ignore"):
+                        A = np.exp(S - m) / l
+                    A[~np.isfinite(A)] = 0.0
+                    out[l0 + p_] = A.max() if A.size else 0.0
+    return out
+

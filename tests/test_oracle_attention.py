@@ -4,6 +4,7 @@ appendix identity a_ij = exp(r_ij - m_i) / l_i)."""
 import math
 
 import numpy as np
+import pytest
 
 from oracle import seer_oracle as O
 from paper_2410_13276_b200 import workloads as W
@@ -181,3 +182,60 @@ def test_maxpool_map_brute_force_and_appendix_identity():
                             a.append(math.exp(r - lse[h, t]))
                     assert abs(gt[h, i, j] - max(a)) <= 1e-13
     np.testing.assert_allclose(gt[:, 0, 0], 1.0)                      # token 0 puts all its mass on key 0
+
+
+# --------------------------------------------------------------------------- max-pooled map on listed blocks
+def test_maxpool_listed_blocks_dense_lists_equal_eq2_map():
+    """Full causal lists: every entry is the B x B max-pool of the dense causal softmax map (Eq. 2)."""
+    w = W.make_small(seed=61, seqlens=[50, 23], hq=4, hkv=2, block=8, head_dim=16)
+    rp, col = O.full_causal_lists(w.cu_seqlens, w.block, w.num_q_heads)
+    got = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, w.block, 0.25)
+    gt = O.maxpool_attention_map(w.q, w.k, w.cu_seqlens, w.num_q_heads, w.num_kv_heads, w.block, 0.25)
+    base = O.row_base(w.cu_seqlens, w.block, w.num_q_heads)
+    for b, nb in enumerate(O.blocks_per_sequence(w.cu_seqlens, w.block)):
+        for h in range(w.num_q_heads):
+            for i in range(int(nb)):
+                r = int(base[b]) + h * int(nb) + i
+                for p_ in range(int(rp[r]), int(rp[r + 1])):
+                    assert got[p_] == pytest.approx(gt[b][h, i, int(col[p_])], rel=1e-12, abs=0)
+
+
+def test_maxpool_listed_blocks_block_one_is_the_softmax_itself():
+    """B = 1: a tile is one (query, key) pair, so the values of a row are its softmax probabilities and sum to 1."""
+    w = W.make_small(seed=62, seqlens=[12], hq=2, hkv=1, block=1, head_dim=8)
+    rng = np.random.default_rng(5)
+    rp, col = [0], []
+    for h in range(2):
+        for i in range(12):
+            keep = sorted(set([i] + [int(j) for j in rng.choice(i + 1, size=min(3, i + 1), replace=False)]))
+            col += keep
+            rp.append(len(col))
+    rp, col = np.array(rp), np.array(col)
+    got = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, 2, 1, 1, 0.3)
+    Q, K = O.bf16_bits_to_f64(w.q), O.bf16_bits_to_f64(w.k)
+    for r in range(24):
+        h, i = divmod(r, 12)
+        js = col[rp[r]:rp[r + 1]]
+        s = np.array([Q[i, h] @ K[j, 0] * 0.3 for j in js])
+        want = np.exp(s - s.max()) / np.exp(s - s.max()).sum()
+        np.testing.assert_allclose(got[rp[r]:rp[r + 1]], want, rtol=1e-12)
+        assert got[rp[r]:rp[r + 1]].sum() == pytest.approx(1.0, abs=1e-12)
+
+
+def test_maxpool_listed_blocks_invariants():
+    w = W.make_small(seed=63, seqlens=[70], hq=2, hkv=1, block=16, head_dim=8)
+    scores = O.gate_scores(w.q, w.k, w.wq, w.wk, w.cu_seqlens, w.block)
+    rp, col = O.block_mask(scores, O.MODE_TOPK_RATIO, keep_num=1, keep_den=2, flags=O.FORCE_DIAG)
+    got = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, 2, 1, 16, 0.35)
+    assert np.all(got > 0) and np.all(got <= 1.0)
+    # order of a row's list does not matter: reversed lists give the reversed values
+    col_r = col.copy()
+    for r in range(len(rp) - 1):
+        col_r[rp[r]:rp[r + 1]] = col[rp[r]:rp[r + 1]][::-1]
+    got_r = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col_r, 2, 1, 16, 0.35)
+    for r in range(len(rp) - 1):
+        np.testing.assert_allclose(got_r[rp[r]:rp[r + 1]], got[rp[r]:rp[r + 1]][::-1], rtol=1e-12)
+    # rows not asked for stay NaN
+    part = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, 2, 1, 16, 0.35, rows=[1])
+    assert np.isnan(part[rp[2]:]).all() and not np.isnan(part[rp[1]:rp[2]]).any()
+

@@ -297,6 +297,17 @@ def main():
         p.gate()                                             # restore the scores of the bench mask
         del wq_v, wk_v
 
+    # the max-pooled attention map on the kept blocks (Eq. 2; a side output for distillation / diagnostics), outside the
+    # timed region: one attention launch that also writes lse, then the block-max pass
+    block_max_ms = None
+    if rank == 0:
+        p.lse = torch.empty((w.num_q_heads, w.total_tokens), dtype=torch.float32, device="cuda")
+        p.attn(); p.block_max(); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); p.block_max(); b.record(stream); torch.cuda.synchronize()
+        block_max_ms = a.elapsed_time(b)
+        p.lse = None; p.bmax = None
+
     # end to end through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
@@ -346,7 +357,7 @@ def main():
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
                             "kernel": "seer_sparse_attn"},
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
-               "gate_variant": gate_var,
+               "gate_variant": gate_var, "block_max_ms": block_max_ms,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:
             dense_blocks = B.seer_causal_blocks(p.shape)

@@ -121,6 +121,18 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
                              const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, void* ws,
                              size_t ws_bytes, void* stream);
 
+/* Max-pooled attention map on the listed blocks (Sec. 3.2, Eq. 2: the 2D max-pooling, window and stride = block, of the
+ * attention map, which the paper uses as the gate's distillation target; here also a diagnostic of what the gate kept).
+ * For every entry p of col_idx, belonging to row (b, h, i) and naming key block j: block_max[p] = the largest softmax
+ * probability exp(scale * q_t . k_s - lse[h, t]) over the causal (t, s) pairs of that 64 x 64 tile, lse being the
+ * [num_q_heads, T] output of seer_sparse_attn for the same lists (so the probabilities are those of the block-sparse
+ * softmax; with full causal lists, those of dense causal attention).  A tile with no causal pair gives 0.
+ * q, k, row_ptr, col_idx as for seer_sparse_attn; lse and block_max (fp32, [nnz]) are device pointers owned by the
+ * caller; no workspace.  Entries outside [0, i] raise SEER_ERR_INVALID_INDEX on the device status and give 0. */
+seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k,
+                                const int32_t* row_ptr, const int32_t* col_idx, const float* lse, float* block_max,
+                                void* stream);
+
 /* Selects the attention kernel used by seer_sparse_attn: 0 = tcgen05 / TMEM / TMA kernel (default),
  * 1 = mma.sync kernel kept as an on-device cross-check.  Returns SEER_ERR_INVALID_ARG for other values. */
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);

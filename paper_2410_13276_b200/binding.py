@@ -26,7 +26,8 @@ STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER
 EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
            "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
-           "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static", "seer_gate_scores_ex"]
+           "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static", "seer_gate_scores_ex",
+           "seer_attn_block_max"]
 
 
 class SeerError(RuntimeError):
@@ -99,6 +100,8 @@ def load_library() -> C.CDLL:
     lib.seer_gate_scores_static.restype = C.c_int
     lib.seer_gate_scores_ex.argtypes = [vp, shp, C.POINTER(seer_gate_options), vp, vp, vp, vp, vp, vp, sz, vp]
     lib.seer_gate_scores_ex.restype = C.c_int
+    lib.seer_attn_block_max.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp]
+    lib.seer_attn_block_max.restype = C.c_int
     lib.seer_set_trace_buffer.argtypes = [vp, vp]
     lib.seer_set_trace_buffer.restype = C.c_int
     _lib = lib
@@ -199,6 +202,11 @@ def seer_gate_scores_ex(ctx: Context, shape: seer_shape, options: seer_gate_opti
     _check(ctx._lib.seer_gate_scores_ex(ctx.handle, C.byref(shape), C.byref(options), _ptr(q), _ptr(k), _ptr(wq),
                                         _ptr(wk), _ptr(scores), _ptr(ws), ws_bytes, _stream(stream)),
            "seer_gate_scores_ex")
+
+
+def seer_attn_block_max(ctx: Context, shape: seer_shape, q, k, row_ptr, col_idx, lse, block_max, stream=None) -> None:
+    _check(ctx._lib.seer_attn_block_max(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(row_ptr), _ptr(col_idx),
+                                        _ptr(lse), _ptr(block_max), _stream(stream)), "seer_attn_block_max")
 
 
 def seer_block_mask(ctx: Context, shape: seer_shape, scores, params: seer_mask_params, row_ptr, col_idx,

@@ -245,10 +245,146 @@ attn_mma_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __res
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------ max-pooled map
+// Sec. 3.2, Eq. 2 (the distillation target of the gate; at inference a recall diagnostic): the 2D max-pool, window and
+// stride B, of the attention map -- here the map the block lists define, a_ts = exp(r_ts - m_t) / l_t (appendix), given
+// through the log-sum-exp the attention kernel wrote.  One value per list entry: the largest probability in that 64 x 64
+// tile.  Same CTA layout as the kernel above, K tiles only; the tile maximum is reduced over the CTA through shared memory.
+constexpr int kBmSmem = kTileBytes * 3 + 64;                   // Q + 2 x K + four per-warp maxima
+
+__global__ void __launch_bounds__(kMmaThreads)
+block_max_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, const float* __restrict__ lse,
+                 float* __restrict__ out, int* __restrict__ status) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const uint32_t sQ = smem_u32(smem);
+  const uint32_t sK0 = sQ + kTileBytes, sK1 = sK0 + kTileBytes;
+  float* wmax = reinterpret_cast<float*>(smem + 3 * kTileBytes);
+
+  const int64_t w = blockIdx.x;
+  const int b = find_sequence(m.blk_off, m.batch, (int)(w / m.num_q_heads));
+  const int nb = m.blk_off[b + 1] - m.blk_off[b];
+  const int local = (int)(w - (int64_t)m.num_q_heads * m.blk_off[b]);
+  const int g = local / (nb * m.group);
+  const int rem = local - g * nb * m.group;
+  const int i = nb - 1 - rem / m.group;
+  const int h = g * m.group + rem % m.group;
+  const int64_t r = (int64_t)m.num_q_heads * m.blk_off[b] + (int64_t)h * nb + i;
+
+  const int s0 = m.cu_seqlens[b];
+  const int slen = m.cu_seqlens[b + 1] - s0;
+  const int q_valid = min(kBlock, slen - i * kBlock);
+  const int l0 = row_ptr[r], l1 = row_ptr[r + 1];
+  const int nlist = l1 - l0;
+  if (nlist <= 0) return;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+  const int64_t tok0 = (int64_t)s0 + (int64_t)i * kBlock;
+
+  load_tile_async(sQ, q, tok0, q_valid, m.num_q_heads, h);
+  cp_async_commit();
+
+  auto fetch = [&](int it, uint32_t dK) -> int {
+    int j = col_idx[l0 + it];
+    if (j < 0 || j > i) {            // corrupt list entry: record it, never dereference it
+      if (threadIdx.x == 0) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
+      j = -1;
+    } else {
+      load_tile_async(dK, k, (int64_t)s0 + (int64_t)j * kBlock, min(kBlock, slen - j * kBlock), m.num_kv_heads, g);
+    }
+    cp_async_commit();
+    return j;
+  };
+  int j_cur = fetch(0, sK0);
+
+  const float sl2 = m.softmax_scale * 1.4426950408889634f;
+  // log2 of the softmax denominator of this thread's two query rows (gid, gid + 8 of the warp's 16)
+  float lse2[2];
+  bool row_ok[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int row = warp * 16 + gid + e * 8;
+    row_ok[e] = row < q_valid;
+    lse2[e] = row_ok[e] ? lse[(int64_t)h * m.total_tokens + tok0 + row] * 1.4426950408889634f : 0.f;
+  }
+
+  uint32_t qf[8][4];
+  cp_async_wait<1>();
+  __syncthreads();
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    ldsm_x4(qf[kk], sQ + tile_off(row, kk * 2 + (lane >> 4)));
+  }
+
+  for (int it = 0; it < nlist; ++it) {
+    const uint32_t cK = (it & 1) ? sK1 : sK0;
+    int j_next = -1;
+    if (it + 1 < nlist) {
+      j_next = fetch(it + 1, (it & 1) ? sK0 : sK1);
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();
+    float tmax = 0.f;                 // probabilities are positive; a tile with no causal pair gives 0
+    if (j_cur >= 0) {
+      float sacc[8][4];
+#pragma unroll
+      for (int n = 0; n < 8; ++n)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) sacc[n][c] = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+        for (int kk = 0; kk < 8; kk += 2) {
+          uint32_t bf[4];
+          ldsm_x4(bf, cK + tile_off(nt * 8 + (lane & 7), kk * 2 + (lane >> 3)));
+          mma_bf16(sacc[nt], qf[kk], bf[0], bf[1]);
+          mma_bf16(sacc[nt], qf[kk + 1], bf[2], bf[3]);
+        }
+      }
+      // the largest logit of each of the two rows, then one exponential per row (exp is monotone)
+      const bool diag = j_cur == i;
+      float xm[2] = {-CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int rr = warp * 16 + gid + (c >> 1) * 8;
+          const int cc = nt * 8 + 2 * tig + (c & 1);
+          if (!(diag && cc > rr)) xm[c >> 1] = fmaxf(xm[c >> 1], sacc[nt][c]);   // keys past the sequence end lie above the diagonal too
+        }
+#pragma unroll
+      for (int e = 0; e < 2; ++e)
+        if (row_ok[e] && xm[e] != -CUDART_INF_F) tmax = fmaxf(tmax, exp2f(xm[e] * sl2 - lse2[e]));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
+    if (lane == 0) wmax[warp] = tmax;
+    __syncthreads();   // also: everyone is done with this K stage before the next prefetch overwrites it
+    if (threadIdx.x == 0) out[l0 + it] = fmaxf(fmaxf(wmax[0], wmax[1]), fmaxf(wmax[2], wmax[3]));
+    __syncthreads();
+    j_cur = j_next;
+  }
+}
+
 seer_status init_attn_mma(seer_ctx* ctx) {
   (void)ctx;
   cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMmaSmem);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(block_max_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBmSmem);
   return e == cudaSuccess ? SEER_OK : SEER_ERR_CUDA;
+}
+
+int launch_block_max(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const int32_t* row_ptr,
+                     const int32_t* col_idx, const float* lse, float* out, cudaStream_t stream) {
+  if (m.rows == 0) return 0;
+  block_max_kernel<<<(unsigned)m.rows, kMmaThreads, kBmSmem, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, row_ptr,
+                                                                       col_idx, lse, out, ctx->d_status);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 1 : -(int)e;
 }
 
 int launch_attn_mma(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,

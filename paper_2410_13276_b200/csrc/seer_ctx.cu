@@ -309,6 +309,26 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   return SEER_OK;
 }
 
+seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k,
+                                const int32_t* row_ptr, const int32_t* col_idx, const float* lse, float* block_max,
+                                void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!ctx || !shape) return SEER_ERR_INVALID_ARG;
+  ShapeTotals t;
+  seer_status st = shape_totals(shape, &t);
+  if (st != SEER_OK) return st;
+  if (t.total_blocks == 0) return SEER_OK;
+  if (!q || !k || !row_ptr || !lse) return SEER_ERR_INVALID_ARG;
+  SeqMeta m; int slot;
+  st = prepare(ctx, shape, stream, &m, &slot);
+  if (st != SEER_OK) return st;
+  int n = launch_block_max(ctx, m, q, k, row_ptr, col_idx, lse, block_max, stream);
+  finish_call(ctx, slot, stream);
+  if (n < 0) return SEER_ERR_CUDA;
+  ctx->launches += n;
+  return SEER_OK;
+}
+
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl) {
   if (!ctx || (impl != 0 && impl != 1)) return SEER_ERR_INVALID_ARG;
   ctx->attn_impl = impl;

@@ -74,6 +74,17 @@ class Prefill:
         [heads, n * 128, 128] matching the pooling subsets in `options`."""
         B.seer_gate_scores_ex(self.ctx, self.shape, options, self.q, self.k, wq, wk, self.scores, self.ws, stream)
 
+    def block_max(self, stream=None):
+        """Max-pooled attention map on the listed blocks (Eq. 2) from the lse of the last `attn` call; returns the
+        device tensor [col_capacity] fp32 aligned with col_idx."""
+        if self.lse is None:
+            raise ValueError("block_max needs the lse output: construct with want_lse=True")
+        if getattr(self, "bmax", None) is None or self.bmax.numel() < self.col_idx.numel():
+            self.bmax = torch.empty(max(self.col_idx.numel(), 1), dtype=torch.float32, device=self.device)
+        B.seer_attn_block_max(self.ctx, self.shape, self.q, self.k, self.row_ptr, self.col_idx, self.lse, self.bmax,
+                              stream)
+        return self.bmax
+
     def mask(self, params: B.seer_mask_params, stream=None):
         B.seer_block_mask(self.ctx, self.shape, self.scores, params, self.row_ptr, self.col_idx, self.col_capacity,
                           self.nnz, None, stream)

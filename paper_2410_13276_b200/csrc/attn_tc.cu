@@ -217,11 +217,6 @@ constexpr uint32_t make_idesc(bool a_mn_major, bool b_mn_major) {
 constexpr uint32_t kIdescS = make_idesc(false, false);
 constexpr uint32_t kIdescPV = make_idesc(true, true);
 
-__device__ __forceinline__ int float_order_int(float x) {   // monotone float -> int map
-  int i = __float_as_int(x);
-  return i ^ ((i >> 31) & 0x7fffffff);
-}
-__device__ __forceinline__ float order_int_float(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -272,6 +267,29 @@ __device__ __forceinline__ int list_fetch(const Item& it, const int32_t* __restr
 __device__ __forceinline__ int list_check(const Item& it, int p, int raw) {
   if (p >= it.nlist) return -1;
   return (raw < 0 || raw > it.i) ? -2 : raw;
+}
+
+// Maximum of each of 16 columns over the 32 lanes of a warp; lanes l and l ^ 1 end with column l >> 1.
+__device__ __forceinline__ float warp_colmax16(const float (&x)[16], int lane) {
+  float a[8], b[4], c[2];
+  {
+    const bool up = (lane & 16) != 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = fmaxf(up ? x[i + 8] : x[i], __shfl_xor_sync(0xffffffffu, up ? x[i] : x[i + 8], 16));
+  }
+  {
+    const bool up = (lane & 8) != 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) b[i] = fmaxf(up ? a[i + 4] : a[i], __shfl_xor_sync(0xffffffffu, up ? a[i] : a[i + 4], 8));
+  }
+  {
+    const bool up = (lane & 4) != 0;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) c[i] = fmaxf(up ? b[i + 2] : b[i], __shfl_xor_sync(0xffffffffu, up ? b[i] : b[i + 2], 4));
+  }
+  const bool up = (lane & 2) != 0;
+  const float d = fmaxf(up ? c[1] : c[0], __shfl_xor_sync(0xffffffffu, up ? c[0] : c[1], 2));
+  return fmaxf(d, __shfl_xor_sync(0xffffffffu, d, 1));
 }
 
 // Sums l[0..63] over the 32 lanes of a warp; lane ends with the totals of columns (2*bitrev-ish) base, base+1
@@ -671,7 +689,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     unsigned char* gsm = smem + kOffGrp + grp * kGrpBytes;
     float* mref = reinterpret_cast<float*>(gsm + kGrpMref);
     float* alpha = reinterpret_cast<float*>(gsm + kGrpAlpha);
-    int* colmax = reinterpret_cast<int*>(gsm + kGrpColmax);
     float* lfin = reinterpret_cast<float*>(gsm + kGrpLfin);
     float* lsum = reinterpret_cast<float*>(gsm + kGrpLsum);
     float* w_a = reinterpret_cast<float*>(smem + kOffW);
@@ -741,26 +758,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             if (masked) softmax_pass<true, true>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
             else softmax_pass<false, true>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
           }
-          if (gt < 64) colmax[gt] = float_order_int(-CUDART_INF_F);
-          named_bar_sync(bar_sync, kGroupThreads);
-#pragma unroll
+          // column maxima of the tile: over the lanes of each warp by shuffles (16 columns at a time: lane pair l, l ^ 1
+          // ends with column l >> 1 of the chunk), over the four warps through shared memory
+#pragma unroll 2
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t sv[16];
             tc_ld16(s_addr + ch * 16, sv);
             tc_wait_ld(sv);
+            float xv[16];
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
               const int c = ch * 16 + e;
               float x = __uint_as_float(sv[e]) * sl2;
               if (!row_live || (diag && key_local > c)) x = -CUDART_INF_F;
-              const int wm = __reduce_max_sync(0xffffffffu, float_order_int(x));
-              if (lane == 0) atomicMax(&colmax[c], wm);
+              xv[e] = x;
             }
+            const float cm = warp_colmax16(xv, lane);
+            if ((lane & 1) == 0) lsum[gw * 64 + ch * 16 + (lane >> 1)] = cm;
           }
           named_bar_sync(bar_sync, kGroupThreads);
           if (gt < 64) {
             const float old = mref[gt];
-            float nm = fmaxf(old, order_int_float(colmax[gt]) + kRefShift);
+            const float cm = fmaxf(fmaxf(lsum[gt], lsum[64 + gt]), fmaxf(lsum[128 + gt], lsum[192 + gt]));
+            float nm = fmaxf(old, cm + kRefShift);
             if (nm == -CUDART_INF_F) nm = 0.f;           // nothing visible in this column yet
             alpha[gt] = old == -CUDART_INF_F ? 0.f : exp2f(old - nm);
             mref[gt] = nm;
@@ -782,7 +802,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             l_part[c] = (t < 2 || a < 9.3e-10f) ? 0.f : l_part[c] * a;
           }
           if (t >= 2) {                                  // this group already accumulated into O^T for this item
-#pragma unroll
+#pragma unroll 1
             for (int ch = 0; ch < 4; ++ch) {
               uint32_t ov[16];
               tc_ld16(tmem + lane_addr + col_o(grp) + ch * 16, ov);

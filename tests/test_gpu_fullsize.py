@@ -121,3 +121,32 @@ def test_threshold_workloads_full_size(rt, name, heads):
     w_spec = W.make_workload(name + "s").masks[0]            # same mask recipe as the full-size workload
     spec = W.MaskSpec(W.MODE_THRESHOLD, threshold=golden_threshold(name), flags=w_spec.flags)
     check_workload(rt, name, [spec], sample_heads=heads, rows_per_head=2)
+
+
+def test_c3_bench_configuration_all_rows_cross_check(rt):
+    """Every output row of the bench workload, not a sample: the tcgen05 kernel against the independent mma.sync kernel
+    (different tiling, layout and softmax scheme; itself checked against the oracle on the small cases) on the same
+    lists.  Both round P and o to bf16, so the bound is the attention tolerance between two results of that kind."""
+    import torch
+    B, Prefill, ctx = rt
+    w = W.make_workload("c3")
+    p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    p.run(B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=10, flags=3))
+    assert p.status() == 0
+    o_tc = p.o.float().clone()
+    lse_tc = p.lse.clone()
+    B.seer_set_attn_impl(ctx, 1)
+    try:
+        p.o.fill_(float("nan"))
+        p.attn()
+        assert p.status() == 0
+    finally:
+        B.seer_set_attn_impl(ctx, 0)
+    o_mma = p.o.float()
+    assert not torch.isnan(o_mma).any() and not torch.isnan(o_tc).any()
+    err = (o_tc - o_mma).abs()
+    assert bool((err <= 2e-2 + 1e-2 * o_mma.abs()).all()), float(err.max())
+    rms = err.pow(2).sum(-1).sqrt() / o_mma.pow(2).sum(-1).sqrt().clamp_min(1e-30)
+    assert float(rms.max()) <= 2e-2, float(rms.max())
+    assert bool(((lse_tc - p.lse).abs() <= 2e-3 + 1e-3 * p.lse.abs()).all())

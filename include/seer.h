@@ -140,12 +140,17 @@ seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);
 /* Synchronises `stream`, returns the device status word (SEER_OK if nothing was raised) and clears it. */
 seer_status seer_poll_device_status(seer_ctx* ctx, void* stream);
 
-/* Whole path from HOST buffers: copies q, k, v, Wq, Wk to the device, runs seer_gate_scores -> seer_block_mask ->
- * seer_sparse_attn and copies o (and lse if lse_host is not NULL) back, all enqueued on `stream` (Sec. 3.3: "Inference with
- * SeerAttention").  Host buffers should be page-locked for the copies to be asynchronous; they must stay valid, and
- * o_host must not be read, until the stream has been synchronised.  `arena` is a caller-owned DEVICE buffer of at least
- * seer_prefill_host_arena_bytes(shape) bytes, 256-byte aligned, that holds every intermediate; the call allocates nothing.
- * col_idx inside the arena is sized for the full causal mask, so SEER_ERR_CAPACITY cannot occur. */
+/* Whole path from HOST buffers (Sec. 3.3: "Inference with SeerAttention"): for one KV head at a time (with the query heads
+ * of its group: the path is independent per KV head) it copies that slice of q, k, v, Wq, Wk to the device, runs
+ * seer_gate_scores -> seer_block_mask -> seer_sparse_attn on it and copies the slice of o (and of lse if lse_host is not
+ * NULL) back.  The copy of slice s + 1 and the read-back of slice s - 1 run on two copy streams of the context while the
+ * kernels of slice s run on `stream`; everything is ordered after the work already on `stream`, and `stream` is complete
+ * only when the last read-back is.  The result is bit for bit that of the three calls on device-resident tensors.
+ * Host buffers should be page-locked for the copies to be asynchronous; they must stay valid, and o_host must not be read,
+ * until `stream` has been synchronised.  `arena` is a caller-owned DEVICE buffer of at least
+ * seer_prefill_host_arena_bytes(shape) bytes, 256-byte aligned, that holds two sets of slice inputs / outputs and one set of
+ * slice intermediates; the call allocates nothing.  col_idx inside the arena is sized for the full causal mask of a slice,
+ * so SEER_ERR_CAPACITY cannot occur.  One call at a time per context. */
 size_t seer_prefill_host_arena_bytes(const seer_shape* shape);
 seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void* q_host, const void* k_host,
                               const void* v_host, const float* Wq_host, const float* Wk_host,

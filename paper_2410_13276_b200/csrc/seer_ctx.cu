@@ -173,6 +173,13 @@ seer_status seer_create(seer_ctx** out, int device) {
          cudaEventCreateWithFlags(&s.ready, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&s.last_use, cudaEventDisableTiming) == cudaSuccess;
   }
+  if (ok) ok = cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < 2; ++i)
+    ok = cudaEventCreateWithFlags(&ctx->ev_h2d[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&ctx->ev_comp[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&ctx->ev_d2h[i], cudaEventDisableTiming) == cudaSuccess;
   if (ok) ok = init_gate(ctx) == SEER_OK && init_mask(ctx) == SEER_OK && init_attn_mma(ctx) == SEER_OK &&
               init_attn_tc(ctx) == SEER_OK;
   if (!ok) { seer_destroy(ctx); return SEER_ERR_CUDA; }
@@ -192,6 +199,14 @@ void seer_destroy(seer_ctx* ctx) {
     if (s.last_use) cudaEventDestroy(s.last_use);
   }
   if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
+  if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
+  if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+  for (int i = 0; i < 2; ++i) {
+    if (ctx->ev_h2d[i]) cudaEventDestroy(ctx->ev_h2d[i]);
+    if (ctx->ev_comp[i]) cudaEventDestroy(ctx->ev_comp[i]);
+    if (ctx->ev_d2h[i]) cudaEventDestroy(ctx->ev_d2h[i]);
+  }
   delete ctx;
 }
 
@@ -358,35 +373,49 @@ seer_status seer_set_trace_buffer(seer_ctx* ctx, void* device_buffer) {
 }
 
 namespace {
+// seer_prefill_host works on one KV head (and the query heads of its group) at a time: a slice is a problem of its own
+// with num_q_heads = G, num_kv_heads = 1.  The arena holds two sets of slice inputs and outputs (copy of slice s + 1 and
+// read-back of slice s - 1 overlap the kernels of slice s) and one set of intermediates.
 struct ArenaLayout {
-  size_t q, k, v, o, wq, wk, scores, row_ptr, col_idx, nnz, lse, ws, total;
+  size_t q[2], k[2], v[2], o[2], lse[2], wq[2], wk[2], scores, row_ptr, col_idx, nnz, ws, total;
 };
-ArenaLayout arena_layout(const seer_shape* s, const ShapeTotals& t) {
+ArenaLayout arena_layout(const seer_shape* slice, const ShapeTotals& t) {   // shape and totals of ONE slice
   ArenaLayout a;
   size_t p = 0;
   auto take = [&](size_t bytes) { size_t at = p; p = align_up(p + bytes, 256); return at; };
   const size_t T = (size_t)t.total_tokens;
-  a.q = take(T * s->num_q_heads * kHeadDim * 2);
-  a.k = take(T * s->num_kv_heads * kHeadDim * 2);
-  a.v = take(T * s->num_kv_heads * kHeadDim * 2);
-  a.o = take(T * s->num_q_heads * kHeadDim * 2);
-  a.wq = take((size_t)s->num_q_heads * kHeadDim * kGateDim * 4);
-  a.wk = take((size_t)s->num_kv_heads * kHeadDim * kGateDim * 4);
+  for (int b = 0; b < 2; ++b) {
+    a.q[b] = take(T * slice->num_q_heads * kHeadDim * 2);
+    a.k[b] = take(T * kHeadDim * 2);
+    a.v[b] = take(T * kHeadDim * 2);
+    a.o[b] = take(T * slice->num_q_heads * kHeadDim * 2);
+    a.lse[b] = take(T * slice->num_q_heads * 4);
+    a.wq[b] = take((size_t)slice->num_q_heads * kHeadDim * kGateDim * 4);
+    a.wk[b] = take((size_t)kHeadDim * kGateDim * 4);
+  }
   a.scores = take((size_t)t.score_elems * 4);
   a.row_ptr = take(((size_t)t.rows + 1) * 4);
   a.col_idx = take((size_t)t.causal_blocks * 4);
   a.nnz = take(8);
-  a.lse = take(T * s->num_q_heads * 4);
-  a.ws = take(gate_workspace_bytes(t, s));
+  a.ws = take(gate_workspace_bytes(t, slice));
   a.total = p;
   return a;
 }
 }  // namespace
 
+static bool slice_of(const seer_shape* shape, seer_shape* slice, ShapeTotals* t) {
+  *slice = *shape;
+  if (shape->num_kv_heads <= 0 || shape->num_q_heads % shape->num_kv_heads != 0) return false;
+  slice->num_q_heads = shape->num_q_heads / shape->num_kv_heads;
+  slice->num_kv_heads = 1;
+  return shape_totals(slice, t) == SEER_OK;
+}
+
 size_t seer_prefill_host_arena_bytes(const seer_shape* shape) {
-  ShapeTotals t;
-  if (shape_totals(shape, &t) != SEER_OK) return 0;
-  return arena_layout(shape, t).total;
+  ShapeTotals full, t;
+  seer_shape slice;
+  if (!shape || shape_totals(shape, &full) != SEER_OK || !slice_of(shape, &slice, &t)) return 0;
+  return arena_layout(&slice, t).total;
 }
 
 seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void* q_host, const void* k_host,
@@ -395,39 +424,66 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
                               size_t arena_bytes, void* stream_) {
   cudaStream_t stream = (cudaStream_t)stream_;
   if (!ctx || !shape || !params) return SEER_ERR_INVALID_ARG;
-  ShapeTotals t;
-  seer_status st = shape_totals(shape, &t);
+  ShapeTotals full, t;
+  seer_status st = shape_totals(shape, &full);
   if (st != SEER_OK) return st;
-  if (t.total_blocks == 0) return SEER_OK;
+  if (full.total_blocks == 0) return SEER_OK;
   if (!q_host || !k_host || !v_host || !Wq_host || !Wk_host || !o_host) return SEER_ERR_INVALID_ARG;
-  const ArenaLayout a = arena_layout(shape, t);
+  seer_shape slice;
+  if (!slice_of(shape, &slice, &t)) return SEER_ERR_INVALID_ARG;
+  const ArenaLayout a = arena_layout(&slice, t);
   if (!ws_ok(arena, arena_bytes, a.total)) return SEER_ERR_WORKSPACE;
   if (cudaSetDevice(ctx->device) != cudaSuccess) return SEER_ERR_CUDA;
   char* d = (char*)arena;
   const size_t T = (size_t)t.total_tokens;
-  const size_t qb = T * shape->num_q_heads * kHeadDim * 2, kb = T * shape->num_kv_heads * kHeadDim * 2;
-  bool ok = cudaMemcpyAsync(d + a.q, q_host, qb, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-            cudaMemcpyAsync(d + a.k, k_host, kb, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-            cudaMemcpyAsync(d + a.v, v_host, kb, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-            cudaMemcpyAsync(d + a.wq, Wq_host, (size_t)shape->num_q_heads * kHeadDim * kGateDim * 4,
-                            cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-            cudaMemcpyAsync(d + a.wk, Wk_host, (size_t)shape->num_kv_heads * kHeadDim * kGateDim * 4,
-                            cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  if (!ok) return SEER_ERR_CUDA;
-  st = seer_gate_scores(ctx, shape, d + a.q, d + a.k, (const float*)(d + a.wq), (const float*)(d + a.wk),
-                        (float*)(d + a.scores), d + a.ws, a.total - a.ws, stream);
-  if (st != SEER_OK) return st;
-  st = seer_block_mask(ctx, shape, (const float*)(d + a.scores), params, (int32_t*)(d + a.row_ptr),
-                       (int32_t*)(d + a.col_idx), t.causal_blocks, (int64_t*)(d + a.nnz), nullptr, 0, stream);
-  if (st != SEER_OK) return st;
-  st = seer_sparse_attn(ctx, shape, d + a.q, d + a.k, d + a.v, (const int32_t*)(d + a.row_ptr),
-                        (const int32_t*)(d + a.col_idx), d + a.o, lse_host ? (float*)(d + a.lse) : nullptr, nullptr, 0,
-                        stream);
-  if (st != SEER_OK) return st;
-  if (cudaMemcpyAsync(o_host, d + a.o, qb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SEER_ERR_CUDA;
-  if (lse_host &&
-      cudaMemcpyAsync(lse_host, d + a.lse, T * shape->num_q_heads * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-    return SEER_ERR_CUDA;
+  const int Hq = shape->num_q_heads, Hkv = shape->num_kv_heads, G = slice.num_q_heads;
+  const size_t head_bytes = (size_t)kHeadDim * 2;                       // one head of one token
+  const size_t wq_bytes = (size_t)G * kHeadDim * kGateDim * 4, wk_bytes = (size_t)kHeadDim * kGateDim * 4;
+  cudaStream_t h2d = ctx->h2d_stream, d2h = ctx->d2h_stream;
+#define SEER_TRY(call) do { if ((call) != cudaSuccess) return SEER_ERR_CUDA; } while (0)
+  // the copy streams start after whatever precedes this call on the caller's stream
+  SEER_TRY(cudaEventRecord(ctx->ev_start, stream));
+  SEER_TRY(cudaStreamWaitEvent(h2d, ctx->ev_start, 0));
+  SEER_TRY(cudaStreamWaitEvent(d2h, ctx->ev_start, 0));
+  for (int g = 0; g < Hkv; ++g) {
+    const int b = g & 1;
+    // ---- host -> device: the slice's heads are strided in the host tensors ([T, H, 128]) and packed on the device
+    if (g >= 2) SEER_TRY(cudaStreamWaitEvent(h2d, ctx->ev_comp[b], 0));   // slice g - 2 has finished with these buffers
+    SEER_TRY(cudaMemcpy2DAsync(d + a.q[b], (size_t)G * head_bytes, (const char*)q_host + (size_t)g * G * head_bytes,
+                               (size_t)Hq * head_bytes, (size_t)G * head_bytes, T, cudaMemcpyHostToDevice, h2d));
+    SEER_TRY(cudaMemcpy2DAsync(d + a.k[b], head_bytes, (const char*)k_host + (size_t)g * head_bytes, (size_t)Hkv * head_bytes,
+                               head_bytes, T, cudaMemcpyHostToDevice, h2d));
+    SEER_TRY(cudaMemcpy2DAsync(d + a.v[b], head_bytes, (const char*)v_host + (size_t)g * head_bytes, (size_t)Hkv * head_bytes,
+                               head_bytes, T, cudaMemcpyHostToDevice, h2d));
+    SEER_TRY(cudaMemcpyAsync(d + a.wq[b], (const char*)Wq_host + (size_t)g * wq_bytes, wq_bytes, cudaMemcpyHostToDevice, h2d));
+    SEER_TRY(cudaMemcpyAsync(d + a.wk[b], (const char*)Wk_host + (size_t)g * wk_bytes, wk_bytes, cudaMemcpyHostToDevice, h2d));
+    SEER_TRY(cudaEventRecord(ctx->ev_h2d[b], h2d));
+    // ---- the three calls on the slice, on the caller's stream
+    SEER_TRY(cudaStreamWaitEvent(stream, ctx->ev_h2d[b], 0));
+    if (g >= 2) SEER_TRY(cudaStreamWaitEvent(stream, ctx->ev_d2h[b], 0));  // o / lse of slice g - 2 have been read back
+    st = seer_gate_scores(ctx, &slice, d + a.q[b], d + a.k[b], (const float*)(d + a.wq[b]), (const float*)(d + a.wk[b]),
+                          (float*)(d + a.scores), d + a.ws, a.total - a.ws, stream);
+    if (st != SEER_OK) return st;
+    st = seer_block_mask(ctx, &slice, (const float*)(d + a.scores), params, (int32_t*)(d + a.row_ptr),
+                         (int32_t*)(d + a.col_idx), t.causal_blocks, (int64_t*)(d + a.nnz), nullptr, 0, stream);
+    if (st != SEER_OK) return st;
+    st = seer_sparse_attn(ctx, &slice, d + a.q[b], d + a.k[b], d + a.v[b], (const int32_t*)(d + a.row_ptr),
+                          (const int32_t*)(d + a.col_idx), d + a.o[b], lse_host ? (float*)(d + a.lse[b]) : nullptr, nullptr,
+                          0, stream);
+    if (st != SEER_OK) return st;
+    SEER_TRY(cudaEventRecord(ctx->ev_comp[b], stream));
+    // ---- device -> host
+    SEER_TRY(cudaStreamWaitEvent(d2h, ctx->ev_comp[b], 0));
+    SEER_TRY(cudaMemcpy2DAsync((char*)o_host + (size_t)g * G * head_bytes, (size_t)Hq * head_bytes, d + a.o[b],
+                               (size_t)G * head_bytes, (size_t)G * head_bytes, T, cudaMemcpyDeviceToHost, d2h));
+    if (lse_host)
+      SEER_TRY(cudaMemcpyAsync(lse_host + (size_t)g * G * T, d + a.lse[b], (size_t)G * T * 4, cudaMemcpyDeviceToHost, d2h));
+    SEER_TRY(cudaEventRecord(ctx->ev_d2h[b], d2h));
+  }
+  // the caller's stream is complete when the last read-backs are
+  SEER_TRY(cudaStreamWaitEvent(stream, ctx->ev_d2h[(Hkv - 1) & 1], 0));
+  if (Hkv >= 2) SEER_TRY(cudaStreamWaitEvent(stream, ctx->ev_d2h[Hkv & 1], 0));
+#undef SEER_TRY
   return SEER_OK;
 }
 

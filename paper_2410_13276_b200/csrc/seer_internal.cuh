@@ -60,6 +60,10 @@ struct seer_ctx {
   seer::MetaSlot slots[seer::kMetaSlots];
   void* tmap_encode = nullptr;   // cuTensorMapEncodeTiled, resolved at run time
   void* trace = nullptr;         // optional device buffer for the attention kernel's timeline (diagnostics)
+  // seer_prefill_host: copy streams and the events of its two-deep pipeline over KV-head slices
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_h2d[2] = {nullptr, nullptr}, ev_comp[2] = {nullptr, nullptr},
+              ev_d2h[2] = {nullptr, nullptr};
 };
 
 namespace seer {

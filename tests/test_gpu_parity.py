@@ -323,3 +323,33 @@ def test_invalid_arguments_are_rejected_on_the_host(rt):
         B.seer_block_mask(ctx, s, buf, B.make_mask_params(7), buf, buf, 16)
     assert e.value.status == 1
     assert B.seer_poll_device_status(ctx) == 0
+
+
+@pytest.mark.parametrize("cfg", [dict(seed=120, seqlens=[130, 0, 777, 64, 65], hq=6, hkv=2),
+                                 dict(seed=121, seqlens=[1500, 333], hq=8, hkv=4),
+                                 dict(seed=122, seqlens=[200], hq=4, hkv=1)], ids=lambda c: f"s{c['seed']}")
+def test_prefill_host_equals_the_three_calls(rt, cfg):
+    """The host-buffer entry point (pipelined over KV-head slices, copies included) returns bit for bit what the three
+    calls return on device-resident tensors."""
+    import torch
+    B, Prefill, ctx = rt
+    w = W.make_small(**cfg)
+    p = make_prefill(rt, w)
+    params = B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=3, flags=3)
+    p.run(params)
+    assert p.status() == 0
+    o_ref, lse_ref = p.o.cpu(), p.lse.cpu()
+    hq = torch.from_numpy(w.q.view(np.int16)).pin_memory()
+    hk = torch.from_numpy(w.k.view(np.int16)).pin_memory()
+    hv = torch.from_numpy(w.v.view(np.int16)).pin_memory()
+    hwq, hwk = torch.from_numpy(w.wq).pin_memory(), torch.from_numpy(w.wk).pin_memory()
+    ho = torch.full((w.total_tokens, w.num_q_heads, 128), -1, dtype=torch.int16).pin_memory()
+    hl = torch.full((w.num_q_heads, w.total_tokens), float("nan"), dtype=torch.float32).pin_memory()
+    arena = torch.empty(B.seer_prefill_host_arena_bytes(p.shape), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                  # twice: the second call reuses the pipeline's events and buffers
+        B.seer_prefill_host(ctx, p.shape, hq, hk, hv, hwq, hwk, params, ho, hl, arena)
+        torch.cuda.synchronize()
+        assert B.seer_poll_device_status(ctx) == 0
+        assert torch.equal(ho.view(torch.bfloat16), o_ref)
+        assert torch.equal(hl, lse_ref)
+

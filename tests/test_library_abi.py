@@ -39,7 +39,9 @@ def test_sizing_helpers_closed_forms(lib):
     assert B.seer_causal_blocks(v) == 27891200
     r = B.make_shape([0, 65, 65, 130], 2, 1)                 # ragged, with an empty sequence
     assert B.seer_mask_rows(r) == 2 * (2 + 0 + 2) and B.seer_scores_elems(r) == 2 * (4 + 0 + 4)
-    assert B.seer_prefill_host_arena_bytes(s) > 3 * 10 ** 9
+    # the host-buffer path works on one KV head (4 query heads) at a time: two sets of slice inputs / outputs
+    # (q, o: 2 x 2 x 134 MB; k, v: 2 x 2 x 33.5 MB) and one set of slice intermediates (scores 67 MB, lists 33.6 MB)
+    assert 0.75e9 < B.seer_prefill_host_arena_bytes(s) < 0.85e9
 
 
 def test_invalid_shapes_are_rejected_without_a_gpu(lib):

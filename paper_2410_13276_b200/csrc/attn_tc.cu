@@ -9,19 +9,23 @@
 // so every MMA row is useful for arbitrary lists (an odd list pads half a tile once).
 //
 // Softmax in this orientation: a thread owns one key row of S^T (64 query columns).  The per-query running reference
-// m[c] lives in shared memory and is only a scaling reference, not the exact maximum: p = 2^(s - m[c]).  As long as no
-// entry of a tile exceeds its reference by more than 2^8 the tile needs no cross-thread reduction at all; otherwise the
-// work group computes exact column maxima, rebases m, rescales its partial sums and the O accumulator, and recomputes
-// the tile.  Row sums are per-thread partials combined once per work item.
+// m[c] is only a scaling reference, not the exact maximum: p = 2^(s - m[c]); it sits 2^7 above the column maximum it was
+// taken from, and every lane keeps a copy of the 64 references in TMEM (a shared-memory read in the inner loop would
+// queue behind the tensor pipe's operand traffic).  As long as no entry of a tile reaches 2^8 times its reference
+// maximum -- seen as "some p >= 2" on the packed bf16 words -- the tile needs no cross-thread reduction at all;
+// otherwise the group computes exact column maxima (warp shuffles, then four values per column through shared memory),
+// moves the references, rescales its partial sums and the O accumulator, and recomputes the tile.  Row sums are
+// per-thread partials combined once per work item.
 //
 // Roles (512 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + issuer of the S^T MMAs, warp 3 = issuer
 // of the P V MMAs (one thread can start a tcgen05.mma only every 64 clocks, so the two products are issued from two
 // threads), warps 4-7 and 8-11 = two softmax groups, warps 12-15 = cp.async producers for V (a warp keeps only ~14 KB of
-// cp.async in flight, so four share a tile).  After the dispatch the helper warpgroups shrink to 72 registers per thread
-// and the softmax warpgroups grow to 184 (setmaxnreg).  The tiles of a work item alternate between the groups (even tiles -> A, odd -> B); each group keeps its own
-// S^T buffers, P^T buffer, O^T accumulator, references and row sums, and the epilogue merges the two partial results
-// through their references.  One persistent CTA per SM walks the work items (longest rows first within each KV head).
-// Every wait is bounded; a wait that runs out raises SEER_ERR_TIMEOUT and the CTA drains and exits.
+// cp.async in flight, so four share a tile).  After the dispatch the helper warpgroups shrink to 56 registers per thread
+// and the softmax warpgroups grow to 200 (setmaxnreg).  The tiles of a work item alternate between the groups (even
+// tiles -> A, odd -> B); each group keeps its own two S^T buffers, two P^T buffers, O^T accumulator, references and row
+// sums, and the epilogue merges the two partial results through their references.  One persistent CTA per SM walks the
+// work items (longest rows first within each KV head).  Every wait is bounded; a wait that runs out raises
+// SEER_ERR_TIMEOUT and the CTA drains and exits.
 #include <cuda.h>
 #include <math_constants.h>
 

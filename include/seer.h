@@ -169,8 +169,8 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
  * intermediate projected vectors and the per-batch offsets live in a fixed array inside the library image: every GPU
  * that loads the library holds SEER_STATIC_SCRATCH_BYTES + 16 KiB for it until the process exits.
  *
- * Limits: shape->batch <= SEER_STATIC_MAX_BATCH and (num_q_heads + num_kv_heads) * total_blocks * 512 bytes (rounded up to
- * 256 per tensor) <= SEER_STATIC_SCRATCH_BYTES, i.e. 16384 (head, block) pairs: e.g. 40 heads x 26000 tokens.  Larger shapes
+ * Limits: shape->batch <= SEER_STATIC_MAX_BATCH and (num_q_heads + num_kv_heads) * total_blocks * 768 bytes (rounded up to
+ * 256 per tensor) <= SEER_STATIC_SCRATCH_BYTES, i.e. 10922 (head, block) pairs: e.g. 40 heads x 17000 tokens.  Larger shapes
  * return SEER_ERR_WORKSPACE and enqueue nothing.
  *
  * First call on a device: looks up the array's device address and raises one kernel's shared-memory limit (no allocation).

@@ -1,9 +1,13 @@
 // AttnGate (Sec. 3.1, Eq. 1) in two kernels:
 //   pool_project_kernel : streams Q and K once (HBM-bound), average-pools each 64-token block per head and
-//                         multiplies the pooled vectors by the head's gate matrix  -> gq, gk (fp32 workspace)
+//                         multiplies the pooled vectors by the head's gate matrix (fp32 on the CUDA cores) -> gq, gk
 //   gate_scores_kernel  : logits = gq gk^T / sqrt(dg) over the causal blocks, row softmax -> scores
-// All gate arithmetic is fp32 on the CUDA cores (tensor-core bf16/tf32 would not hold the 1e-3 relative bound
-// on softmax outputs when logits reach tens).
+// The logits need fp32-grade products (plain bf16 or tf32 tensor-core inputs would not hold the 1e-3 relative bound on
+// softmax outputs when logits reach tens), so gq and gk are stored as three bf16 planes each, x = hi + mid + lo with
+// every part the bf16 rounding of what is left, and the product is taken on the tensor cores (mma.sync, fp32
+// accumulation) as the six terms hi*hi + hi*mid + mid*hi + hi*lo + lo*hi + mid*mid: what is dropped is below 2^-24 of
+// the product.
+#include <cuda_bf16.h>
 #include <math_constants.h>
 
 #include <cstddef>
@@ -15,6 +19,19 @@ namespace seer {
 
 // ----------------------------------------------------------------------------------------------- kernel 1
 constexpr int kPoolThreads = 256;
+
+// x = hi + mid + lo, each part the bf16 (round-to-nearest-even) of the remainder; the three planes of a tensor lie
+// `plane` elements apart.
+__device__ __forceinline__ void store_split3(uint16_t* __restrict__ dst, size_t plane, float x) {
+  const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+  const float r1 = x - __bfloat162float(hi);
+  const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+  const float r2 = r1 - __bfloat162float(mid);
+  const __nv_bfloat16 lo = __float2bfloat16_rn(r2);
+  dst[0] = __bfloat16_as_ushort(hi);
+  dst[plane] = __bfloat16_as_ushort(mid);
+  dst[2 * plane] = __bfloat16_as_ushort(lo);
+}
 
 __device__ __forceinline__ uint4 ld_stream_16(const void* p) {
   uint4 r;
@@ -34,8 +51,8 @@ __device__ __forceinline__ void acc_bf16x8(float (&a)[8], const uint4& u) {
 // neighbouring 256-byte segments of the same token rows.
 __global__ void __launch_bounds__(kPoolThreads)
 pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-                    const float* __restrict__ Wq, const float* __restrict__ Wk, float* __restrict__ gq,
-                    float* __restrict__ gk) {
+                    const float* __restrict__ Wq, const float* __restrict__ Wk, uint16_t* __restrict__ gq,
+                    uint16_t* __restrict__ gk) {
   __shared__ __align__(16) float pooled[kPoolChunk][kHeadDim];
 
   const int heads_total = m.num_q_heads + m.num_kv_heads;
@@ -46,7 +63,8 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
   const int h = is_q ? hh : hh - m.num_q_heads;
   const uint16_t* __restrict__ x = is_q ? q : k;
   const float* __restrict__ W = (is_q ? Wq : Wk) + (size_t)h * kHeadDim * kGateDim;
-  float* __restrict__ out = is_q ? gq : gk;
+  uint16_t* __restrict__ out = is_q ? gq : gk;
+  const size_t plane = (size_t)H * m.total_blocks * kGateDim;   // elements between the hi / mid / lo planes
 
   const int b = find_sequence(m.chunk_off, m.batch, chunk);
   const int s0 = m.cu_seqlens[b], s1 = m.cu_seqlens[b + 1];
@@ -102,7 +120,7 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const int bi = grp * 8 + j;
-    if (bi < nblk) out[obase + (size_t)bi * kGateDim + o] = acc[j];
+    if (bi < nblk) store_split3(out + obase + (size_t)bi * kGateDim + o, plane, acc[j]);
   }
 }
 
@@ -132,8 +150,8 @@ constexpr int kPoolExSmem = kPoolChunk * 3 * kHeadDim * (int)sizeof(float);   //
 
 __global__ void __launch_bounds__(kPoolThreads)
 pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-                       const float* __restrict__ Wq, const float* __restrict__ Wk, float* __restrict__ gq,
-                       float* __restrict__ gk, uint32_t pool_q, uint32_t pool_k, float rope_theta) {
+                       const float* __restrict__ Wq, const float* __restrict__ Wk, uint16_t* __restrict__ gq,
+                       uint16_t* __restrict__ gk, uint32_t pool_q, uint32_t pool_k, float rope_theta) {
   __shared__ __align__(16) float pooled[kPoolChunk][3 * kHeadDim];
 
   const int heads_total = m.num_q_heads + m.num_kv_heads;
@@ -147,7 +165,8 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
   const int width = nparts * kHeadDim;                       // rows of the head's gate matrix
   const uint16_t* __restrict__ x = is_q ? q : k;
   const float* __restrict__ W = (is_q ? Wq : Wk) + (size_t)h * width * kGateDim;
-  float* __restrict__ out = is_q ? gq : gk;
+  uint16_t* __restrict__ out = is_q ? gq : gk;
+  const size_t plane = (size_t)H * m.total_blocks * kGateDim;   // elements between the hi / mid / lo planes
   // offsets of the parts inside the concatenated vector (order: average, max, min)
   const int off_avg = 0;
   const int off_max = (methods & SEER_POOL_AVG) ? kHeadDim : 0;
@@ -243,36 +262,55 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const int bi = grp * 8 + j;
-    if (bi < nblk) out[obase + (size_t)bi * kGateDim + o] = acc[j];
+    if (bi < nblk) store_split3(out + obase + (size_t)bi * kGateDim + o, plane, acc[j]);
   }
 }
 
 // ----------------------------------------------------------------------------------------------- kernel 2
+// 64 score rows of one head per CTA, walked over the causal columns 64 at a time (the next column tile is copied in
+// while the current one is multiplied).  Eight warps; warp w owns rows 16 (w & 3) .. + 15 and the column half w >> 2
+// (mma.sync m16n8k16, bf16 in, fp32 out): per 16-wide k step three A fragments (hi, mid, lo planes of gq) and, for each
+// of its four 8-column groups, three B fragments of gk; six MMAs per group.  Tiles sit in shared memory as
+// [plane][64 rows][128 k] bf16 with the 16-byte chunks of a row XOR-swizzled by the row (conflict-free ldmatrix).
 constexpr int kScoreThreads = 256;
-constexpr int kScoreSmem = 2 * kGateDim * kScoreTile * (int)sizeof(float) + 2 * kScoreTile * (int)sizeof(float);
+constexpr int kPlaneTile = kScoreTile * kGateDim * 2;                       // 16 KB: one plane of a 64 x 128 tile
+constexpr int kScoreSmem = 9 * kPlaneTile + 6 * kScoreTile * (int)sizeof(float);   // A planes, two sets of B planes, row statistics
 
-// Loads a [64 rows x 128] fp32 tile (rows r0.. of src, row stride kGateDim) transposed into dst[k][row].
-__device__ __forceinline__ void load_tile_transposed(float* dst, const float* __restrict__ src, int r0, int rows_valid) {
-  for (int idx = threadIdx.x; idx < kScoreTile * (kGateDim / 4); idx += kScoreThreads) {
-    const int row = idx & (kScoreTile - 1);
-    const int k4 = idx / kScoreTile;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row < rows_valid) v = __ldg(reinterpret_cast<const float4*>(src + (size_t)(r0 + row) * kGateDim) + k4);
-    dst[(k4 * 4 + 0) * kScoreTile + row] = v.x;
-    dst[(k4 * 4 + 1) * kScoreTile + row] = v.y;
-    dst[(k4 * 4 + 2) * kScoreTile + row] = v.z;
-    dst[(k4 * 4 + 3) * kScoreTile + row] = v.w;
+__device__ __forceinline__ uint32_t gs_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t gs_tile_off(int row, int chunk) { return (uint32_t)(row * 256 + ((chunk ^ (row & 7)) << 4)); }
+__device__ __forceinline__ void gs_ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void gs_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// Copies rows r0 .. r0+63 of the three planes of src ([rows][128] bf16 each, `plane` elements apart) into dst; rows at or
+// beyond rows_valid are zero-filled.
+__device__ __forceinline__ void gs_load_planes(uint32_t dst, const uint16_t* __restrict__ src, size_t plane, int r0,
+                                               int rows_valid) {
+  for (int idx = threadIdx.x; idx < 3 * kScoreTile * 16; idx += kScoreThreads) {
+    const int pl = idx / (kScoreTile * 16), rem = idx - pl * (kScoreTile * 16);
+    const int row = rem >> 4, chunk = rem & 15;
+    const bool ok = row < rows_valid;
+    const uint16_t* g = src + (size_t)pl * plane + (size_t)(r0 + (ok ? row : 0)) * kGateDim + chunk * 8;
+    const int sz = ok ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + (uint32_t)pl * kPlaneTile + gs_tile_off(row, chunk)),
+                 "l"(g), "r"(sz) : "memory");
   }
 }
 
 // grid.x = total_tiles * Hq (head fastest; tiles are visited from the last rows, the longest, to the first)
 __global__ void __launch_bounds__(kScoreThreads)
-gate_scores_kernel(SeqMeta m, const float* __restrict__ gq, const float* __restrict__ gk, float* __restrict__ scores) {
-  extern __shared__ __align__(16) float smem[];
-  float* As = smem;                              // [128][64]  gq tile, k-major
-  float* Bs = smem + kGateDim * kScoreTile;      // [128][64]  gk tile, k-major
-  float* row_m = Bs + kGateDim * kScoreTile;     // [64]
-  float* row_l = row_m + kScoreTile;             // [64]
+gate_scores_kernel(SeqMeta m, const uint16_t* __restrict__ gq, const uint16_t* __restrict__ gk, float* __restrict__ scores) {
+  extern __shared__ __align__(128) unsigned char gs_smem[];
+  const uint32_t sA = gs_smem_u32(gs_smem), sB0 = sA + 3 * kPlaneTile;
+  float* row_m = reinterpret_cast<float*>(gs_smem + 9 * kPlaneTile);     // [64]
+  float* row_l = row_m + kScoreTile;                                      // [64]
+  float* part_m = row_l + kScoreTile;                                     // [2 column halves][64]
+  float* part_l = part_m + 2 * kScoreTile;
 
   const int tile_g = m.total_tiles - 1 - (int)(blockIdx.x / m.num_q_heads);
   const int h = blockIdx.x % m.num_q_heads;
@@ -281,104 +319,161 @@ gate_scores_kernel(SeqMeta m, const float* __restrict__ gq, const float* __restr
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
   const int i0 = (tile_g - m.tile_off[b]) * kScoreTile;
   const int rows_valid = min(kScoreTile, nb - i0);
-  const float* gq_h = gq + ((size_t)h * m.total_blocks + m.blk_off[b]) * kGateDim;
-  const float* gk_g = gk + ((size_t)g * m.total_blocks + m.blk_off[b]) * kGateDim;
+  const size_t plane_q = (size_t)m.num_q_heads * m.total_blocks * kGateDim;
+  const size_t plane_k = (size_t)m.num_kv_heads * m.total_blocks * kGateDim;
+  const uint16_t* gq_h = gq + ((size_t)h * m.total_blocks + m.blk_off[b]) * kGateDim;
+  const uint16_t* gk_g = gk + ((size_t)g * m.total_blocks + m.blk_off[b]) * kGateDim;
   float* sc = scores + m.score_off[b] + (size_t)h * nb * nb;
 
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wr = warp & 3, wc = warp >> 2;                               // row group, column half
+  const int gid = lane >> 2, tig = lane & 3;
   const float scale = rsqrtf((float)kGateDim);
-  const bool vec_ok = (nb & 3) == 0 && (m.score_off[b] & 3) == 0;
-
-  load_tile_transposed(As, gq_h, i0, rows_valid);
-
-  float run_m[4], run_l[4];
-#pragma unroll
-  for (int r = 0; r < 4; ++r) { run_m[r] = -CUDART_INF_F; run_l[r] = 0.f; }
+  const bool vec_ok = (nb & 1) == 0 && (m.score_off[b] & 1) == 0;        // 8-byte stores of column pairs
 
   const int last_col = i0 + rows_valid - 1;
-  for (int j0 = 0; j0 <= last_col; j0 += kScoreTile) {
-    __syncthreads();  // previous tile's Bs reads done (and As visible on the first pass)
-    load_tile_transposed(Bs, gk_g, j0, min(kScoreTile, nb - j0));
+  gs_load_planes(sA, gq_h, plane_q, i0, rows_valid);
+  gs_load_planes(sB0, gk_g, plane_k, 0, min(kScoreTile, nb));
+  asm volatile("cp.async.commit_group;" ::: "memory");
+
+  float run_m[2] = {-CUDART_INF_F, -CUDART_INF_F}, run_l[2] = {0.f, 0.f};
+  // the warp's A fragments (16 rows x 128 k, three planes) stay in registers for the whole row tile
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  uint32_t a[8][3][4];
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+    for (int pl = 0; pl < 3; ++pl) {
+      const int row = wr * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      gs_ldsm_x4(a[ks][pl], sA + (uint32_t)pl * kPlaneTile + gs_tile_off(row, ks * 2 + (lane >> 4)));
+    }
+  int buf = 0;
+  for (int j0 = 0; j0 <= last_col; j0 += kScoreTile, buf ^= 1) {
+    const uint32_t sB = sB0 + (uint32_t)buf * 3 * kPlaneTile;
+    __syncthreads();                                   // the other B buffer's fragments have been read
+    if (j0 + kScoreTile <= last_col)
+      gs_load_planes(sB0 + (uint32_t)(buf ^ 1) * 3 * kPlaneTile, gk_g, plane_k, j0 + kScoreTile, min(kScoreTile, nb - j0 - kScoreTile));
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 1;" ::: "memory");   // everything but the copy just started has landed
     __syncthreads();
     float acc[4][4];
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
+    for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-      for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
-#pragma unroll 8
-    for (int kk = 0; kk < kGateDim; ++kk) {
-      const float4 a = *reinterpret_cast<const float4*>(As + kk * kScoreTile + ty * 4);
-      const float4 bb = *reinterpret_cast<const float4*>(Bs + kk * kScoreTile + tx * 4);
-      const float av[4] = {a.x, a.y, a.z, a.w};
-      const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+      for (int c = 0; c < 4; ++c) acc[nt][c] = 0.f;
 #pragma unroll
-      for (int r = 0; r < 4; ++r)
+    for (int kk = 0; kk < 8; kk += 2) {                // two 16-wide k steps per pass (one B ldmatrix.x4 covers both)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], bv[c], acc[r][c]);
+      for (int nt = 0; nt < 4; ++nt) {
+        uint32_t bf[3][4];                             // [plane]: b0, b1 of step kk, then of step kk + 1
+#pragma unroll
+        for (int pl = 0; pl < 3; ++pl)
+          gs_ldsm_x4(bf[pl], sB + (uint32_t)pl * kPlaneTile + gs_tile_off((wc * 4 + nt) * 8 + (lane & 7), kk * 2 + (lane >> 3)));
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2) {
+          // smallest terms first: hi*lo, lo*hi, mid*mid, then hi*mid, mid*hi, then hi*hi
+          gs_mma(acc[nt], a[kk + s2][0], bf[2][2 * s2], bf[2][2 * s2 + 1]);
+          gs_mma(acc[nt], a[kk + s2][2], bf[0][2 * s2], bf[0][2 * s2 + 1]);
+          gs_mma(acc[nt], a[kk + s2][1], bf[1][2 * s2], bf[1][2 * s2 + 1]);
+          gs_mma(acc[nt], a[kk + s2][0], bf[1][2 * s2], bf[1][2 * s2 + 1]);
+          gs_mma(acc[nt], a[kk + s2][1], bf[0][2 * s2], bf[0][2 * s2 + 1]);
+          gs_mma(acc[nt], a[kk + s2][0], bf[0][2 * s2], bf[0][2 * s2 + 1]);
+        }
+      }
     }
+    // thread holds rows (gid, gid + 8) of the warp's 16 and columns (4 wc + nt) * 8 + 2 * tig + {0, 1}
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int i = i0 + ty * 4 + r;
+    for (int e = 0; e < 2; ++e) {
+      const int i = i0 + wr * 16 + gid + e * 8;
       if (i >= nb) continue;
-      const int jb = j0 + tx * 4;
-      float x[4];
+      float x[4][2];
       float tmax = -CUDART_INF_F;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        x[c] = (jb + c <= i) ? acc[r][c] * scale : -CUDART_INF_F;
-        tmax = fmaxf(tmax, x[c]);
-      }
-      if (jb <= i) {
-        const float nm = fmaxf(run_m[r], tmax);
-        float s = 0.f;
+      for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) s += (jb + c <= i) ? expf(x[c] - nm) : 0.f;
-        run_l[r] = run_l[r] * expf(run_m[r] - nm) + s;   // exp(-inf) = 0 on the first contribution
-        run_m[r] = nm;
-        float* dst = sc + (size_t)i * nb + jb;
-        if (vec_ok && jb + 3 <= i) {
-          *reinterpret_cast<float4*>(dst) = make_float4(x[0], x[1], x[2], x[3]);
+        for (int c = 0; c < 2; ++c) {
+          const int j = j0 + (wc * 4 + nt) * 8 + 2 * tig + c;
+          x[nt][c] = j <= i ? acc[nt][2 * e + c] * scale : -CUDART_INF_F;
+          tmax = fmaxf(tmax, x[nt][c]);
+        }
+      if (tmax == -CUDART_INF_F) continue;             // nothing causal for this thread in this tile
+      const float nm = fmaxf(run_m[e], tmax);
+      float sum = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int c = 0; c < 2; ++c) sum += x[nt][c] == -CUDART_INF_F ? 0.f : __expf(x[nt][c] - nm);
+      run_l[e] = run_l[e] * __expf(run_m[e] - nm) + sum;  // exp(-inf) = 0 on the first contribution
+      run_m[e] = nm;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        const int j = j0 + (wc * 4 + nt) * 8 + 2 * tig;
+        float* dst = sc + (size_t)i * nb + j;
+        if (vec_ok && j + 1 <= i) {
+          *reinterpret_cast<float2*>(dst) = make_float2(x[nt][0], x[nt][1]);
         } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            if (jb + c <= i) dst[c] = x[c];
+          if (j <= i) dst[0] = x[nt][0];
+          if (j + 1 <= i) dst[1] = x[nt][1];
         }
       }
     }
   }
-  // combine the 16 partial (max, sum) pairs of each row
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  // combine the partial (max, sum) pairs of each row: the four lanes of a quad, then the two column halves
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    float mm = run_m[r], ll = run_l[r];
+  for (int e = 0; e < 2; ++e) {
+    float mm = run_m[e], ll = run_l[e];
 #pragma unroll
-    for (int off = 1; off < 16; off <<= 1) {
+    for (int off = 1; off < 4; off <<= 1) {
       const float om = __shfl_xor_sync(0xffffffffu, mm, off);
       const float ol = __shfl_xor_sync(0xffffffffu, ll, off);
       const float nm = fmaxf(mm, om);
-      const float fa = (mm == -CUDART_INF_F) ? 0.f : expf(mm - nm);
-      const float fb = (om == -CUDART_INF_F) ? 0.f : expf(om - nm);
+      const float fa = (mm == -CUDART_INF_F) ? 0.f : __expf(mm - nm);
+      const float fb = (om == -CUDART_INF_F) ? 0.f : __expf(om - nm);
       ll = ll * fa + ol * fb;
       mm = nm;
     }
-    if (tx == 0) { row_m[ty * 4 + r] = mm; row_l[ty * 4 + r] = ll; }
+    if (tig == 0) { part_m[wc * kScoreTile + wr * 16 + gid + e * 8] = mm; part_l[wc * kScoreTile + wr * 16 + gid + e * 8] = ll; }
   }
   __syncthreads();
-  // normalise in place: the logits this CTA just wrote are re-read (L2) and replaced by exp(x - m) / l
-  for (int r = 0; r < rows_valid; ++r) {
+  if (threadIdx.x < kScoreTile) {
+    const float m0 = part_m[threadIdx.x], m1 = part_m[kScoreTile + threadIdx.x];
+    const float nm = fmaxf(m0, m1);
+    const float f0 = (m0 == -CUDART_INF_F) ? 0.f : __expf(m0 - nm), f1 = (m1 == -CUDART_INF_F) ? 0.f : __expf(m1 - nm);
+    row_m[threadIdx.x] = nm;
+    row_l[threadIdx.x] = part_l[threadIdx.x] * f0 + part_l[kScoreTile + threadIdx.x] * f1;
+  }
+  __syncthreads();
+  // normalise in place: the logits this CTA just wrote are re-read (L2) and replaced by exp(x - m) / l; a warp per row,
+  // four columns per lane and step, so that many independent loads are in flight
+  const bool vec4 = (nb & 3) == 0 && (m.score_off[b] & 3) == 0;
+  for (int r = warp; r < rows_valid; r += kScoreThreads / 32) {
     const int i = i0 + r;
     const float mm = row_m[r];
     const float inv = 1.0f / row_l[r];
     float* dst = sc + (size_t)i * nb;
-    for (int j = threadIdx.x; j <= i; j += kScoreThreads) dst[j] = expf(dst[j] - mm) * inv;
+    if (vec4) {
+      const int full = (i + 1) & ~3;                   // columns 0 .. full-1 in whole float4s
+      for (int j = lane * 4; j < full; j += 128) {
+        float4 v = *reinterpret_cast<float4*>(dst + j);
+        v.x = __expf(v.x - mm) * inv; v.y = __expf(v.y - mm) * inv; v.z = __expf(v.z - mm) * inv; v.w = __expf(v.w - mm) * inv;
+        *reinterpret_cast<float4*>(dst + j) = v;
+      }
+      for (int j = full + lane; j <= i; j += 32) dst[j] = __expf(dst[j] - mm) * inv;
+    } else {
+      for (int j = lane; j <= i; j += 32) dst[j] = __expf(dst[j] - mm) * inv;
+    }
   }
 }
 
 int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const float* Wq, const float* Wk,
                 float* scores, void* ws, cudaStream_t stream) {
   (void)ctx;
-  size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * sizeof(float) + 255) / 256 * 256;
-  float* gq = (float*)ws;
-  float* gk = (float*)((char*)ws + gq_bytes);
+  // three bf16 planes per tensor (hi, mid, lo of the fp32 value)
+  size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * 6 + 255) / 256 * 256;
+  uint16_t* gq = (uint16_t*)ws;
+  uint16_t* gk = (uint16_t*)((char*)ws + gq_bytes);
   const unsigned grid1 = (unsigned)m.total_chunks * (unsigned)(m.num_q_heads + m.num_kv_heads);
   pool_project_kernel<<<grid1, kPoolThreads, 0, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, Wq, Wk, gq, gk);
   const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
@@ -390,9 +485,10 @@ int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, c
 int launch_gate_ex(seer_ctx* ctx, const SeqMeta& m, const seer_gate_options& opt, const void* q, const void* k,
                    const float* Wq, const float* Wk, float* scores, void* ws, cudaStream_t stream) {
   (void)ctx;
-  size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * sizeof(float) + 255) / 256 * 256;
-  float* gq = (float*)ws;
-  float* gk = (float*)((char*)ws + gq_bytes);
+  // three bf16 planes per tensor (hi, mid, lo of the fp32 value)
+  size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * 6 + 255) / 256 * 256;
+  uint16_t* gq = (uint16_t*)ws;
+  uint16_t* gk = (uint16_t*)((char*)ws + gq_bytes);
   const unsigned grid1 = (unsigned)m.total_chunks * (unsigned)(m.num_q_heads + m.num_kv_heads);
   pool_project_ex_kernel<<<grid1, kPoolThreads, 0, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, Wq, Wk, gq, gk,
                                                               opt.pool_q, opt.pool_k, opt.rope_theta);

@@ -50,9 +50,9 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
 }
 
 size_t gate_workspace_bytes(const ShapeTotals& t, const seer_shape* s) {
-  // projected pooled Q [Hq, blocks, dg] and K [Hkv, blocks, dg], fp32
-  size_t gq = align_up((size_t)s->num_q_heads * t.total_blocks * kGateDim * sizeof(float), 256);
-  size_t gk = align_up((size_t)s->num_kv_heads * t.total_blocks * kGateDim * sizeof(float), 256);
+  // projected pooled Q [Hq, blocks, dg] and K [Hkv, blocks, dg], each as three bf16 planes (hi, mid, lo of the fp32 value)
+  size_t gq = align_up((size_t)s->num_q_heads * t.total_blocks * kGateDim * 6, 256);
+  size_t gk = align_up((size_t)s->num_kv_heads * t.total_blocks * kGateDim * 6, 256);
   return gq + gk;
 }
 

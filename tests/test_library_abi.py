@@ -33,7 +33,7 @@ def test_sizing_helpers_closed_forms(lib):
     assert B.seer_mask_rows(s) == 32 * 2048
     assert B.seer_scores_elems(s) == 32 * 2048 * 2048
     assert B.seer_causal_blocks(s) == 32 * 2048 * 2049 // 2 == 67141632
-    assert B.seer_workspace_bytes(s) == (32 + 8) * 2048 * 128 * 4
+    assert B.seer_workspace_bytes(s) == (32 + 8) * 2048 * 128 * 6     # projected pooled Q, K: three bf16 planes each
     v = B.make_shape([0, 8192, 8192 + 16384, 8192 + 16384 + 32768, 122880], 40, 8)
     assert B.seer_mask_rows(v) == 40 * (128 + 256 + 512 + 1024) == 76800
     assert B.seer_causal_blocks(v) == 27891200

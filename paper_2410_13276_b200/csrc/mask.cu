@@ -88,34 +88,64 @@ count_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, in
   if (lane == 0) row_ptr[r + 1] = c;
 }
 
-// Single CTA: in-place inclusive scan of row_ptr[1..rows]; row_ptr[0] = 0.
+// Single CTA: in-place inclusive scan of row_ptr[1..rows]; row_ptr[0] = 0.  Tiles of 4096 counts go through shared
+// memory (coalesced loads and stores), four consecutive counts per thread, warp shuffles inside a warp, one carry per tile.
 __global__ void __launch_bounds__(1024)
 scan_kernel(int64_t rows, int32_t* __restrict__ row_ptr, int64_t col_capacity, int64_t* __restrict__ nnz_out,
             int* __restrict__ status) {
-  __shared__ long long part[1024];
-  const int t = threadIdx.x;
-  const int64_t per = (rows + 1023) / 1024;
-  const int64_t lo = min(rows, t * per), hi = min(rows, lo + per);
-  long long s = 0;
-  for (int64_t r = lo; r < hi; ++r) s += row_ptr[r + 1];
-  part[t] = s;
-  __syncthreads();
-  for (int off = 1; off < 1024; off <<= 1) {
-    long long v = t >= off ? part[t - off] : 0;
+  __shared__ int32_t tile[4096];
+  __shared__ long long warp_tot[32];
+  __shared__ long long carry_s;
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  long long carry = 0;
+  for (int64_t base = 0; base < rows; base += 4096) {
+    const int n = (int)min((int64_t)4096, rows - base);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int idx = t + k * 1024;
+      tile[idx] = idx < n ? row_ptr[base + idx + 1] : 0;
+    }
     __syncthreads();
-    part[t] += v;
+    long long v[4];
+    v[0] = tile[4 * t];
+    v[1] = v[0] + tile[4 * t + 1];
+    v[2] = v[1] + tile[4 * t + 2];
+    v[3] = v[2] + tile[4 * t + 3];
+    long long incl = v[3];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const long long o = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += o;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-  }
-  long long run = part[t] - s;   // exclusive prefix of this thread's segment
-  for (int64_t r = lo; r < hi; ++r) {
-    run += row_ptr[r + 1];
-    row_ptr[r + 1] = (int32_t)run;
+    if (warp == 0) {
+      long long w = warp_tot[lane];
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const long long o = __shfl_up_sync(0xffffffffu, w, off);
+        if (lane >= off) w += o;
+      }
+      warp_tot[lane] = w;                              // inclusive over warps
+      if (lane == 31) carry_s = w;                     // total of the tile
+    }
+    __syncthreads();
+    const long long before = carry + (warp > 0 ? warp_tot[warp - 1] : 0) + (incl - v[3]);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) tile[4 * t + k] = (int32_t)(before + v[k]);
+    carry += carry_s;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int idx = t + k * 1024;
+      if (idx < n) row_ptr[base + idx + 1] = tile[idx];
+    }
+    __syncthreads();
   }
   if (t == 0) {
     row_ptr[0] = 0;
-    const long long nnz = part[1023];
-    if (nnz_out) *nnz_out = nnz;
-    if (nnz > col_capacity) atomicCAS(status, 0, (int)SEER_ERR_CAPACITY);
+    if (nnz_out) *nnz_out = carry;
+    if (carry > col_capacity) atomicCAS(status, 0, (int)SEER_ERR_CAPACITY);
   }
 }
 
@@ -152,12 +182,16 @@ fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, con
   uint32_t* keys = key_smem + (size_t)warp * stage_cap;
   const bool staged = n <= stage_cap;
   int c = 0;
+  uint32_t k_and = 0xffffffffu, k_or = 0u;     // over the candidates' keys: the bits all of them share are k_and | ~k_or
   for (int j = lane; j < n; j += 32) {
     const uint32_t kk = is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]);
     if (staged) keys[j] = kk;
     c += kk != 0u;
+    if (kk != 0u) { k_and &= kk; k_or |= kk; }
   }
   const int ncand = warp_sum(c);
+  k_and = __reduce_and_sync(0xffffffffu, k_and);
+  k_or = __reduce_or_sync(0xffffffffu, k_or);
   __syncwarp();
   auto key_at = [&](int j) -> uint32_t {
     return staged ? keys[j] : (is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]));
@@ -173,9 +207,14 @@ fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, con
     // Radix select, 8 bits per pass from the top: histogram the current digit of the keys that match the prefix found
     // so far (warp-private shared-memory bins), walk the bins from the largest digit down until `remaining` is covered.
     uint32_t* hist = hist_smem + warp * 256;
-    uint32_t prefix = 0u, prefix_mask = 0u;
+    // The scores of a row are often close together; the leading bits all candidate keys share need no pass: the passes
+    // start at the first 8-bit digit in which two keys differ.
+    const uint32_t differ = k_and ^ k_or;                                 // bit set: not all keys agree there
+    const int top_shift = differ == 0u ? 0 : ((31 - __clz(differ)) >> 3) << 3;   // shift of the highest differing digit
+    uint32_t prefix_mask = top_shift >= 24 ? 0u : ~((1u << (top_shift + 8)) - 1u);
+    uint32_t prefix = k_or & prefix_mask;                                 // the shared leading digits
     int remaining = take;           // rank (1-based, from the top) still to locate inside the current prefix class
-    for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int shift = top_shift; shift >= 0; shift -= 8) {
       for (int b = lane; b < 256; b += 32) hist[b] = 0u;
       __syncwarp();
       for (int j = lane; j < n; j += 32) {

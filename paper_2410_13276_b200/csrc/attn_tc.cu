@@ -618,7 +618,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tr.ev(11, g);
           if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
           tr.ev(12, g);
-          fence_async_smem();     // K was written through the generic proxy (cp.async); the MMA reads through the async proxy
           tc_fence_after();
           const uint64_t kd = kd0 + (uint64_t)(slot * (kKVBytes >> 4));
           const uint32_t d = tmem + col_s(grp, buf);

@@ -297,6 +297,26 @@ def main():
         p.gate()                                             # restore the scores of the bench mask
         del wq_v, wk_v
 
+    # gate and mask in one call with the scores held one band at a time (no quadratic buffer), outside the timed
+    # region; the lists must equal those of the two separate calls bit for bit
+    fused = None
+    if rank == 0:
+        band_mb = 128
+        rp_ref, col_ref = p.row_ptr.clone(), p.col_idx[:nnz].clone()
+        for _ in range(3):
+            p.gate_mask(params, band_bytes=band_mb << 20)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(5):
+            p.gate_mask(params, band_bytes=band_mb << 20)
+        b.record(stream); torch.cuda.synchronize()
+        fused = {"band_mb": band_mb, "ms": a.elapsed_time(b) / 5, "separate_ms": gate_ms + mask_ms,
+                 "scratch_bytes": int(p.ws_fused.numel()), "separate_bytes": int(p.ws.numel() + p.scores.numel() * 4),
+                 "lists_equal": bool(torch.equal(p.row_ptr, rp_ref) and torch.equal(p.col_idx[:nnz], col_ref))}
+        p.ws_fused = None
+        del rp_ref, col_ref
+
     # the max-pooled attention map on the kept blocks (Eq. 2; a side output for distillation / diagnostics), outside the
     # timed region: one attention launch that also writes lse, then the block-max pass
     block_max_ms = None
@@ -357,7 +377,7 @@ def main():
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
                             "kernel": "seer_sparse_attn"},
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
-               "gate_variant": gate_var, "block_max_ms": block_max_ms,
+               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:
             dense_blocks = B.seer_causal_blocks(p.shape)

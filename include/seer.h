@@ -214,6 +214,30 @@ seer_status seer_gate_scores_ex(seer_ctx* ctx, const seer_shape* shape, const se
                                 const void* k, const float* Wq, const float* Wk, float* scores, void* ws, size_t ws_bytes,
                                 void* stream);
 
+/* Gate and block mask in one call, without the quadratic score matrix (calls 1 and 2 fused at the level of the stream;
+ * Sec. 3.1 and 3.3, Eq. 1, 3, 4).
+ *
+ * seer_gate_scores + seer_block_mask need scores[num_q_heads * sum nb^2] in device memory: 537 MB at 131072 tokens and
+ * 32 heads, 34 GB at a million tokens.  This call projects the pooled Q and K once and then walks the rows of the CSR
+ * structure in bands: the scores of a band (whole sequences, else whole heads of a sequence, else runs of 64-row tiles
+ * of one head) are written to a scratch buffer, the band's rows are counted, row_ptr is continued from the previous
+ * band, and the band's lists are written, before the next band overwrites the scratch.  A band of up to ~100 MB stays in
+ * the L2 cache, so the scores never reach DRAM.
+ *
+ * Results (row_ptr, col_idx, *nnz_out) are identical, bit for bit, to seer_gate_scores (options == NULL) or
+ * seer_gate_scores_ex (options != NULL) followed by seer_block_mask with the same params: the same kernels compute
+ * the same scores in the same order.  Arguments, layouts, ownership and errors are those of these calls.
+ *
+ * Workspace: DEVICE memory, 256-byte aligned, seer_gate_mask_workspace_bytes(shape, band_bytes) bytes: the projected
+ * vectors (seer_workspace_bytes) followed by the band scratch.  The call uses whatever follows the projected vectors
+ * as scratch, so `band_bytes` is the caller's choice; at least 64 rows of the longest sequence (64 * max nb * 4 + 16
+ * bytes) are needed and the size query never returns less.  SEER_ERR_WORKSPACE if ws is smaller than that. */
+size_t seer_gate_mask_workspace_bytes(const seer_shape* shape, size_t band_bytes);
+seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const seer_gate_options* options, const void* q,
+                                 const void* k, const float* Wq, const float* Wk, const seer_mask_params* params,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, void* ws,
+                                 size_t ws_bytes, void* stream);
+
 /* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, the tcgen05 attention kernel runs in an
  * instrumented instantiation.  CTA 0 adds up the SM clocks its pipeline roles spend between marked points, on every
  * 8th tile (role r at uint64 offset r * 8192: 48 tags x (clock sum, count)); every CTA writes its wall time in ns at

@@ -27,7 +27,7 @@ EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
            "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
            "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static", "seer_gate_scores_ex",
-           "seer_attn_block_max"]
+           "seer_attn_block_max", "seer_gate_mask_workspace_bytes", "seer_gate_block_mask"]
 
 
 class SeerError(RuntimeError):
@@ -102,6 +102,11 @@ def load_library() -> C.CDLL:
     lib.seer_gate_scores_ex.restype = C.c_int
     lib.seer_attn_block_max.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp]
     lib.seer_attn_block_max.restype = C.c_int
+    lib.seer_gate_mask_workspace_bytes.argtypes = [shp, sz]
+    lib.seer_gate_mask_workspace_bytes.restype = sz
+    lib.seer_gate_block_mask.argtypes = [vp, shp, C.POINTER(seer_gate_options), vp, vp, vp, vp, C.POINTER(seer_mask_params),
+                                         vp, vp, i64, vp, vp, sz, vp]
+    lib.seer_gate_block_mask.restype = C.c_int
     lib.seer_set_trace_buffer.argtypes = [vp, vp]
     lib.seer_set_trace_buffer.restype = C.c_int
     _lib = lib
@@ -202,6 +207,22 @@ def seer_gate_scores_ex(ctx: Context, shape: seer_shape, options: seer_gate_opti
     _check(ctx._lib.seer_gate_scores_ex(ctx.handle, C.byref(shape), C.byref(options), _ptr(q), _ptr(k), _ptr(wq),
                                         _ptr(wk), _ptr(scores), _ptr(ws), ws_bytes, _stream(stream)),
            "seer_gate_scores_ex")
+
+
+def seer_gate_mask_workspace_bytes(shape: seer_shape, band_bytes: int) -> int:
+    return int(load_library().seer_gate_mask_workspace_bytes(C.byref(shape), band_bytes))
+
+
+def seer_gate_block_mask(ctx: Context, shape: seer_shape, options: Optional[seer_gate_options], q, k, wq, wk,
+                         params: seer_mask_params, row_ptr, col_idx, col_capacity: Optional[int], nnz_out, ws,
+                         stream=None) -> None:
+    if col_capacity is None:
+        col_capacity = 0 if col_idx is None else col_idx.numel()
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    opt = None if options is None else C.byref(options)
+    _check(ctx._lib.seer_gate_block_mask(ctx.handle, C.byref(shape), opt, _ptr(q), _ptr(k), _ptr(wq), _ptr(wk),
+                                         C.byref(params), _ptr(row_ptr), _ptr(col_idx), col_capacity, _ptr(nnz_out),
+                                         _ptr(ws), ws_bytes, _stream(stream)), "seer_gate_block_mask")
 
 
 def seer_attn_block_max(ctx: Context, shape: seer_shape, q, k, row_ptr, col_idx, lse, block_max, stream=None) -> None:

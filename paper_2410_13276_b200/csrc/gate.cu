@@ -302,9 +302,12 @@ __device__ __forceinline__ void gs_load_planes(uint32_t dst, const uint16_t* __r
   }
 }
 
-// grid.x = total_tiles * Hq (head fastest; tiles are visited from the last rows, the longest, to the first)
+// grid.x = band.tiles * band.heads (head fastest; tiles are visited from the last rows, the longest, to the first).  The
+// band is a rectangle of (64-row score tile, query head) pairs; the whole problem is the band (0, total_tiles, 0, Hq, 0).
+// Scores of the band are written at their offset in the full matrix minus band.score_base.
 __global__ void __launch_bounds__(kScoreThreads)
-gate_scores_kernel(SeqMeta m, const uint16_t* __restrict__ gq, const uint16_t* __restrict__ gk, float* __restrict__ scores) {
+gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, const uint16_t* __restrict__ gk,
+                   float* __restrict__ scores) {
   extern __shared__ __align__(128) unsigned char gs_smem[];
   const uint32_t sA = gs_smem_u32(gs_smem), sB0 = sA + 3 * kPlaneTile;
   float* row_m = reinterpret_cast<float*>(gs_smem + 9 * kPlaneTile);     // [64]
@@ -312,8 +315,8 @@ gate_scores_kernel(SeqMeta m, const uint16_t* __restrict__ gq, const uint16_t* _
   float* part_m = row_l + kScoreTile;                                     // [2 column halves][64]
   float* part_l = part_m + 2 * kScoreTile;
 
-  const int tile_g = m.total_tiles - 1 - (int)(blockIdx.x / m.num_q_heads);
-  const int h = blockIdx.x % m.num_q_heads;
+  const int tile_g = band.tile_lo + band.tiles - 1 - (int)(blockIdx.x / band.heads);
+  const int h = band.head_lo + (int)(blockIdx.x % band.heads);
   const int g = h / m.group;
   const int b = find_sequence(m.tile_off, m.batch, tile_g);
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
@@ -323,13 +326,14 @@ gate_scores_kernel(SeqMeta m, const uint16_t* __restrict__ gq, const uint16_t* _
   const size_t plane_k = (size_t)m.num_kv_heads * m.total_blocks * kGateDim;
   const uint16_t* gq_h = gq + ((size_t)h * m.total_blocks + m.blk_off[b]) * kGateDim;
   const uint16_t* gk_g = gk + ((size_t)g * m.total_blocks + m.blk_off[b]) * kGateDim;
-  float* sc = scores + m.score_off[b] + (size_t)h * nb * nb;
+  const int64_t sc_off = m.score_off[b] + (int64_t)h * nb * nb - band.score_base;
+  float* sc = scores + sc_off;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wr = warp & 3, wc = warp >> 2;                               // row group, column half
   const int gid = lane >> 2, tig = lane & 3;
   const float scale = rsqrtf((float)kGateDim);
-  const bool vec_ok = (nb & 1) == 0 && (m.score_off[b] & 1) == 0;        // 8-byte stores of column pairs
+  const bool vec_ok = (nb & 1) == 0 && (sc_off & 1) == 0;                // 8-byte stores of column pairs
 
   const int last_col = i0 + rows_valid - 1;
   gs_load_planes(sA, gq_h, plane_q, i0, rows_valid);
@@ -447,7 +451,7 @@ gate_scores_kernel(SeqMeta m, const uint16_t* __restrict__ gq, const uint16_t* _
   __syncthreads();
   // normalise in place: the logits this CTA just wrote are re-read (L2) and replaced by exp(x - m) / l; a warp per row,
   // four columns per lane and step, so that many independent loads are in flight
-  const bool vec4 = (nb & 3) == 0 && (m.score_off[b] & 3) == 0;
+  const bool vec4 = (nb & 3) == 0 && (sc_off & 3) == 0;
   for (int r = warp; r < rows_valid; r += kScoreThreads / 32) {
     const int i = i0 + r;
     const float mm = row_m[r];
@@ -476,8 +480,13 @@ int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, c
   uint16_t* gk = (uint16_t*)((char*)ws + gq_bytes);
   const unsigned grid1 = (unsigned)m.total_chunks * (unsigned)(m.num_q_heads + m.num_kv_heads);
   pool_project_kernel<<<grid1, kPoolThreads, 0, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, Wq, Wk, gq, gk);
+  if (scores == nullptr) {                             // projection only: the scores follow band by band
+    cudaError_t e0 = cudaGetLastError();
+    return e0 == cudaSuccess ? 1 : -(int)e0;
+  }
+  const ScoreBand all = {0, m.total_tiles, 0, m.num_q_heads, 0};
   const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
-  gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, gq, gk, scores);
+  gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, all, gq, gk, scores);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 2 : -(int)e;
 }
@@ -492,10 +501,27 @@ int launch_gate_ex(seer_ctx* ctx, const SeqMeta& m, const seer_gate_options& opt
   const unsigned grid1 = (unsigned)m.total_chunks * (unsigned)(m.num_q_heads + m.num_kv_heads);
   pool_project_ex_kernel<<<grid1, kPoolThreads, 0, stream>>>(m, (const uint16_t*)q, (const uint16_t*)k, Wq, Wk, gq, gk,
                                                               opt.pool_q, opt.pool_k, opt.rope_theta);
+  if (scores == nullptr) {                             // projection only: the scores follow band by band
+    cudaError_t e0 = cudaGetLastError();
+    return e0 == cudaSuccess ? 1 : -(int)e0;
+  }
+  const ScoreBand all = {0, m.total_tiles, 0, m.num_q_heads, 0};
   const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
-  gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, gq, gk, scores);
+  gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, all, gq, gk, scores);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 2 : -(int)e;
+}
+
+// Scores of one band from the projected vectors launch_gate_ex(scores = nullptr) left in `ws`.
+int launch_gate_scores_band(const SeqMeta& m, const ScoreBand& band, const void* ws, float* scores, cudaStream_t stream) {
+  size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * 6 + 255) / 256 * 256;
+  const uint16_t* gq = (const uint16_t*)ws;
+  const uint16_t* gk = (const uint16_t*)((const char*)ws + gq_bytes);
+  const unsigned grid = (unsigned)band.tiles * (unsigned)band.heads;
+  if (grid == 0) return 0;
+  gate_scores_kernel<<<grid, kScoreThreads, kScoreSmem, stream>>>(m, band, gq, gk, scores);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 1 : -(int)e;
 }
 
 // ----------------------------------------------------------------------------------------------- allocation-free variant

@@ -19,16 +19,21 @@ struct RowInfo {
   bool valid;
 };
 
-__device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const float* __restrict__ scores, int64_t r) {
+// Rows [row_lo, row_hi) of the CSR structure whose scores sit at (offset in the full matrix - score_base) in `scores`.
+struct RowBand {
+  int64_t row_lo, row_hi, score_base;
+};
+
+__device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const RowBand& band, const float* __restrict__ scores, int64_t r) {
   RowInfo ri;
-  ri.valid = r < m.rows;
+  ri.valid = r < band.row_hi;
   if (!ri.valid) { ri.s = nullptr; ri.i = 0; return ri; }
   const int b = find_sequence(m.blk_off, m.batch, (int)(r / m.num_q_heads));
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
   const int64_t local = r - (int64_t)m.num_q_heads * m.blk_off[b];
   const int h = (int)(local / nb);
   ri.i = (int)(local - (int64_t)h * nb);
-  ri.s = scores + m.score_off[b] + ((size_t)h * nb + ri.i) * nb;
+  ri.s = scores + (m.score_off[b] + ((int64_t)h * nb + ri.i) * nb - band.score_base);
   return ri;
 }
 
@@ -68,10 +73,10 @@ __device__ __forceinline__ int warp_sum(int v) {
 }
 
 __global__ void __launch_bounds__(kMaskWarps * 32)
-count_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, int32_t* __restrict__ row_ptr) {
+count_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask_params p, int32_t* __restrict__ row_ptr) {
   const int lane = threadIdx.x & 31;
-  const int64_t r = (int64_t)blockIdx.x * kMaskWarps + (threadIdx.x >> 5);
-  const RowInfo ri = decode_row(m, scores, r);
+  const int64_t r = band.row_lo + (int64_t)blockIdx.x * kMaskWarps + (threadIdx.x >> 5);
+  const RowInfo ri = decode_row(m, band, scores, r);
   if (!ri.valid) return;
   const int n = ri.i + 1;
   int c = 0;
@@ -88,16 +93,17 @@ count_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, in
   if (lane == 0) row_ptr[r + 1] = c;
 }
 
-// Single CTA: in-place inclusive scan of row_ptr[1..rows]; row_ptr[0] = 0.  Tiles of 4096 counts go through shared
-// memory (coalesced loads and stores), four consecutive counts per thread, warp shuffles inside a warp, one carry per tile.
+// Single CTA: in-place inclusive scan of row_ptr[1..rows].  `first`: row_ptr[0] = 0; otherwise the scan continues from
+// row_ptr[0], the last entry of the rows scanned before.  Tiles of 4096 counts go through shared memory (coalesced loads
+// and stores), four consecutive counts per thread, warp shuffles inside a warp, one carry per tile.
 __global__ void __launch_bounds__(1024)
-scan_kernel(int64_t rows, int32_t* __restrict__ row_ptr, int64_t col_capacity, int64_t* __restrict__ nnz_out,
+scan_kernel(int64_t rows, int32_t* __restrict__ row_ptr, int first, int64_t col_capacity, int64_t* __restrict__ nnz_out,
             int* __restrict__ status) {
   __shared__ int32_t tile[4096];
   __shared__ long long warp_tot[32];
   __shared__ long long carry_s;
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-  long long carry = 0;
+  long long carry = first ? 0 : row_ptr[0];
   for (int64_t base = 0; base < rows; base += 4096) {
     const int n = (int)min((int64_t)4096, rows - base);
 #pragma unroll
@@ -143,20 +149,20 @@ scan_kernel(int64_t rows, int32_t* __restrict__ row_ptr, int64_t col_capacity, i
     __syncthreads();
   }
   if (t == 0) {
-    row_ptr[0] = 0;
+    if (first) row_ptr[0] = 0;
     if (nnz_out) *nnz_out = carry;
     if (carry > col_capacity) atomicCAS(status, 0, (int)SEER_ERR_CAPACITY);
   }
 }
 
 __global__ void __launch_bounds__(kMaskWarps * 32)
-fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, const int32_t* __restrict__ row_ptr,
+fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask_params p, const int32_t* __restrict__ row_ptr,
             int32_t* __restrict__ col_idx, int64_t col_capacity, int stage_cap) {
   extern __shared__ uint32_t key_smem[];
   uint32_t* hist_smem = key_smem + (size_t)kMaskWarps * stage_cap;   // 256 bins per warp
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t r = (int64_t)blockIdx.x * kMaskWarps + warp;
-  const RowInfo ri = decode_row(m, scores, r);
+  const int64_t r = band.row_lo + (int64_t)blockIdx.x * kMaskWarps + warp;
+  const RowInfo ri = decode_row(m, band, scores, r);
   if (!ri.valid) return;
   const int n = ri.i + 1;
   const int32_t out0 = row_ptr[r], out1 = row_ptr[r + 1];
@@ -280,6 +286,21 @@ fill_kernel(SeqMeta m, const float* __restrict__ scores, seer_mask_params p, con
   }
 }
 
+int launch_mask_band(seer_ctx* ctx, const SeqMeta& m, const float* scores, int64_t score_base, int64_t row_lo,
+                     int64_t row_hi, bool first, const seer_mask_params& p, int32_t* row_ptr, int32_t* col_idx,
+                     int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream) {
+  if (row_hi <= row_lo) return 0;
+  const RowBand band = {row_lo, row_hi, score_base};
+  const unsigned grid = (unsigned)((row_hi - row_lo + kMaskWarps - 1) / kMaskWarps);
+  count_kernel<<<grid, kMaskWarps * 32, 0, stream>>>(m, band, scores, p, row_ptr);
+  scan_kernel<<<1, 1024, 0, stream>>>(row_hi - row_lo, row_ptr + row_lo, first ? 1 : 0, col_capacity, nnz_out, ctx->d_status);
+  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // longer rows re-read their scores instead
+  const size_t smem = (size_t)kMaskWarps * (stage_cap + 256) * sizeof(uint32_t);
+  fill_kernel<<<grid, kMaskWarps * 32, smem, stream>>>(m, band, scores, p, row_ptr, col_idx, col_capacity, stage_cap);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 3 : -(int)e;
+}
+
 int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer_mask_params& p, int32_t* row_ptr,
                 int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream) {
   if (m.rows == 0) {
@@ -287,14 +308,7 @@ int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer
     if (nnz_out) cudaMemsetAsync(nnz_out, 0, sizeof(int64_t), stream);
     return 0;
   }
-  const unsigned grid = (unsigned)((m.rows + kMaskWarps - 1) / kMaskWarps);
-  count_kernel<<<grid, kMaskWarps * 32, 0, stream>>>(m, scores, p, row_ptr);
-  scan_kernel<<<1, 1024, 0, stream>>>(m.rows, row_ptr, col_capacity, nnz_out, ctx->d_status);
-  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // longer rows re-read their scores instead
-  const size_t smem = (size_t)kMaskWarps * (stage_cap + 256) * sizeof(uint32_t);
-  fill_kernel<<<grid, kMaskWarps * 32, smem, stream>>>(m, scores, p, row_ptr, col_idx, col_capacity, stage_cap);
-  cudaError_t e = cudaGetLastError();
-  return e == cudaSuccess ? 3 : -(int)e;
+  return launch_mask_band(ctx, m, scores, 0, 0, m.rows, true, p, row_ptr, col_idx, col_capacity, nnz_out, stream);
 }
 
 seer_status init_mask(seer_ctx* ctx) {

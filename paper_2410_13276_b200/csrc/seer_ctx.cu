@@ -344,6 +344,122 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
   return SEER_OK;
 }
 
+// ---- gate and mask in one call, the scores held one band at a time
+namespace {
+constexpr size_t kBandSlackElems = 4;   // the band's base is rounded down to a multiple of four elements
+
+size_t min_band_bytes(const ShapeTotals& t) { return ((size_t)kScoreTile * (size_t)t.max_nb + kBandSlackElems) * sizeof(float); }
+}  // namespace
+
+size_t seer_gate_mask_workspace_bytes(const seer_shape* shape, size_t band_bytes) {
+  ShapeTotals t;
+  if (shape_totals(shape, &t) != SEER_OK) return 0;
+  const size_t need = min_band_bytes(t);
+  return gate_workspace_bytes(t, shape) + align_up(band_bytes > need ? band_bytes : need, 256);
+}
+
+seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const seer_gate_options* opt, const void* q,
+                                 const void* k, const float* Wq, const float* Wk, const seer_mask_params* p,
+                                 int32_t* row_ptr, int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, void* ws,
+                                 size_t ws_bytes, void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!ctx || !shape || !p) return SEER_ERR_INVALID_ARG;
+  if (opt) {
+    const uint32_t all = SEER_POOL_AVG | SEER_POOL_MAX | SEER_POOL_MIN;
+    if (opt->pool_q == 0 || opt->pool_k == 0 || (opt->pool_q & ~all) || (opt->pool_k & ~all)) return SEER_ERR_INVALID_ARG;
+    if (!(opt->rope_theta >= 0.f) || opt->rope_theta > 3.0e38f) return SEER_ERR_INVALID_ARG;
+  }
+  ShapeTotals t;
+  seer_status st = shape_totals(shape, &t);
+  if (st != SEER_OK) return st;
+  if (!row_ptr || col_capacity < 0 || (col_capacity > 0 && !col_idx)) return SEER_ERR_INVALID_ARG;
+  if (p->mode != SEER_TOPK_RATIO && p->mode != SEER_TOPK_COUNT && p->mode != SEER_THRESHOLD) return SEER_ERR_INVALID_ARG;
+  if (p->mode == SEER_TOPK_RATIO && (p->keep_num < 0 || p->keep_den < 1)) return SEER_ERR_INVALID_ARG;
+  if (p->flags & ~(uint32_t)(SEER_FORCE_DIAG | SEER_FORCE_SINK)) return SEER_ERR_INVALID_ARG;
+  if (t.total_blocks > 0 && (!q || !k || !Wq || !Wk)) return SEER_ERR_INVALID_ARG;
+  const size_t gate_bytes = gate_workspace_bytes(t, shape);
+  if (t.total_blocks > 0 && !ws_ok(ws, ws_bytes, gate_bytes + min_band_bytes(t))) return SEER_ERR_WORKSPACE;
+  SeqMeta m; int slot;
+  st = prepare(ctx, shape, stream, &m, &slot);
+  if (st != SEER_OK) return st;
+  if (t.total_blocks == 0) {
+    int n0 = launch_mask(ctx, m, nullptr, *p, row_ptr, col_idx, col_capacity, nnz_out, stream);
+    finish_call(ctx, slot, stream);
+    return n0 < 0 ? SEER_ERR_CUDA : SEER_OK;
+  }
+  float* band_buf = (float*)((char*)ws + gate_bytes);
+  const int64_t cap = (int64_t)((ws_bytes - gate_bytes) / sizeof(float)) - (int64_t)kBandSlackElems;   // elements per band
+  int64_t launched = 0;
+  bool bad = false, first = true;
+  {
+    int n = opt ? launch_gate_ex(ctx, m, *opt, q, k, Wq, Wk, nullptr, ws, stream)
+                : launch_gate(ctx, m, q, k, Wq, Wk, nullptr, ws, stream);
+    if (n < 0) bad = true; else launched += n;
+  }
+  // One band after the other, in CSR row order: scores of the band -> counts -> row_ptr (continued) -> lists.
+  auto run_band = [&](int tile_lo, int tiles, int head_lo, int heads, int64_t base, int64_t row_lo, int64_t row_hi) {
+    if (bad || row_hi <= row_lo) return;
+    const ScoreBand band = {tile_lo, tiles, head_lo, heads, base & ~(int64_t)3};
+    int n = launch_gate_scores_band(m, band, ws, band_buf, stream);
+    if (n >= 0) {
+      launched += n;
+      n = launch_mask_band(ctx, m, band_buf, band.score_base, row_lo, row_hi, first, *p, row_ptr, col_idx, col_capacity,
+                           nnz_out, stream);
+    }
+    if (n < 0) { bad = true; return; }
+    launched += n;
+    first = false;
+  };
+  const int32_t* cu = shape->cu_seqlens_host;
+  const int Hq = shape->num_q_heads;
+  auto blocks_of = [&](int b) { return ((int64_t)cu[b + 1] - cu[b] + kBlock - 1) / kBlock; };
+  int64_t blk_off = 0, tile_off = 0, score_off = 0;    // of sequence b
+  for (int b = 0; b < shape->batch && !bad;) {
+    const int64_t nb = blocks_of(b);
+    if ((int64_t)Hq * nb * nb <= cap) {
+      // whole sequences, as many as fit
+      int b1 = b;
+      int64_t blocks = 0, tiles = 0, elems = 0;
+      while (b1 < shape->batch) {
+        const int64_t n1 = blocks_of(b1);
+        if (elems + (int64_t)Hq * n1 * n1 > cap) break;
+        elems += (int64_t)Hq * n1 * n1; blocks += n1; tiles += (n1 + kScoreTile - 1) / kScoreTile;
+        ++b1;
+      }
+      run_band((int)tile_off, (int)tiles, 0, Hq, score_off, Hq * blk_off, Hq * (blk_off + blocks));
+      blk_off += blocks; tile_off += tiles; score_off += elems;
+      b = b1;
+      continue;
+    }
+    const int64_t ntile = (nb + kScoreTile - 1) / kScoreTile;
+    if (nb * nb <= cap) {
+      // whole heads of this sequence
+      const int hb = (int)(cap / (nb * nb));
+      for (int h0 = 0; h0 < Hq; h0 += hb) {
+        const int h1 = h0 + hb < Hq ? h0 + hb : Hq;
+        run_band((int)tile_off, (int)ntile, h0, h1 - h0, score_off + (int64_t)h0 * nb * nb, Hq * blk_off + (int64_t)h0 * nb,
+                 Hq * blk_off + (int64_t)h1 * nb);
+      }
+    } else {
+      // runs of 64-row tiles of one head
+      const int64_t tb = cap / ((int64_t)kScoreTile * nb);   // >= 1: the workspace check above
+      for (int h = 0; h < Hq; ++h)
+        for (int64_t t0 = 0; t0 < ntile; t0 += tb) {
+          const int64_t t1 = t0 + tb < ntile ? t0 + tb : ntile;
+          const int64_t i0 = t0 * kScoreTile, i1 = t1 * kScoreTile < nb ? t1 * kScoreTile : nb;
+          run_band((int)(tile_off + t0), (int)(t1 - t0), h, 1, score_off + ((int64_t)h * nb + i0) * nb,
+                   Hq * blk_off + (int64_t)h * nb + i0, Hq * blk_off + (int64_t)h * nb + i1);
+        }
+    }
+    blk_off += nb; tile_off += ntile; score_off += (int64_t)Hq * nb * nb;
+    ++b;
+  }
+  finish_call(ctx, slot, stream);
+  if (bad) return SEER_ERR_CUDA;
+  ctx->launches += launched;
+  return SEER_OK;
+}
+
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl) {
   if (!ctx || (impl != 0 && impl != 1)) return SEER_ERR_INVALID_ARG;
   ctx->attn_impl = impl;

@@ -39,6 +39,15 @@ struct SeqMeta {
   float softmax_scale;
 };
 
+// A rectangle of (64-row score tile, query head) pairs whose scores are produced and consumed together; tiles are
+// numbered over the whole batch (tile_off).  score_base is the offset, in the full score matrix, of the band's first
+// element: the band's scores live at (full offset - score_base) in whatever buffer the kernels are given.
+struct ScoreBand {
+  int32_t tile_lo, tiles;
+  int32_t head_lo, heads;
+  int64_t score_base;
+};
+
 struct MetaSlot {
   std::vector<int32_t> key;    // cu_seqlens + Hq: what the slot currently describes
   void* dev = nullptr;
@@ -87,6 +96,12 @@ int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, c
                 float* scores, void* ws, cudaStream_t stream);
 int launch_gate_ex(seer_ctx* ctx, const SeqMeta& m, const seer_gate_options& opt, const void* q, const void* k,
                    const float* Wq, const float* Wk, float* scores, void* ws, cudaStream_t stream);
+int launch_gate_scores_band(const SeqMeta& m, const ScoreBand& band, const void* ws, float* scores, cudaStream_t stream);
+// Mask rows [row_lo, row_hi) from a band of scores; `first` starts row_ptr at 0, later bands continue from the
+// previous band's last entry.
+int launch_mask_band(seer_ctx* ctx, const SeqMeta& m, const float* scores, int64_t score_base, int64_t row_lo,
+                     int64_t row_hi, bool first, const seer_mask_params& p, int32_t* row_ptr, int32_t* col_idx,
+                     int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream);
 int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer_mask_params& p, int32_t* row_ptr,
                 int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream);
 int launch_attn_mma(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,

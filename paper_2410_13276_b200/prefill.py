@@ -74,6 +74,17 @@ class Prefill:
         [heads, n * 128, 128] matching the pooling subsets in `options`."""
         B.seer_gate_scores_ex(self.ctx, self.shape, options, self.q, self.k, wq, wk, self.scores, self.ws, stream)
 
+    def gate_mask(self, params: B.seer_mask_params, *, band_bytes: int = 128 << 20, options=None, wq=None, wk=None,
+                  stream=None):
+        """Gate and mask in one call, the scores held one band at a time in a scratch of `band_bytes` (never the whole
+        score matrix); fills row_ptr / col_idx / nnz exactly as gate() + mask() do."""
+        need = B.seer_gate_mask_workspace_bytes(self.shape, band_bytes)
+        if getattr(self, "ws_fused", None) is None or self.ws_fused.numel() != need:
+            self.ws_fused = torch.empty(max(need, 256), dtype=torch.uint8, device=self.device)
+        B.seer_gate_block_mask(self.ctx, self.shape, options, self.q, self.k, self.wq if wq is None else wq,
+                               self.wk if wk is None else wk, params, self.row_ptr, self.col_idx, self.col_capacity,
+                               self.nnz, self.ws_fused, stream)
+
     def block_max(self, stream=None):
         """Max-pooled attention map on the listed blocks (Eq. 2) from the lse of the last `attn` call; returns the
         device tensor [col_capacity] fp32 aligned with col_idx."""

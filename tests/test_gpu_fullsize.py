@@ -66,6 +66,13 @@ def check_workload(rt, name, specs, sample_heads, rows_per_head=3):
         p.attn()
         assert p.status() == 0
         rp, col = p.lists_host()
+        # the banded gate + mask call (no score matrix) gives the same lists, bit for bit
+        p.row_ptr.fill_(-1)
+        p.gate_mask(params)
+        assert p.status() == 0
+        rp_f, col_f = p.lists_host()
+        assert np.array_equal(rp_f, rp) and np.array_equal(col_f, col), name
+        p.ws_fused = None
         # (d) properties at any size
         counts = np.diff(rp)
         assert rp[0] == 0 and rp[-1] == len(col) == int(p.nnz.item())

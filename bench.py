@@ -317,6 +317,29 @@ def main():
         p.ws_fused = None
         del rp_ref, col_ref
 
+    # the same layer with 128-token gate blocks (gate and mask at B = 128, lists expanded for the 64-token attention
+    # tiles), outside the timed region
+    block128 = None
+    if rank == 0:
+        p.scores = None                                      # one score matrix at a time
+        p2 = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, device=local, ctx=p.ctx, want_lse=False, block=128)
+        p2.q, p2.k, p2.v, p2.wq, p2.wk, p2.o = p.q, p.k, p.v, p.wq, p.wk, p.o
+        for _ in range(2):
+            p2.gate(); p2.mask(params); p2.attn()
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        e[0].record(stream); p2.gate(); e[1].record(stream)
+        B.seer_block_mask(p2.ctx, p2.shape, p2.scores, params, p2.row_ptr, p2.col_idx, p2.col_capacity, p2.nnz, None)
+        e[2].record(stream); p2.expand(); e[3].record(stream); p2.attn(); e[4].record(stream)
+        torch.cuda.synchronize()
+        n64 = int(p2.nnz64.item())
+        t = [e[i].elapsed_time(e[i + 1]) for i in range(4)]
+        block128 = {"gate_ms": t[0], "mask_ms": t[1], "expand_ms": t[2], "attn_ms": t[3], "kept_blocks_128": int(p2.nnz.item()),
+                    "kept_blocks_64": n64, "attn_tflops": n64 * FLOP_PER_BLOCK / (t[3] * 1e-3) / 1e12}
+        del p2
+        p.scores = torch.empty(max(B.seer_scores_elems(p.shape), 1), dtype=torch.float32, device="cuda")
+        p.gate(); p.mask(params)                             # back to the bench lists
+
     # the max-pooled attention map on the kept blocks (Eq. 2; a side output for distillation / diagnostics), outside the
     # timed region: one attention launch that also writes lse, then the block-max pass
     block_max_ms = None
@@ -377,7 +400,7 @@ def main():
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
                             "kernel": "seer_sparse_attn"},
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
-               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused,
+               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:
             dense_blocks = B.seer_causal_blocks(p.shape)

@@ -31,7 +31,8 @@
  *    row_ptr      int32 [rows + 1], col_idx int32 [nnz]: CSR lists of KV block indices, local to the sequence,
  *                 ascending, unique, 0 <= j <= i
  *
- * Supported: head_dim = 128, gate_dim = 128, block = 64, num_q_heads a multiple of num_kv_heads, batch <= 4096.
+ * Supported: head_dim = 128, gate_dim = 128, block = 64 (every call) or 128 (gate and mask calls; the attention takes
+ * their lists through seer_expand_block_lists), num_q_heads a multiple of num_kv_heads, batch <= 4096.
  * Anything else returns SEER_ERR_UNSUPPORTED.
  */
 #ifndef SEER_H_
@@ -70,7 +71,8 @@ typedef struct {
   int32_t num_q_heads;
   int32_t num_kv_heads;
   int32_t head_dim;               /* 128 */
-  int32_t block;                  /* 64: gate pooling window = attention tile (Sec. 4: B fixed at 64) */
+  int32_t block;                  /* 64: gate pooling window = attention tile (Sec. 4: B fixed at 64); or 128, see
+                                     seer_expand_block_lists */
   int32_t gate_dim;               /* 128: output width of the gate's linear layers */
   float softmax_scale;            /* attention logit scale; <= 0 selects 1/sqrt(head_dim) (Sec. 2) */
 } seer_shape;
@@ -237,6 +239,25 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
                                  const void* k, const float* Wq, const float* Wk, const seer_mask_params* params,
                                  int32_t* row_ptr, int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, void* ws,
                                  size_t ws_bytes, void* stream);
+
+/* 128-token gate blocks (Sec. 4 evaluates 64; the kernel section mentions 128-sized tiles).
+ *
+ * shape->block may be 64 or 128.  With 128, seer_gate_scores / _ex / _static, seer_block_mask and seer_gate_block_mask
+ * work on 128-token blocks throughout: nb = ceil(S / 128) per sequence, scores [num_q_heads, nb, nb], CSR rows and block
+ * indices in units of 128 tokens, block-level RoPE with base theta / 128.  The attention kernels tile by 64 tokens, so
+ * seer_sparse_attn, seer_attn_block_max and seer_prefill_host return SEER_ERR_UNSUPPORTED for block = 128; instead
+ * seer_expand_block_lists rewrites the 128-token lists as 64-token lists that select exactly the same (query, key)
+ * pairs, and seer_sparse_attn runs on those with the same shape at block = 64:
+ *   block j -> (2j, 2j + 1); query rows 2i and 2i + 1 inherit the list of row i; in the diagonal block, row 2i takes 2i
+ *   only (2i + 1 lies in its future), row 2i + 1 takes both.
+ * `shape` is the 128-token shape; row_ptr / col_idx the lists seer_block_mask produced for it (DEVICE, read only);
+ * row_ptr64 [num_q_heads * sum ceil(S / 64) + 1] and col_idx64 [col_capacity64] are written (DEVICE, caller-owned;
+ * four times the entries of col_idx always suffice); *nnz_out (DEVICE int64, may be NULL) receives the entry count.
+ * SEER_ERR_CAPACITY through the device status if col_capacity64 is too small (row_ptr64 and *nnz_out are still
+ * complete).  An entry j > i is passed on as (2j, 2j + 1) and reported by the attention call. */
+seer_status seer_expand_block_lists(seer_ctx* ctx, const seer_shape* shape, const int32_t* row_ptr, const int32_t* col_idx,
+                                    int32_t* row_ptr64, int32_t* col_idx64, int64_t col_capacity64, int64_t* nnz_out,
+                                    void* stream);
 
 /* Diagnostics (the paper has no counterpart): when `device_buffer` is not NULL, the tcgen05 attention kernel runs in an
  * instrumented instantiation.  CTA 0 adds up the SM clocks its pipeline roles spend between marked points, on every

@@ -27,7 +27,8 @@ EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
            "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
            "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static", "seer_gate_scores_ex",
-           "seer_attn_block_max", "seer_gate_mask_workspace_bytes", "seer_gate_block_mask"]
+           "seer_attn_block_max", "seer_gate_mask_workspace_bytes", "seer_gate_block_mask",
+           "seer_expand_block_lists"]
 
 
 class SeerError(RuntimeError):
@@ -107,6 +108,8 @@ def load_library() -> C.CDLL:
     lib.seer_gate_block_mask.argtypes = [vp, shp, C.POINTER(seer_gate_options), vp, vp, vp, vp, C.POINTER(seer_mask_params),
                                          vp, vp, i64, vp, vp, sz, vp]
     lib.seer_gate_block_mask.restype = C.c_int
+    lib.seer_expand_block_lists.argtypes = [vp, shp, vp, vp, vp, vp, i64, vp, vp]
+    lib.seer_expand_block_lists.restype = C.c_int
     lib.seer_set_trace_buffer.argtypes = [vp, vp]
     lib.seer_set_trace_buffer.restype = C.c_int
     _lib = lib
@@ -223,6 +226,15 @@ def seer_gate_block_mask(ctx: Context, shape: seer_shape, options: Optional[seer
     _check(ctx._lib.seer_gate_block_mask(ctx.handle, C.byref(shape), opt, _ptr(q), _ptr(k), _ptr(wq), _ptr(wk),
                                          C.byref(params), _ptr(row_ptr), _ptr(col_idx), col_capacity, _ptr(nnz_out),
                                          _ptr(ws), ws_bytes, _stream(stream)), "seer_gate_block_mask")
+
+
+def seer_expand_block_lists(ctx: Context, shape: seer_shape, row_ptr, col_idx, row_ptr64, col_idx64,
+                            col_capacity64: Optional[int] = None, nnz_out=None, stream=None) -> None:
+    if col_capacity64 is None:
+        col_capacity64 = 0 if col_idx64 is None else col_idx64.numel()
+    _check(ctx._lib.seer_expand_block_lists(ctx.handle, C.byref(shape), _ptr(row_ptr), _ptr(col_idx), _ptr(row_ptr64),
+                                            _ptr(col_idx64), col_capacity64, _ptr(nnz_out), _stream(stream)),
+           "seer_expand_block_lists")
 
 
 def seer_attn_block_max(ctx: Context, shape: seer_shape, q, k, row_ptr, col_idx, lse, block_max, stream=None) -> None:

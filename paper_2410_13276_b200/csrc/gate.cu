@@ -77,12 +77,12 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
   const size_t row_stride = (size_t)H * kHeadDim;  // elements between consecutive tokens
 
   for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
-    const int t0 = s0 + (i0 + bi) * kBlock;
-    const int cnt = min(kBlock, s1 - t0);
+    const int t0 = s0 + (i0 + bi) * m.block;
+    const int cnt = min(m.block, s1 - t0);
     const uint16_t* base = x + (size_t)t0 * row_stride + (size_t)h * kHeadDim + cchunk * 8;
     float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-    for (int it = 0; it < kBlock / 2; it += 8) {
+    for (int it = 0; it < m.block / 2; it += 8) {
       uint4 u[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -183,14 +183,14 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
   const size_t row_stride = (size_t)H * kHeadDim;
 
   for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
-    const int t0 = s0 + (i0 + bi) * kBlock;
-    const int cnt = min(kBlock, s1 - t0);
+    const int t0 = s0 + (i0 + bi) * m.block;
+    const int cnt = min(m.block, s1 - t0);
     const uint16_t* base = x + (size_t)t0 * row_stride + (size_t)h * kHeadDim + cchunk * 8;
     float a[8], hi[8], lo[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) { a[j] = 0.f; hi[j] = -CUDART_INF_F; lo[j] = CUDART_INF_F; }
 #pragma unroll 1
-    for (int it = 0; it < kBlock / 2; it += 8) {
+    for (int it = 0; it < m.block / 2; it += 8) {
       uint4 u[8];
       bool live[8];
 #pragma unroll
@@ -246,7 +246,7 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
     for (int j = 0; j < 8; ++j) pooled[grp * 8 + j][o] = acc[j];
     __syncthreads();
     const int f = o & (kGateDim / 2 - 1);
-    const double freq = pow((double)rope_theta / (double)kBlock, -2.0 * (double)f / (double)kGateDim);
+    const double freq = pow((double)rope_theta / (double)m.block, -2.0 * (double)f / (double)kGateDim);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int bi = grp * 8 + j;
@@ -579,7 +579,7 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   hm.score[0] = 0;
   for (int b = 0; b < shape->batch; ++b) {
     hm.cu[b] = shape->cu_seqlens_host[b];
-    const int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + kBlock - 1) / kBlock;
+    const int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + shape->block - 1) / shape->block;
     hm.blk[b + 1] = hm.blk[b] + nb;
     hm.chunk[b + 1] = hm.chunk[b] + (nb + kPoolChunk - 1) / kPoolChunk;
     hm.tile[b + 1] = hm.tile[b] + (nb + kScoreTile - 1) / kScoreTile;
@@ -607,6 +607,7 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   m.rows = t.rows;
   m.score_elems = t.score_elems;
   m.softmax_scale = 0.f;   // unused by the gate
+  m.block = shape->block;
   // The two kernels below are the ones seer_gate_scores launches; only the scratch pointer differs.  Nothing in the
   // scratch has to start at zero: the first kernel writes every projected vector the second one reads.
   const int n = launch_gate(nullptr, m, q, k, Wq, Wk, scores, base + kStaticMetaBytes, stream);

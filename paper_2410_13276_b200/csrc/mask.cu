@@ -311,6 +311,70 @@ int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer
   return launch_mask_band(ctx, m, scores, 0, 0, m.rows, true, p, row_ptr, col_idx, col_capacity, nnz_out, stream);
 }
 
+// ----------------------------------------------------------------------------------------------- 128-token lists -> 64-token lists
+// A 128-token block j is the pair of 64-token blocks (2j, 2j + 1); the query rows of 128-token block i are the 64-token
+// rows 2i and 2i + 1.  Causality inside the diagonal block: row 2i sees 2i only, row 2i + 1 sees 2i and 2i + 1.  Every
+// other listed block j < i contributes both halves to both rows (they exist: only a sequence's last block can be
+// shorter than 65 tokens).  An entry j > i is not causal; it is passed on as (2j, 2j + 1) and the attention call
+// reports it.  One warp per 64-token row; `fill` = false counts, true writes.
+template <bool kFill>
+__global__ void __launch_bounds__(kMaskWarps * 32)
+expand_kernel(SeqMeta m128, SeqMeta m64, const int32_t* __restrict__ row_ptr128, const int32_t* __restrict__ col_idx128,
+              int32_t* __restrict__ row_ptr64, int32_t* __restrict__ col_idx64, int64_t col_capacity64) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * kMaskWarps + (threadIdx.x >> 5);
+  if (r >= m64.rows) return;
+  const int b = find_sequence(m64.blk_off, m64.batch, (int)(r / m64.num_q_heads));
+  const int nb64 = m64.blk_off[b + 1] - m64.blk_off[b], nb128 = m128.blk_off[b + 1] - m128.blk_off[b];
+  const int64_t local = r - (int64_t)m64.num_q_heads * m64.blk_off[b];
+  const int h = (int)(local / nb64);
+  const int i64 = (int)(local - (int64_t)h * nb64);
+  const int i128 = i64 >> 1;
+  const bool odd = (i64 & 1) != 0;
+  const int64_t src = (int64_t)m128.num_q_heads * m128.blk_off[b] + (int64_t)h * nb128 + i128;
+  const int32_t s0 = row_ptr128[src], s1 = row_ptr128[src + 1];
+  int32_t out0 = 0;
+  if (kFill) {
+    out0 = row_ptr64[r];
+    if ((int64_t)row_ptr64[r + 1] > col_capacity64) return;    // does not fit; status already raised by the scan
+  }
+  int written = 0;
+  for (int base = s0; base < s1; base += 32) {
+    const int e = base + lane;
+    const int j = e < s1 ? col_idx128[e] : -1;
+    const int c = e < s1 ? ((j == i128 && !odd) ? 1 : 2) : 0;
+    int incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (kFill && c > 0) {
+      int32_t* dst = col_idx64 + out0 + written + incl - c;
+      dst[0] = 2 * j;
+      if (c == 2) dst[1] = 2 * j + 1;
+    }
+    written += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (!kFill && lane == 0) row_ptr64[r + 1] = written;
+}
+
+int launch_expand_lists(seer_ctx* ctx, const SeqMeta& m128, const SeqMeta& m64, const int32_t* row_ptr128,
+                        const int32_t* col_idx128, int32_t* row_ptr64, int32_t* col_idx64, int64_t col_capacity64,
+                        int64_t* nnz_out, cudaStream_t stream) {
+  if (m64.rows == 0) {
+    cudaMemsetAsync(row_ptr64, 0, sizeof(int32_t), stream);
+    if (nnz_out) cudaMemsetAsync(nnz_out, 0, sizeof(int64_t), stream);
+    return 0;
+  }
+  const unsigned grid = (unsigned)((m64.rows + kMaskWarps - 1) / kMaskWarps);
+  expand_kernel<false><<<grid, kMaskWarps * 32, 0, stream>>>(m128, m64, row_ptr128, col_idx128, row_ptr64, col_idx64, col_capacity64);
+  scan_kernel<<<1, 1024, 0, stream>>>(m64.rows, row_ptr64, 1, col_capacity64, nnz_out, ctx->d_status);
+  expand_kernel<true><<<grid, kMaskWarps * 32, 0, stream>>>(m128, m64, row_ptr128, col_idx128, row_ptr64, col_idx64, col_capacity64);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 3 : -(int)e;
+}
+
 seer_status init_mask(seer_ctx* ctx) {
   (void)ctx;
   cudaError_t e = cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -19,7 +19,8 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
   if (!s || !s->cu_seqlens_host || s->batch < 1) return SEER_ERR_INVALID_ARG;
   if (s->num_q_heads < 1 || s->num_kv_heads < 1) return SEER_ERR_INVALID_ARG;
   if (s->batch > kMaxBatch) return SEER_ERR_UNSUPPORTED;
-  if (s->head_dim != kHeadDim || s->block != kBlock || s->gate_dim != kGateDim) return SEER_ERR_UNSUPPORTED;
+  if (s->head_dim != kHeadDim || (s->block != kBlock && s->block != 2 * kBlock) || s->gate_dim != kGateDim)
+    return SEER_ERR_UNSUPPORTED;
   if (s->num_q_heads % s->num_kv_heads != 0) return SEER_ERR_UNSUPPORTED;
   const int32_t* cu = s->cu_seqlens_host;
   if (cu[0] != 0) return SEER_ERR_INVALID_ARG;
@@ -27,7 +28,7 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
   int32_t max_nb = 0;
   for (int b = 0; b < s->batch; ++b) {
     if (cu[b + 1] < cu[b]) return SEER_ERR_INVALID_ARG;
-    int64_t nb = ((int64_t)cu[b + 1] - cu[b] + kBlock - 1) / kBlock;
+    int64_t nb = ((int64_t)cu[b + 1] - cu[b] + s->block - 1) / s->block;
     blocks += nb;
     chunks += (nb + kPoolChunk - 1) / kPoolChunk;
     tiles += (nb + kScoreTile - 1) / kScoreTile;
@@ -66,6 +67,7 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   const int n = shape->batch + 1;
   std::vector<int32_t> key(shape->cu_seqlens_host, shape->cu_seqlens_host + n);
   key.push_back(shape->num_q_heads);
+  key.push_back(shape->block);
   int slot = -1;
   for (int i = 0; i < kMetaSlots; ++i)
     if (ctx->slots[i].key == key) { slot = i; break; }
@@ -86,7 +88,7 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
     blk[0] = 0; chk[0] = 0; til[0] = 0; sc[0] = 0;
     for (int b = 0; b < shape->batch; ++b) {
       cu[b] = shape->cu_seqlens_host[b];
-      int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + kBlock - 1) / kBlock;
+      int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + shape->block - 1) / shape->block;
       blk[b + 1] = blk[b] + nb;
       chk[b + 1] = chk[b] + (nb + kPoolChunk - 1) / kPoolChunk;
       til[b + 1] = til[b] + (nb + kScoreTile - 1) / kScoreTile;
@@ -120,6 +122,7 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   m->rows = t.rows;
   m->score_elems = t.score_elems;
   m->softmax_scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 0.08838834764831845f;  // 1/sqrt(128)
+  m->block = shape->block;
   *slot_out = slot;
   return SEER_OK;
 }
@@ -311,6 +314,7 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   ShapeTotals t;
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
+  if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;   // 128-token lists go through seer_expand_block_lists first
   if (t.total_blocks == 0) return SEER_OK;
   if (!q || !k || !v || !row_ptr || !o) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
@@ -332,6 +336,7 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
   ShapeTotals t;
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
+  if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;
   if (t.total_blocks == 0) return SEER_OK;
   if (!q || !k || !row_ptr || !lse) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
@@ -412,7 +417,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
   };
   const int32_t* cu = shape->cu_seqlens_host;
   const int Hq = shape->num_q_heads;
-  auto blocks_of = [&](int b) { return ((int64_t)cu[b + 1] - cu[b] + kBlock - 1) / kBlock; };
+  auto blocks_of = [&](int b) { return ((int64_t)cu[b + 1] - cu[b] + shape->block - 1) / shape->block; };
   int64_t blk_off = 0, tile_off = 0, score_off = 0;    // of sequence b
   for (int b = 0; b < shape->batch && !bad;) {
     const int64_t nb = blocks_of(b);
@@ -457,6 +462,33 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
   finish_call(ctx, slot, stream);
   if (bad) return SEER_ERR_CUDA;
   ctx->launches += launched;
+  return SEER_OK;
+}
+
+seer_status seer_expand_block_lists(seer_ctx* ctx, const seer_shape* shape, const int32_t* row_ptr, const int32_t* col_idx,
+                                    int32_t* row_ptr64, int32_t* col_idx64, int64_t col_capacity64, int64_t* nnz_out,
+                                    void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!ctx || !shape) return SEER_ERR_INVALID_ARG;
+  if (shape->block != 2 * kBlock) return SEER_ERR_UNSUPPORTED;
+  seer_shape fine = *shape;
+  fine.block = kBlock;
+  ShapeTotals t128, t64;
+  seer_status st = shape_totals(shape, &t128);
+  if (st == SEER_OK) st = shape_totals(&fine, &t64);
+  if (st != SEER_OK) return st;
+  if (!row_ptr64 || col_capacity64 < 0 || (col_capacity64 > 0 && !col_idx64)) return SEER_ERR_INVALID_ARG;
+  if (t128.total_blocks > 0 && !row_ptr) return SEER_ERR_INVALID_ARG;
+  SeqMeta m128, m64; int slot128, slot64;
+  st = prepare(ctx, shape, stream, &m128, &slot128);
+  if (st != SEER_OK) return st;
+  st = prepare(ctx, &fine, stream, &m64, &slot64);
+  if (st != SEER_OK) { finish_call(ctx, slot128, stream); return st; }
+  int n = launch_expand_lists(ctx, m128, m64, row_ptr, col_idx, row_ptr64, col_idx64, col_capacity64, nnz_out, stream);
+  finish_call(ctx, slot128, stream);
+  finish_call(ctx, slot64, stream);
+  if (n < 0) return SEER_ERR_CUDA;
+  ctx->launches += n;
   return SEER_OK;
 }
 
@@ -543,6 +575,7 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
   ShapeTotals full, t;
   seer_status st = shape_totals(shape, &full);
   if (st != SEER_OK) return st;
+  if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;
   if (full.total_blocks == 0) return SEER_OK;
   if (!q_host || !k_host || !v_host || !Wq_host || !Wk_host || !o_host) return SEER_ERR_INVALID_ARG;
   seer_shape slice;

@@ -10,7 +10,7 @@
 
 namespace seer {
 
-constexpr int kBlock = 64;      // gate block = attention tile
+constexpr int kBlock = 64;      // attention tile; the gate block is 64 or 128 tokens (SeqMeta::block)
 constexpr int kHeadDim = 128;
 constexpr int kGateDim = 128;
 constexpr int kMaxBatch = 4096;
@@ -37,6 +37,7 @@ struct SeqMeta {
   int64_t rows;                // Hq * total_blocks
   int64_t score_elems;
   float softmax_scale;
+  int32_t block;               // tokens per gate block: 64, or 128 (gate and mask only)
 };
 
 // A rectangle of (64-row score tile, query head) pairs whose scores are produced and consumed together; tiles are
@@ -102,6 +103,10 @@ int launch_gate_scores_band(const SeqMeta& m, const ScoreBand& band, const void*
 int launch_mask_band(seer_ctx* ctx, const SeqMeta& m, const float* scores, int64_t score_base, int64_t row_lo,
                      int64_t row_hi, bool first, const seer_mask_params& p, int32_t* row_ptr, int32_t* col_idx,
                      int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream);
+// 128-token block lists -> the 64-token lists the attention kernels take (m128 and m64 describe the same batch).
+int launch_expand_lists(seer_ctx* ctx, const SeqMeta& m128, const SeqMeta& m64, const int32_t* row_ptr128,
+                        const int32_t* col_idx128, int32_t* row_ptr64, int32_t* col_idx64, int64_t col_capacity64,
+                        int64_t* nnz_out, cudaStream_t stream);
 int launch_mask(seer_ctx* ctx, const SeqMeta& m, const float* scores, const seer_mask_params& p, int32_t* row_ptr,
                 int32_t* col_idx, int64_t col_capacity, int64_t* nnz_out, cudaStream_t stream);
 int launch_attn_mma(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,

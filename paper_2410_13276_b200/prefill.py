@@ -21,7 +21,7 @@ def _bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:
 class Prefill:
     def __init__(self, cu_seqlens, num_q_heads: int, num_kv_heads: int, *, device: int = 0,
                  ctx: Optional[B.Context] = None, softmax_scale: float = 0.0, col_capacity: Optional[int] = None,
-                 want_lse: bool = True):
+                 want_lse: bool = True, block: int = 64):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device("cuda", device)
@@ -29,7 +29,11 @@ class Prefill:
         self.ctx = ctx or B.Context(device)
         self.cu = np.asarray(cu_seqlens, dtype=np.int32)
         self.hq, self.hkv = num_q_heads, num_kv_heads
-        self.shape = B.make_shape(self.cu, num_q_heads, num_kv_heads, softmax_scale=softmax_scale)
+        self.block = block
+        self.shape = B.make_shape(self.cu, num_q_heads, num_kv_heads, softmax_scale=softmax_scale, block=block)
+        # the attention kernels tile by 64 tokens: 128-token lists are expanded for them (seer_expand_block_lists)
+        self.attn_shape = self.shape if block == 64 else B.make_shape(self.cu, num_q_heads, num_kv_heads,
+                                                                      softmax_scale=softmax_scale, block=64)
         self.T = int(self.cu[-1])
         self.rows = B.seer_mask_rows(self.shape)
         self.causal_blocks = B.seer_causal_blocks(self.shape)
@@ -43,6 +47,10 @@ class Prefill:
         self.col_idx = torch.empty(max(cap, 1), dtype=torch.int32, device=d)
         self.col_capacity = cap
         self.nnz = torch.zeros(1, dtype=torch.int64, device=d)
+        if block != 64:
+            self.row_ptr64 = torch.zeros(B.seer_mask_rows(self.attn_shape) + 1, dtype=torch.int32, device=d)
+            self.col_idx64 = torch.empty(max(4 * cap, 1), dtype=torch.int32, device=d)
+            self.nnz64 = torch.zeros(1, dtype=torch.int64, device=d)
         self.q = self.k = self.v = self.wq = self.wk = None
         self.o = torch.empty((self.T, num_q_heads, 128), dtype=torch.bfloat16, device=d)
         self.lse = torch.empty((num_q_heads, self.T), dtype=torch.float32, device=d) if want_lse else None
@@ -84,6 +92,8 @@ class Prefill:
         B.seer_gate_block_mask(self.ctx, self.shape, options, self.q, self.k, self.wq if wq is None else wq,
                                self.wk if wk is None else wk, params, self.row_ptr, self.col_idx, self.col_capacity,
                                self.nnz, self.ws_fused, stream)
+        if self.block != 64:
+            self.expand(stream)
 
     def block_max(self, stream=None):
         """Max-pooled attention map on the listed blocks (Eq. 2) from the lse of the last `attn` call; returns the
@@ -99,10 +109,17 @@ class Prefill:
     def mask(self, params: B.seer_mask_params, stream=None):
         B.seer_block_mask(self.ctx, self.shape, self.scores, params, self.row_ptr, self.col_idx, self.col_capacity,
                           self.nnz, None, stream)
+        if self.block != 64:
+            self.expand(stream)
+
+    def expand(self, stream=None):
+        """128-token lists -> the 64-token lists the attention takes."""
+        B.seer_expand_block_lists(self.ctx, self.shape, self.row_ptr, self.col_idx, self.row_ptr64, self.col_idx64, None,
+                                  self.nnz64, stream)
 
     def attn(self, stream=None):
-        B.seer_sparse_attn(self.ctx, self.shape, self.q, self.k, self.v, self.row_ptr, self.col_idx, self.o, self.lse,
-                           None, stream)
+        rp, col = (self.row_ptr, self.col_idx) if self.block == 64 else (self.row_ptr64, self.col_idx64)
+        B.seer_sparse_attn(self.ctx, self.attn_shape, self.q, self.k, self.v, rp, col, self.o, self.lse, None, stream)
 
     def run(self, params: B.seer_mask_params, stream=None):
         self.gate(stream)
@@ -112,6 +129,12 @@ class Prefill:
     # ---- downloads
     def scores_host(self) -> np.ndarray:
         return self.scores[: B.seer_scores_elems(self.shape)].cpu().numpy()
+
+    def lists64_host(self):
+        """The expanded 64-token lists of a 128-token problem."""
+        rp = self.row_ptr64.cpu().numpy().astype(np.int64)
+        n = min(int(rp[-1]), self.col_idx64.numel())
+        return rp, self.col_idx64[:n].cpu().numpy()
 
     def lists_host(self):
         rp = self.row_ptr.cpu().numpy().astype(np.int64)

@@ -301,7 +301,7 @@ def test_invalid_arguments_are_rejected_on_the_host(rt):
     B, Prefill, ctx = rt
     import torch
     buf = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
-    for bad in (dict(head_dim=64), dict(block=128), dict(gate_dim=64)):
+    for bad in (dict(head_dim=64), dict(block=32), dict(block=256), dict(gate_dim=64)):
         s = B.make_shape([0, 128], 2, 1, **bad)
         with pytest.raises(B.SeerError) as e:
             B.seer_gate_scores(ctx, s, buf, buf, buf, buf, buf, buf)

@@ -39,6 +39,17 @@ def test_sizing_helpers_closed_forms(lib):
     assert B.seer_causal_blocks(v) == 27891200
     r = B.make_shape([0, 65, 65, 130], 2, 1)                 # ragged, with an empty sequence
     assert B.seer_mask_rows(r) == 2 * (2 + 0 + 2) and B.seer_scores_elems(r) == 2 * (4 + 0 + 4)
+    # 128-token gate blocks: a quarter of the score matrix, half the rows; other block sizes are rejected
+    s128 = B.make_shape([0, 131072], 32, 8, block=128)
+    assert B.seer_mask_rows(s128) == 32 * 1024 and B.seer_scores_elems(s128) == 32 * 1024 * 1024
+    assert B.seer_causal_blocks(s128) == 32 * 1024 * 1025 // 2
+    r128 = B.make_shape([0, 65, 65, 194], 2, 1, block=128)   # 65 tokens: one block of 128, two of 64
+    assert B.seer_mask_rows(r128) == 2 * (1 + 0 + 2)
+    assert B.seer_mask_rows(B.make_shape([0, 128], 2, 1, block=32)) == -1
+    assert B.seer_mask_rows(B.make_shape([0, 128], 2, 1, block=256)) == -1
+    # gate + mask in one call: the projected vectors plus the band scratch, never less than 64 rows of the longest sequence
+    assert B.seer_gate_mask_workspace_bytes(s, 128 << 20) == B.seer_workspace_bytes(s) + (128 << 20)
+    assert B.seer_gate_mask_workspace_bytes(s, 0) == B.seer_workspace_bytes(s) + (64 * 2048 + 4) * 4 + 240
     # the host-buffer path works on one KV head (4 query heads) at a time: two sets of slice inputs / outputs
     # (q, o: 2 x 2 x 134 MB; k, v: 2 x 2 x 33.5 MB) and one set of slice intermediates (scores 67 MB, lists 33.6 MB)
     assert 0.75e9 < B.seer_prefill_host_arena_bytes(s) < 0.85e9

@@ -18,6 +18,9 @@ What it follows
   of unselected blocks are skipped, i.e. dense attention A = softmax(QK^T/sqrt(d))
   (Sec. 2) with the unselected blocks removed from every softmax row
   (`sparse_attention`).
+* Chunked prefill (the queries are the last S_q positions of a sequence of S_k keys): the same definitions with the
+  query positions shifted (`chunk_offsets`, `gate_scores_chunk`, `block_mask_chunk`, `sparse_attention_chunk`); rows
+  keep the numbering of the whole sequence, so a chunk's results are rows of the whole problem's.
 * 2D-max-pooled attention map used as distillation target, Sec. 3.2 / Eq. 2 and
   the appendix's a_ij = exp(r_ij - m_i) / l_i (`maxpool_attention_map`).
 
@@ -105,16 +108,17 @@ def gate_logits(gq: np.ndarray, gk: np.ndarray) -> np.ndarray:
     return L
 
 
-def causal_softmax_rows(L: np.ndarray) -> np.ndarray:
+def causal_softmax_rows(L: np.ndarray, first: int = 0) -> np.ndarray:
     """Row softmax of Eq. 1 restricted to the causal blocks j <= i of row i
     (a query block cannot attend to later key blocks, and the rows must sum
-    to 1 as Sec. 3.2 states).  Entries j > i are returned as 0."""
-    nb = L.shape[-1]
+    to 1 as Sec. 3.2 states).  Entries j > i are returned as 0.  `first` is the
+    block position of row 0 (rows are query blocks first, first + 1, ...)."""
     S = np.zeros_like(L)
-    for i in range(nb):
-        row = L[..., i, : i + 1]
+    for r in range(L.shape[-2]):
+        i = first + r
+        row = L[..., r, : i + 1]
         e = np.exp(row - row.max(axis=-1, keepdims=True))
-        S[..., i, : i + 1] = e / e.sum(axis=-1, keepdims=True)
+        S[..., r, : i + 1] = e / e.sum(axis=-1, keepdims=True)
     return S
 
 
@@ -169,16 +173,16 @@ def pool_compose(x_bits: np.ndarray, cu_seqlens, B: int, methods: int) -> list:
     return out
 
 
-def block_rope(g: np.ndarray, theta: float, B: int) -> np.ndarray:
+def block_rope(g: np.ndarray, theta: float, B: int, first: int = 0) -> np.ndarray:
     """Sec. 3.1, "Block-level RoPE in AttnGate": rotary position encoding applied after the gate's linear layer,
     at block granularity, with the reduced base theta' = theta / B.  g is [H, nb, dg] for one sequence; block i
-    is position i.  Standard rotary form (a reading, the paper gives none): pair (c, c + dg/2), frequency
+    is position first + i.  Standard rotary form (a reading, the paper gives none): pair (c, c + dg/2), frequency
     theta'^(-2c/dg), (x_c, x_{c+dg/2}) -> (x_c cos a - x_{c+dg/2} sin a, x_{c+dg/2} cos a + x_c sin a), a = i * frequency."""
     H, nb, dg = g.shape
     half = dg // 2
     base = float(theta) / float(B)
     freq = base ** (-2.0 * np.arange(half, dtype=np.float64) / dg)          # [half]
-    ang = np.arange(nb, dtype=np.float64)[:, None] * freq[None, :]           # [nb, half]
+    ang = (first + np.arange(nb, dtype=np.float64))[:, None] * freq[None, :]  # [nb, half]
     c, s = np.cos(ang), np.sin(ang)
     x1, x2 = g[..., :half], g[..., half:]
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
@@ -336,6 +340,89 @@ def sparse_attention(q_bits, k_bits, v_bits, cu_seqlens, row_ptr, col_idx, num_q
                 ls[dead] = -np.inf
                 o[tq, h, :] = out
                 lse[h, tq] = ls
+    return o, lse
+
+
+# --------------------------------------------------------------------------- chunked prefill
+def chunk_offsets(cu_seqlens_q, cu_seqlens_k, B: int) -> np.ndarray:
+    """Per sequence, the block position of the chunk's first query block: the S_q queries are the last S_q positions
+    of the S_k keys and the chunk starts on a block boundary (a reading: the paper evaluates whole prompts; serving
+    stacks split them into block-aligned chunks)."""
+    sq = np.diff(np.asarray(cu_seqlens_q, dtype=np.int64))
+    sk = np.diff(np.asarray(cu_seqlens_k, dtype=np.int64))
+    if np.any(sq > sk) or np.any(((sk - sq) % B != 0) & (sq > 0)):
+        raise ValueError("a chunk must end its sequence and start on a block boundary")
+    return np.where(sq > 0, (sk - sq) // B, (sk + B - 1) // B)     # a sequence without queries: past its last block
+
+
+def gate_scores_chunk(q_bits, k_bits, wq, wk, cu_seqlens_q, cu_seqlens_k, B: int, pool_q: int = POOL_AVG,
+                      pool_k: int = POOL_AVG, rope_theta: float = 0.0) -> list:
+    """Eq. 1 for a chunk: q_bits holds only the chunk's tokens.  Returns per sequence the fp32 array
+    [Hq, nbq, nbk]; row r is query block off + r of the sequence and its softmax runs over key blocks j <= off + r."""
+    off = chunk_offsets(cu_seqlens_q, cu_seqlens_k, B)
+    pq = pool_compose(q_bits, cu_seqlens_q, B, pool_q)
+    pk = pool_compose(k_bits, cu_seqlens_k, B, pool_k)
+    out = []
+    for b in range(len(pq)):
+        gq, gk = project(pq[b], wq), project(pk[b], wk)
+        if rope_theta > 0.0:
+            gq, gk = block_rope(gq, rope_theta, B, first=int(off[b])), block_rope(gk, rope_theta, B)
+        Hq, nbq, dg = gq.shape
+        G = Hq // gk.shape[0]
+        L = np.empty((Hq, nbq, gk.shape[1]), dtype=np.float64)
+        for h in range(Hq):
+            L[h] = gq[h] @ gk[h // G].T / math.sqrt(dg)
+        out.append(causal_softmax_rows(L, first=int(off[b])).astype(np.float32))
+    return out
+
+
+def block_mask_chunk(scores: list, mode: int, *, keep_num=1, keep_den=1, k=0, threshold=0.0, flags=FORCE_DIAG):
+    """Lists for a chunk from its [Hq, nbq, nbk] score arrays, in the row numbering of the whole sequences: the CSR
+    structure has Hq * nbk rows per sequence and the rows of the blocks before the chunk are empty."""
+    row_ptr, cols = [0], []
+    for S in scores:
+        Hq, nbq, nbk = S.shape
+        off = nbk - nbq
+        for h in range(Hq):
+            for i in range(nbk):
+                if i >= off:
+                    cols.extend(select_row(S[h, i - off], i, mode, keep_num=keep_num, keep_den=keep_den, k=k,
+                                           threshold=threshold, flags=flags))
+                row_ptr.append(len(cols))
+    return np.asarray(row_ptr, dtype=np.int64), np.asarray(cols, dtype=np.int32)
+
+
+def sparse_attention_chunk(q_bits, k_bits, v_bits, cu_seqlens_q, cu_seqlens_k, row_ptr, col_idx, num_q_heads: int,
+                           num_kv_heads: int, B: int, scale: float):
+    """Block-sparse attention of a chunk: query token u of sequence b (0 <= u < S_q) sits at position S_k - S_q + u and
+    sees the keys at positions <= its own inside the key blocks listed for row (b, head, its block), rows numbered
+    over the whole sequence.  Returns o [Tq, Hq, d] and lse [Hq, Tq]; a token with no key gets o = 0, lse = -inf."""
+    Tq, Hq, d = q_bits.shape
+    G = num_q_heads // num_kv_heads
+    o = np.zeros((Tq, Hq, d), dtype=np.float64)
+    lse = np.full((Hq, Tq), -np.inf, dtype=np.float64)
+    base = row_base(cu_seqlens_k, B, num_q_heads)
+    for b in range(len(cu_seqlens_k) - 1):
+        k0, k1 = int(cu_seqlens_k[b]), int(cu_seqlens_k[b + 1])
+        q0, q1 = int(cu_seqlens_q[b]), int(cu_seqlens_q[b + 1])
+        Sk, Sq = k1 - k0, q1 - q0
+        nbk = (Sk + B - 1) // B
+        for h in range(num_q_heads):
+            Kh = bf16_bits_to_f64(k_bits[k0:k1, h // G, :])
+            Vh = bf16_bits_to_f64(v_bits[k0:k1, h // G, :])
+            for u in range(Sq):
+                pos = Sk - Sq + u
+                r = int(base[b]) + h * nbk + pos // B
+                keys = [t for j in col_idx[int(row_ptr[r]):int(row_ptr[r + 1])]
+                        for t in range(int(j) * B, min((int(j) + 1) * B, Sk)) if t <= pos]
+                if not keys:
+                    continue
+                qv = bf16_bits_to_f64(q_bits[q0 + u, h, :])
+                sc = (Kh[keys] @ qv) * scale
+                m = sc.max()
+                p = np.exp(sc - m)
+                o[q0 + u, h, :] = (p @ Vh[keys]) / p.sum()
+                lse[h, q0 + u] = m + math.log(p.sum())
     return o, lse
 
 

@@ -79,16 +79,46 @@ def peaks():
 
 
 class ClockSampler:
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """nvidia-smi polled every 100 ms from before the warm-up (its start-up alone takes a few hundred ms); stop()
+    keeps the samples taken between mark_start() and mark_end().  When the timed region was too short for three
+    samples, the caller keeps the same load running a little longer before mark_end() and the result says so."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.t0 = self.t1 = None
+        self.extended = False
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
                                        "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
+
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
+    def _rows(self):
+        import datetime
+        out = []
+        try:
+            lines = [l.strip() for l in open(self.f.name) if l.strip()]
+        except OSError:
+            return out
+        for l in lines:
+            r = l.split(", ")
+            try:
+                ts = datetime.datetime.strptime(r[0].strip(), "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                out.append((ts, float(r[1]), float(r[2]), float(r[3]), [v.strip().lower() == "active" for v in r[4:8]]))
+            except (ValueError, IndexError):
+                continue
+        return out
+
+    def count_since_start(self) -> int:
+        return sum(1 for r in self._rows() if self.t0 is not None and r[0] >= self.t0)
 
     def stop(self):
         if self.p is None:
@@ -99,22 +129,18 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.p.kill()
         self.f.flush()
-        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        rows = self._rows()
         os.unlink(self.f.name)
-        sm, mx, reasons, power = [], [], set(), []
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
-            except (ValueError, IndexError):
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.strip().lower() == "active":
-                    reasons.add(n)
-        if not sm:
+        t0 = self.t0 if self.t0 is not None else 0.0
+        t1 = self.t1 if self.t1 is not None else time.time()
+        rows = [r for r in rows if t0 <= r[0] <= t1 + 0.05]
+        if not rows:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
-                "power_w_max": max(power), "samples": len(sm)}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in rows for n, v in zip(names, r[4]) if v})
+        return {"sm_mhz": float(np.median([r[1] for r in rows])), "sm_max_mhz": float(max(r[2] for r in rows)),
+                "reasons": reasons, "power_w_max": max(r[3] for r in rows), "samples": len(rows),
+                "load_extended_for_sampling": self.extended}
 
 
 def cpu_oracle_sample(w, rp, col, budget_rows=None):
@@ -225,6 +251,7 @@ def main():
     params = B.make_mask_params(spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
                                 threshold=spec.threshold or 0.0, flags=spec.flags)
     stream = torch.cuda.current_stream()
+    sampler = ClockSampler(local) if rank == 0 else None     # polls from here on; only the timed region's samples are kept
 
     def barrier():
         if world > 1:
@@ -238,9 +265,10 @@ def main():
     nnz = int(p.nnz.item())
 
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    sampler = ClockSampler(local) if rank == 0 else None
     l0 = B.seer_launch_count(p.ctx)
     barrier()
+    if sampler:
+        sampler.mark_start()
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for s in range(args.steps):
@@ -252,7 +280,16 @@ def main():
     barrier()
     total_ms = t_start.elapsed_time(t_end)
     launches = B.seer_launch_count(p.ctx) - l0
-    clocks = sampler.stop() if sampler else None
+    clocks = None
+    if sampler:
+        # a short timed region may have seen fewer than three samples: keep the same load running (untimed) until it has
+        t_lim = time.time() + 3.0
+        while sampler.count_since_start() < 3 and time.time() < t_lim:
+            sampler.extended = True
+            p.gate(); p.mask(params); p.attn()
+            torch.cuda.synchronize()
+        sampler.mark_end()
+        clocks = sampler.stop()
     assert p.status() == 0
     if world > 1:
         t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
@@ -340,6 +377,34 @@ def main():
         p.scores = torch.empty(max(B.seer_scores_elems(p.shape), 1), dtype=torch.float32, device="cuda")
         p.gate(); p.mask(params)                             # back to the bench lists
 
+    # chunked prefill: the last 8192 tokens of the same layer as queries against all its keys (block-aligned chunk;
+    # rows and lists keep the numbering of the whole sequence), outside the timed region
+    chunked = None
+    if rank == 0 and w.total_tokens >= 16384 and len(w.cu_seqlens) == 2:
+        ct = 8192
+        p.scores = None
+        p3 = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, device=local, ctx=p.ctx, want_lse=False,
+                     cu_seqlens_q=[0, ct])
+        p3.q = p.q[w.total_tokens - ct:].contiguous()
+        p3.k, p3.v, p3.wq, p3.wk = p.k, p.v, p.wq, p.wk
+        for _ in range(2):
+            p3.run(params)
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record(stream); p3.gate(); e[1].record(stream); p3.mask(params); e[2].record(stream); p3.attn(); e[3].record(stream)
+        torch.cuda.synchronize()
+        n3 = int(p3.nnz.item())
+        t = [e[i].elapsed_time(e[i + 1]) for i in range(3)]
+        o3 = p3.o
+        del p3
+        p.scores = torch.empty(max(B.seer_scores_elems(p.shape), 1), dtype=torch.float32, device="cuda")
+        p.gate(); p.mask(params); p.attn()                   # the whole layer again: the chunk must equal its last rows
+        torch.cuda.synchronize()
+        same = bool(torch.equal(o3, p.o[w.total_tokens - ct:]))
+        chunked = {"chunk_tokens": ct, "gate_ms": t[0], "mask_ms": t[1], "attn_ms": t[2], "kept_blocks": n3,
+                   "attn_tflops": n3 * FLOP_PER_BLOCK / (t[2] * 1e-3) / 1e12, "o_equals_rows_of_whole_run": same}
+        del o3
+
     # the max-pooled attention map on the kept blocks (Eq. 2; a side output for distillation / diagnostics), outside the
     # timed region: one attention launch that also writes lse, then the block-max pass
     block_max_ms = None
@@ -400,7 +465,7 @@ def main():
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
                             "kernel": "seer_sparse_attn"},
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
-               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128,
+               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128, "chunked_prefill": chunked,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:
             dense_blocks = B.seer_causal_blocks(p.shape)

@@ -75,7 +75,23 @@ typedef struct {
                                      seer_expand_block_lists */
   int32_t gate_dim;               /* 128: output width of the gate's linear layers */
   float softmax_scale;            /* attention logit scale; <= 0 selects 1/sqrt(head_dim) (Sec. 2) */
+  const int32_t* cu_seqlens_q_host; /* HOST [batch + 1] or NULL.  NULL: every sequence has as many queries as keys.
+                                     Otherwise chunked prefill, see below */
 } seer_shape;
+
+/* Chunked prefill (the paper prefills whole prompts; a serving stack feeds them in pieces against a growing KV cache).
+ *
+ * With cu_seqlens_q_host set, sequence b has S_k = cu_seqlens[b+1] - cu_seqlens[b] keys and S_q = cu_q[b+1] - cu_q[b]
+ * queries, which are the LAST S_q positions of the sequence; S_q <= S_k, and the chunk starts on a block boundary
+ * ((S_k - S_q) a multiple of `block`) unless S_q = 0.  q, o are [cu_q[batch], num_q_heads, head_dim] and lse
+ * [num_q_heads, cu_q[batch]]: they hold the chunk's tokens only; k, v hold all S_k tokens.
+ * Everything indexed by blocks keeps the numbering of the whole sequence: nb_b = ceil(S_k / block), the score matrix is
+ * [num_q_heads][nb_b][nb_b] per sequence, the CSR structure has num_q_heads * nb_b rows per sequence, and block-level
+ * RoPE rotates a query block by its position in the sequence.  Only the rows of the chunk's query blocks are produced:
+ * score rows before the chunk are not written, their CSR rows are empty, and lists given for them are ignored by the
+ * attention.  The results are those of the whole problem restricted to the chunk (same kernels, same arithmetic).
+ * A score buffer of full size is only needed by the separate gate and mask calls; seer_gate_block_mask needs none.
+ * Not supported with a chunk (SEER_ERR_UNSUPPORTED): seer_prefill_host, seer_gate_scores_static. */
 
 /* Sizing helpers (pure host arithmetic; return 0 / -1 on an invalid shape). */
 size_t seer_workspace_bytes(const seer_shape* shape); /* enough for any of the three calls */

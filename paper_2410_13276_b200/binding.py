@@ -41,7 +41,7 @@ class SeerError(RuntimeError):
 class seer_shape(C.Structure):
     _fields_ = [("batch", C.c_int32), ("cu_seqlens_host", C.POINTER(C.c_int32)), ("num_q_heads", C.c_int32),
                 ("num_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("block", C.c_int32), ("gate_dim", C.c_int32),
-                ("softmax_scale", C.c_float)]
+                ("softmax_scale", C.c_float), ("cu_seqlens_q_host", C.POINTER(C.c_int32))]
 
 
 class seer_mask_params(C.Structure):
@@ -140,11 +140,15 @@ def _check(status: int, where: str) -> None:
 
 
 def make_shape(cu_seqlens: Sequence[int], num_q_heads: int, num_kv_heads: int, *, head_dim: int = 128,
-               block: int = 64, gate_dim: int = 128, softmax_scale: float = 0.0) -> seer_shape:
+               block: int = 64, gate_dim: int = 128, softmax_scale: float = 0.0, cu_seqlens_q=None) -> seer_shape:
+    """cu_seqlens_q (optional): chunked prefill, the queries are the last cu_q[b+1] - cu_q[b] positions of sequence b."""
     cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    cuq = None if cu_seqlens_q is None else np.ascontiguousarray(np.asarray(cu_seqlens_q, dtype=np.int32))
+    if cuq is not None and len(cuq) != len(cu):
+        raise ValueError("cu_seqlens_q must have batch + 1 entries")
     s = seer_shape(len(cu) - 1, cu.ctypes.data_as(C.POINTER(C.c_int32)), num_q_heads, num_kv_heads, head_dim, block,
-                   gate_dim, softmax_scale)
-    s._keepalive = cu          # the struct points into this array
+                   gate_dim, softmax_scale, None if cuq is None else cuq.ctypes.data_as(C.POINTER(C.c_int32)))
+    s._keepalive = (cu, cuq)   # the struct points into these arrays
     return s
 
 

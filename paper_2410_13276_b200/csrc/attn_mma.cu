@@ -77,13 +77,17 @@ attn_mma_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __res
   const int s0 = m.cu_seqlens[b];
   const int slen = m.cu_seqlens[b + 1] - s0;
   const int q_valid = min(kBlock, slen - i * kBlock);
+  // chunked prefill: q / o / lse hold the last positions only (token index shifted by qdelta); blocks before the chunk do nothing
+  if (m.chunked && i < m.qoff[b]) return;
+  const int64_t tok0 = (int64_t)s0 + (int64_t)i * kBlock + (m.chunked ? m.qdelta[b] : 0);
+  const int64_t lse_stride = m.chunked ? m.total_q_tokens : m.total_tokens;
   const int l0 = row_ptr[r], l1 = row_ptr[r + 1];
   const int nlist = l1 - l0;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
 
-  load_tile_async(sQ, q, (int64_t)s0 + (int64_t)i * kBlock, q_valid, m.num_q_heads, h);
+  load_tile_async(sQ, q, tok0, q_valid, m.num_q_heads, h);
   cp_async_commit();
 
   auto fetch = [&](int it, uint32_t dK, uint32_t dV) -> int {
@@ -224,7 +228,6 @@ attn_mma_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __res
     asm volatile("st.shared.b32 [%0], %1;" ::"r"(sQ + tile_off(r0 + 8, n) + tig * 4), "r"(hi) : "memory");
   }
   __syncwarp();
-  const int64_t tok0 = (int64_t)s0 + (int64_t)i * kBlock;
 #pragma unroll
   for (int rr = 0; rr < 16; rr += 2) {
     const int row = warp * 16 + rr + (lane >> 4);
@@ -240,7 +243,7 @@ attn_mma_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __res
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int row = warp * 16 + gid + e * 8;
-      if (row < q_valid) lse[(int64_t)h * m.total_tokens + tok0 + row] = lse_v[e];
+      if (row < q_valid) lse[(int64_t)h * lse_stride + tok0 + row] = lse_v[e];
     }
   }
 }
@@ -278,10 +281,12 @@ block_max_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __re
   const int l0 = row_ptr[r], l1 = row_ptr[r + 1];
   const int nlist = l1 - l0;
   if (nlist <= 0) return;
+  if (m.chunked && i < m.qoff[b]) return;                // chunked prefill: a block before the chunk
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gid = lane >> 2, tig = lane & 3;
-  const int64_t tok0 = (int64_t)s0 + (int64_t)i * kBlock;
+  const int64_t tok0 = (int64_t)s0 + (int64_t)i * kBlock + (m.chunked ? m.qdelta[b] : 0);   // in q / lse
+  const int64_t lse_stride = m.chunked ? m.total_q_tokens : m.total_tokens;
 
   load_tile_async(sQ, q, tok0, q_valid, m.num_q_heads, h);
   cp_async_commit();
@@ -307,7 +312,7 @@ block_max_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __re
   for (int e = 0; e < 2; ++e) {
     const int row = warp * 16 + gid + e * 8;
     row_ok[e] = row < q_valid;
-    lse2[e] = row_ok[e] ? lse[(int64_t)h * m.total_tokens + tok0 + row] * 1.4426950408889634f : 0.f;
+    lse2[e] = row_ok[e] ? lse[(int64_t)h * lse_stride + tok0 + row] * 1.4426950408889634f : 0.f;
   }
 
   uint32_t qf[8][4];

@@ -234,10 +234,13 @@ __device__ __forceinline__ float ex2f(float x) {
 }
 
 struct Item {
-  int b, h, g, i, nb, s0, slen, l0, nlist, ntiles, q_valid;
+  int b, h, g, i, nb, s0, slen, l0, nlist, ntiles, q_valid, dq;
   int64_t row;
 };
 
+// kChunk: chunked prefill.  q / o / lse hold the last positions of each sequence only: their token index is the k / v
+// token index plus dq, and query blocks before the chunk have nothing to do whatever their lists say.
+template <bool kChunk>
 __device__ __forceinline__ Item decode_item(const SeqMeta& m, const int32_t* __restrict__ row_ptr, int64_t w) {
   Item it;
   it.b = find_sequence(m.blk_off, m.batch, (int)(w / m.num_q_heads));
@@ -253,6 +256,11 @@ __device__ __forceinline__ Item decode_item(const SeqMeta& m, const int32_t* __r
   it.q_valid = min(kBlock, it.slen - it.i * kBlock);
   it.l0 = row_ptr[it.row];
   it.nlist = row_ptr[it.row + 1] - it.l0;
+  it.dq = 0;
+  if (kChunk) {
+    it.dq = m.qdelta[it.b];
+    if (it.i < m.qoff[it.b]) { it.nlist = 0; it.q_valid = 0; }   // no tiles, and no row of o / lse is written
+  }
   it.ntiles = (it.nlist + 1) >> 1;
   return it;
 }
@@ -445,7 +453,7 @@ __device__ __forceinline__ uint32_t softmax_pass(uint32_t s_addr, uint32_t m_add
 }
 
 // ------------------------------------------------------------------------------------------------ kernel
-template <bool kTrace>
+template <bool kTrace, bool kChunk>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, SeqMeta m, const int32_t* __restrict__ row_ptr,
@@ -503,11 +511,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       uint32_t k = 0, g = 0, slot = 0, use = 0;
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
+        const Item it = decode_item<kChunk>(m, row_ptr, w);
         if (it.ntiles == 0) continue;
         if (!mbar_wait(sh, Q_EMPTY, (k & 1u) ^ 1u, status)) break;
         mbar_expect_tx(sh.bar(Q_FULL), kQBytes);
-        const int tq = it.s0 + it.i * kBlock;
+        const int tq = it.s0 + it.i * kBlock + (kChunk ? it.dq : 0);
         tma_load_3d(sh.base + kOffQ, &map_q, sh.bar(Q_FULL), 0, it.h, tq);
         tma_load_3d(sh.base + kOffQ + kHalfQ, &map_q, sh.bar(Q_FULL), 64, it.h, tq);
         ++k;
@@ -561,7 +569,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     uint32_t g = 0;
     bool ok = true;
     for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-      const Item it = decode_item(m, row_ptr, w);
+      const Item it = decode_item<kChunk>(m, row_ptr, w);
       if (it.ntiles == 0) continue;
       int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
       const unsigned char* seq_base = xg + ((size_t)it.s0 * m.num_kv_heads + it.g) * (kHeadDim * 2) + (size_t)chunk * 16 +
@@ -607,7 +615,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint64_t qd = make_desc(sh.base + kOffQ, 16, 1024);
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
+        const Item it = decode_item<kChunk>(m, row_ptr, w);
         if (it.ntiles == 0) continue;
         if (!mbar_wait(sh, Q_FULL, k & 1u, status)) break;
         for (int t = 0; t < it.ntiles; ++t, ++g) {
@@ -646,7 +654,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024);   // P^T buffer (group, buf) lies 2 * group + buf buffers on
       bool ok = true;
       for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item(m, row_ptr, w);
+        const Item it = decode_item<kChunk>(m, row_ptr, w);
         for (int t = 0; t < it.ntiles; ++t, ++g) {
           const int grp = t & 1;
           const uint32_t cn = grp ? cnt_b : cnt_a, st = g & 1u;
@@ -710,8 +718,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     for (int64_t w = blockIdx.x; w < m.rows; w += gridDim.x) {
       tr.sample(0);
-      const Item it = decode_item(m, row_ptr, w);
-      const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock;
+      const Item it = decode_item<kChunk>(m, row_ptr, w);
+      const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock + (kChunk ? it.dq : 0);   // first row of the item in q / o / lse
       const int tiles_a = (it.ntiles + 1) >> 1, tiles_b = it.ntiles >> 1;
       const int my_tiles = grp == 0 ? tiles_a : tiles_b;
       float l_part[64];
@@ -871,7 +879,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           out_lse = (mm + log2f(l)) * 0.6931471805599453f;
         }
         w_a[gt] = wa; w_b[gt] = wb;
-        if (lse != nullptr && gt < it.q_valid) lse[(int64_t)it.h * m.total_tokens + tok0 + gt] = out_lse;
+        if (lse != nullptr && gt < it.q_valid) lse[(int64_t)it.h * (kChunk ? m.total_q_tokens : m.total_tokens) + tok0 + gt] = out_lse;
       }
       named_bar_sync(5, 2 * kGroupThreads);
       // each group merges and stores 32 of the 64 query columns: staging [32 q][128 d] bf16 in its own P^T buffer
@@ -953,9 +961,11 @@ seer_status init_attn_tc(seer_ctx* ctx) {
       qres != cudaDriverEntryPointSuccess)
     return SEER_ERR_CUDA;
   ctx->tmap_encode = fn;
-  cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(tc::attn_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(tc::attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
   return e == cudaSuccess ? SEER_OK : SEER_ERR_CUDA;
 }
 
@@ -965,15 +975,18 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
   // the input pointers must be 16-byte aligned for TMA
   if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15) != 0) return -(int)cudaErrorMisalignedAddress;
   CUtensorMap mq, mk, mv;
-  if (!tc::make_map(ctx, &mq, q, m.total_tokens, m.num_q_heads) || !tc::make_map(ctx, &mk, k, m.total_tokens, m.num_kv_heads) ||
+  if (!tc::make_map(ctx, &mq, q, m.total_q_tokens, m.num_q_heads) || !tc::make_map(ctx, &mk, k, m.total_tokens, m.num_kv_heads) ||
       !tc::make_map(ctx, &mv, v, m.total_tokens, m.num_kv_heads))
     return -(int)cudaErrorInvalidValue;
   const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, m.rows);
-  if (ctx->trace != nullptr)   // the instrumented instantiation
-    tc::attn_tc_kernel<true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
+  if (m.chunked)               // chunked prefill (never instrumented)
+    tc::attn_tc_kernel<false, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
+                                                                          ctx->d_status, (unsigned long long*)ctx->trace);
+  else if (ctx->trace != nullptr)   // the instrumented instantiation
+    tc::attn_tc_kernel<true, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
                                                                     ctx->d_status, (unsigned long long*)ctx->trace);
   else
-    tc::attn_tc_kernel<false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
+    tc::attn_tc_kernel<false, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
                                                                     ctx->d_status, (unsigned long long*)ctx->trace);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;

@@ -75,11 +75,15 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int half = lane >> 4, cchunk = lane & 15;
   const size_t row_stride = (size_t)H * kHeadDim;  // elements between consecutive tokens
+  // chunked prefill: q holds the last positions only; query blocks before the chunk are skipped (projected as zeros)
+  const int q_first = (m.chunked && is_q) ? m.qoff[b] : 0;
+  const int q_shift = (m.chunked && is_q) ? m.qdelta[b] : 0;
+  if (i0 + nblk <= q_first) return;
 
   for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
     const int t0 = s0 + (i0 + bi) * m.block;
-    const int cnt = min(m.block, s1 - t0);
-    const uint16_t* base = x + (size_t)t0 * row_stride + (size_t)h * kHeadDim + cchunk * 8;
+    const int cnt = (i0 + bi < q_first) ? 0 : min(m.block, s1 - t0);
+    const uint16_t* base = x + ((ptrdiff_t)t0 + q_shift) * (ptrdiff_t)row_stride + (size_t)h * kHeadDim + cchunk * 8;
     float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
     for (int it = 0; it < m.block / 2; it += 8) {
@@ -92,7 +96,7 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc_bf16x8(a, u[j]);
     }
-    const float inv = 1.0f / (float)cnt;
+    const float inv = cnt > 0 ? 1.0f / (float)cnt : 0.f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       a[j] += __shfl_xor_sync(0xffffffffu, a[j], 16);
@@ -181,11 +185,15 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int half = lane >> 4, cchunk = lane & 15;
   const size_t row_stride = (size_t)H * kHeadDim;
+  // chunked prefill: q holds the last positions only; query blocks before the chunk are skipped (projected as zeros)
+  const int q_first = (m.chunked && is_q) ? m.qoff[b] : 0;
+  const int q_shift = (m.chunked && is_q) ? m.qdelta[b] : 0;
+  if (i0 + nblk <= q_first) return;
 
   for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
     const int t0 = s0 + (i0 + bi) * m.block;
-    const int cnt = min(m.block, s1 - t0);
-    const uint16_t* base = x + (size_t)t0 * row_stride + (size_t)h * kHeadDim + cchunk * 8;
+    const int cnt = (i0 + bi < q_first) ? 0 : min(m.block, s1 - t0);
+    const uint16_t* base = x + ((ptrdiff_t)t0 + q_shift) * (ptrdiff_t)row_stride + (size_t)h * kHeadDim + cchunk * 8;
     float a[8], hi[8], lo[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) { a[j] = 0.f; hi[j] = -CUDART_INF_F; lo[j] = CUDART_INF_F; }
@@ -205,12 +213,13 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
         if (live[j]) { max_bf16x8(hi, u[j]); min_bf16x8(lo, u[j]); }   // rows past the end of the sequence take no part
       }
     }
-    const float inv = 1.0f / (float)cnt;
+    const float inv = cnt > 0 ? 1.0f / (float)cnt : 0.f;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       a[j] = (a[j] + __shfl_xor_sync(0xffffffffu, a[j], 16)) * inv;
       hi[j] = fmaxf(hi[j], __shfl_xor_sync(0xffffffffu, hi[j], 16));
       lo[j] = fminf(lo[j], __shfl_xor_sync(0xffffffffu, lo[j], 16));
+      if (cnt == 0) { hi[j] = 0.f; lo[j] = 0.f; }      // a skipped block: zeros, not the identities of max and min
     }
     if (half == 0) {
       if (methods & SEER_POOL_AVG) {
@@ -322,6 +331,7 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
   const int i0 = (tile_g - m.tile_off[b]) * kScoreTile;
   const int rows_valid = min(kScoreTile, nb - i0);
+  if (m.chunked && i0 + rows_valid <= m.qoff[b]) return;   // chunked prefill: a tile of query blocks before the chunk
   const size_t plane_q = (size_t)m.num_q_heads * m.total_blocks * kGateDim;
   const size_t plane_k = (size_t)m.num_kv_heads * m.total_blocks * kGateDim;
   const uint16_t* gq_h = gq + ((size_t)h * m.total_blocks + m.blk_off[b]) * kGateDim;
@@ -559,6 +569,7 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   ShapeTotals t;
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
+  if (shape->cu_seqlens_q_host) return SEER_ERR_UNSUPPORTED;   // no chunked prefill through the built-in scratch
   if (t.total_blocks == 0) return SEER_OK;
   if (!q || !k || !Wq || !Wk || !scores) return SEER_ERR_INVALID_ARG;
   // sizes beyond the built-in scratch are refused, never truncated
@@ -608,6 +619,8 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   m.score_elems = t.score_elems;
   m.softmax_scale = 0.f;   // unused by the gate
   m.block = shape->block;
+  m.qoff = nullptr; m.qdelta = nullptr; m.chunked = 0;
+  m.total_q_tokens = (int32_t)t.total_tokens;
   // The two kernels below are the ones seer_gate_scores launches; only the scratch pointer differs.  Nothing in the
   // scratch has to start at zero: the first kernel writes every projected vector the second one reads.
   const int n = launch_gate(nullptr, m, q, k, Wq, Wk, scores, base + kStaticMetaBytes, stream);

@@ -17,6 +17,7 @@ struct RowInfo {
   const float* s;   // scores of this row
   int i;            // query block index (row has n = i + 1 causal blocks)
   bool valid;
+  bool skip;        // chunked prefill: a query block before the chunk, its list is empty
 };
 
 // Rows [row_lo, row_hi) of the CSR structure whose scores sit at (offset in the full matrix - score_base) in `scores`.
@@ -27,6 +28,7 @@ struct RowBand {
 __device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const RowBand& band, const float* __restrict__ scores, int64_t r) {
   RowInfo ri;
   ri.valid = r < band.row_hi;
+  ri.skip = false;
   if (!ri.valid) { ri.s = nullptr; ri.i = 0; return ri; }
   const int b = find_sequence(m.blk_off, m.batch, (int)(r / m.num_q_heads));
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
@@ -34,6 +36,7 @@ __device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const RowBand& b
   const int h = (int)(local / nb);
   ri.i = (int)(local - (int64_t)h * nb);
   ri.s = scores + (m.score_off[b] + ((int64_t)h * nb + ri.i) * nb - band.score_base);
+  ri.skip = m.chunked && ri.i < m.qoff[b];
   return ri;
 }
 
@@ -80,7 +83,9 @@ count_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mas
   if (!ri.valid) return;
   const int n = ri.i + 1;
   int c = 0;
-  if (p.mode == SEER_THRESHOLD) {
+  if (ri.skip) {
+    // nothing listed
+  } else if (p.mode == SEER_THRESHOLD) {
     for (int j = lane; j < n; j += 32) c += (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold) ? 1 : 0;
     c = warp_sum(c);
   } else {
@@ -163,7 +168,7 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t r = band.row_lo + (int64_t)blockIdx.x * kMaskWarps + warp;
   const RowInfo ri = decode_row(m, band, scores, r);
-  if (!ri.valid) return;
+  if (!ri.valid || ri.skip) return;
   const int n = ri.i + 1;
   const int32_t out0 = row_ptr[r], out1 = row_ptr[r + 1];
   if ((int64_t)out1 > col_capacity) return;   // this row (and all later ones) do not fit; status already raised

@@ -13,7 +13,9 @@ constexpr size_t kOffBlk = kOffCu + sizeof(int32_t) * (kMaxBatch + 1 + 3);
 constexpr size_t kOffChunk = kOffBlk + sizeof(int32_t) * (kMaxBatch + 1 + 3);
 constexpr size_t kOffTile = kOffChunk + sizeof(int32_t) * (kMaxBatch + 1 + 3);
 constexpr size_t kOffScore = kOffTile + sizeof(int32_t) * (kMaxBatch + 1 + 3);
-constexpr size_t kSlotBytes = kOffScore + sizeof(int64_t) * (kMaxBatch + 1);
+constexpr size_t kOffQoff = kOffScore + sizeof(int64_t) * (kMaxBatch + 1);
+constexpr size_t kOffQdelta = kOffQoff + sizeof(int32_t) * (kMaxBatch + 4);
+constexpr size_t kSlotBytes = kOffQdelta + sizeof(int32_t) * (kMaxBatch + 4);
 
 seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
   if (!s || !s->cu_seqlens_host || s->batch < 1) return SEER_ERR_INVALID_ARG;
@@ -24,6 +26,16 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
   if (s->num_q_heads % s->num_kv_heads != 0) return SEER_ERR_UNSUPPORTED;
   const int32_t* cu = s->cu_seqlens_host;
   if (cu[0] != 0) return SEER_ERR_INVALID_ARG;
+  if (const int32_t* cq = s->cu_seqlens_q_host) {
+    // the queries are the last positions of each sequence and start on a block boundary
+    if (cq[0] != 0) return SEER_ERR_INVALID_ARG;
+    for (int b = 0; b < s->batch; ++b) {
+      if (cu[b + 1] < cu[b]) return SEER_ERR_INVALID_ARG;
+      const int64_t sq = (int64_t)cq[b + 1] - cq[b], sk = (int64_t)cu[b + 1] - cu[b];
+      if (sq < 0 || sq > sk) return SEER_ERR_INVALID_ARG;
+      if (sq > 0 && (sk - sq) % s->block != 0) return SEER_ERR_UNSUPPORTED;
+    }
+  }
   int64_t blocks = 0, chunks = 0, tiles = 0, sq = 0, causal = 0;
   int32_t max_nb = 0;
   for (int b = 0; b < s->batch; ++b) {
@@ -37,6 +49,7 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
     if (nb > max_nb) max_nb = (int32_t)nb;
   }
   t->total_tokens = cu[s->batch];
+  t->total_q_tokens = s->cu_seqlens_q_host ? s->cu_seqlens_q_host[s->batch] : cu[s->batch];
   t->total_blocks = blocks;
   t->total_chunks = chunks;
   t->total_tiles = tiles;
@@ -68,6 +81,7 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   std::vector<int32_t> key(shape->cu_seqlens_host, shape->cu_seqlens_host + n);
   key.push_back(shape->num_q_heads);
   key.push_back(shape->block);
+  if (shape->cu_seqlens_q_host) key.insert(key.end(), shape->cu_seqlens_q_host, shape->cu_seqlens_q_host + n);
   int slot = -1;
   for (int i = 0; i < kMetaSlots; ++i)
     if (ctx->slots[i].key == key) { slot = i; break; }
@@ -85,6 +99,8 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
     int32_t* chk = (int32_t*)(h + kOffChunk);
     int32_t* til = (int32_t*)(h + kOffTile);
     int64_t* sc = (int64_t*)(h + kOffScore);
+    int32_t* qo = (int32_t*)(h + kOffQoff);
+    int32_t* qd = (int32_t*)(h + kOffQdelta);
     blk[0] = 0; chk[0] = 0; til[0] = 0; sc[0] = 0;
     for (int b = 0; b < shape->batch; ++b) {
       cu[b] = shape->cu_seqlens_host[b];
@@ -93,6 +109,12 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
       chk[b + 1] = chk[b] + (nb + kPoolChunk - 1) / kPoolChunk;
       til[b + 1] = til[b] + (nb + kScoreTile - 1) / kScoreTile;
       sc[b + 1] = sc[b] + (int64_t)shape->num_q_heads * nb * nb;
+      qo[b] = 0; qd[b] = 0;
+      if (const int32_t* cq = shape->cu_seqlens_q_host) {
+        const int32_t sq = cq[b + 1] - cq[b], sk = shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b];
+        qo[b] = sq > 0 ? (sk - sq) / shape->block : nb;          // no queries: past the last block
+        qd[b] = cq[b] - (shape->cu_seqlens_host[b] + (sk - sq));  // first query token <-> key token cu[b] + sk - sq
+      }
     }
     cu[shape->batch] = shape->cu_seqlens_host[shape->batch];
     if (cudaMemcpyAsync(s.dev, s.pinned, kSlotBytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SEER_ERR_CUDA;
@@ -123,6 +145,10 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   m->score_elems = t.score_elems;
   m->softmax_scale = shape->softmax_scale > 0.f ? shape->softmax_scale : 0.08838834764831845f;  // 1/sqrt(128)
   m->block = shape->block;
+  m->qoff = (const int32_t*)(d + kOffQoff);
+  m->qdelta = (const int32_t*)(d + kOffQdelta);
+  m->total_q_tokens = (int32_t)t.total_q_tokens;
+  m->chunked = shape->cu_seqlens_q_host ? 1 : 0;
   *slot_out = slot;
   return SEER_OK;
 }
@@ -575,7 +601,7 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
   ShapeTotals full, t;
   seer_status st = shape_totals(shape, &full);
   if (st != SEER_OK) return st;
-  if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;
+  if (shape->block != kBlock || shape->cu_seqlens_q_host) return SEER_ERR_UNSUPPORTED;
   if (full.total_blocks == 0) return SEER_OK;
   if (!q_host || !k_host || !v_host || !Wq_host || !Wk_host || !o_host) return SEER_ERR_INVALID_ARG;
   seer_shape slice;

@@ -38,6 +38,11 @@ struct SeqMeta {
   int64_t score_elems;
   float softmax_scale;
   int32_t block;               // tokens per gate block: 64, or 128 (gate and mask only)
+  // chunked prefill (all zero without a chunk): the queries of sequence b are its last positions
+  const int32_t* qoff;         // [batch] block position of the chunk's first query block
+  const int32_t* qdelta;       // [batch] token index in q / o / lse = token index in k / v + qdelta
+  int32_t total_q_tokens;      // tokens in q / o / lse
+  int32_t chunked;             // 1 if the shape carries cu_seqlens_q
 };
 
 // A rectangle of (64-row score tile, query head) pairs whose scores are produced and consumed together; tiles are
@@ -85,7 +90,7 @@ void finish_call(seer_ctx* ctx, int slot, cudaStream_t stream);
 
 // Host-only shape arithmetic (no CUDA calls): returns SEER_OK and fills totals.
 struct ShapeTotals {
-  int64_t total_tokens, total_blocks, total_chunks, total_tiles, rows, score_elems, causal_blocks;
+  int64_t total_tokens, total_q_tokens, total_blocks, total_chunks, total_tiles, rows, score_elems, causal_blocks;
   int32_t max_nb;
 };
 seer_status shape_totals(const seer_shape* shape, ShapeTotals* t);

@@ -21,7 +21,7 @@ def _bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:
 class Prefill:
     def __init__(self, cu_seqlens, num_q_heads: int, num_kv_heads: int, *, device: int = 0,
                  ctx: Optional[B.Context] = None, softmax_scale: float = 0.0, col_capacity: Optional[int] = None,
-                 want_lse: bool = True, block: int = 64):
+                 want_lse: bool = True, block: int = 64, cu_seqlens_q=None):
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         self.device = torch.device("cuda", device)
@@ -30,11 +30,16 @@ class Prefill:
         self.cu = np.asarray(cu_seqlens, dtype=np.int32)
         self.hq, self.hkv = num_q_heads, num_kv_heads
         self.block = block
-        self.shape = B.make_shape(self.cu, num_q_heads, num_kv_heads, softmax_scale=softmax_scale, block=block)
+        # chunked prefill: q / o / lse hold the last cu_q[b+1] - cu_q[b] positions of each sequence only
+        self.cu_q = None if cu_seqlens_q is None else np.asarray(cu_seqlens_q, dtype=np.int32)
+        self.shape = B.make_shape(self.cu, num_q_heads, num_kv_heads, softmax_scale=softmax_scale, block=block,
+                                  cu_seqlens_q=self.cu_q)
         # the attention kernels tile by 64 tokens: 128-token lists are expanded for them (seer_expand_block_lists)
         self.attn_shape = self.shape if block == 64 else B.make_shape(self.cu, num_q_heads, num_kv_heads,
-                                                                      softmax_scale=softmax_scale, block=64)
+                                                                      softmax_scale=softmax_scale, block=64,
+                                                                      cu_seqlens_q=self.cu_q)
         self.T = int(self.cu[-1])
+        self.Tq = self.T if self.cu_q is None else int(self.cu_q[-1])
         self.rows = B.seer_mask_rows(self.shape)
         self.causal_blocks = B.seer_causal_blocks(self.shape)
         if self.rows < 0:
@@ -52,8 +57,8 @@ class Prefill:
             self.col_idx64 = torch.empty(max(4 * cap, 1), dtype=torch.int32, device=d)
             self.nnz64 = torch.zeros(1, dtype=torch.int64, device=d)
         self.q = self.k = self.v = self.wq = self.wk = None
-        self.o = torch.empty((self.T, num_q_heads, 128), dtype=torch.bfloat16, device=d)
-        self.lse = torch.empty((num_q_heads, self.T), dtype=torch.float32, device=d) if want_lse else None
+        self.o = torch.empty((self.Tq, num_q_heads, 128), dtype=torch.bfloat16, device=d)
+        self.lse = torch.empty((num_q_heads, self.Tq), dtype=torch.float32, device=d) if want_lse else None
 
     # ---- uploads (plain copies)
     def set_inputs(self, q_bits, k_bits, v_bits, wq=None, wk=None):

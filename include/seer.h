@@ -120,6 +120,8 @@ typedef struct {
   uint32_t flags;    /* SEER_FORCE_DIAG keeps block i, SEER_FORCE_SINK keeps block 0, in every row.  In the TopK modes
                         forced blocks count toward k_i; the other places go to the best remaining blocks ordered by
                         (score descending, block index ascending).  NaN scores are never selected. */
+  int32_t dense_tail_blocks; /* >= 0: the last dense_tail_blocks query blocks of every sequence keep all their causal
+                        blocks whatever their scores ("sparsity in the context, not in the question", Sec. 4) */
 } seer_mask_params;
 
 /* 2. Binary block mask (Sec. 3.3, Eq. 3 TopK / Eq. 4 threshold) as CSR index lists.

@@ -262,17 +262,22 @@ def select_row(score_row: np.ndarray, i: int, mode: int, *, keep_num=1, keep_den
     return sorted(forced | set(order[:take].tolist()))
 
 
-def block_mask(scores: list, mode: int, *, keep_num=1, keep_den=1, k=0, threshold=0.0, flags=FORCE_DIAG):
+def block_mask(scores: list, mode: int, *, keep_num=1, keep_den=1, k=0, threshold=0.0, flags=FORCE_DIAG, dense_tail=0):
     """All rows of all sequences -> CSR index lists (row_ptr int64 [R+1], col_idx int32 [nnz]).
-    `scores` is the per-sequence list of [Hq, nb, nb] fp32 arrays."""
+    `scores` is the per-sequence list of [Hq, nb, nb] fp32 arrays.  dense_tail: the last `dense_tail` query blocks
+    of every sequence keep all their causal blocks (Sec. 4: sparsity is applied to the context, not to the question
+    that ends the prompt)."""
     row_ptr = [0]
     cols = []
     for S in scores:
         Hq, nb, _ = S.shape
         for h in range(Hq):
             for i in range(nb):
-                lst = select_row(S[h, i], i, mode, keep_num=keep_num, keep_den=keep_den, k=k,
-                                 threshold=threshold, flags=flags)
+                if i >= nb - dense_tail:
+                    lst = list(range(i + 1))
+                else:
+                    lst = select_row(S[h, i], i, mode, keep_num=keep_num, keep_den=keep_den, k=k,
+                                     threshold=threshold, flags=flags)
                 cols.extend(lst)
                 row_ptr.append(len(cols))
     return np.asarray(row_ptr, dtype=np.int64), np.asarray(cols, dtype=np.int32)
@@ -376,7 +381,8 @@ def gate_scores_chunk(q_bits, k_bits, wq, wk, cu_seqlens_q, cu_seqlens_k, B: int
     return out
 
 
-def block_mask_chunk(scores: list, mode: int, *, keep_num=1, keep_den=1, k=0, threshold=0.0, flags=FORCE_DIAG):
+def block_mask_chunk(scores: list, mode: int, *, keep_num=1, keep_den=1, k=0, threshold=0.0, flags=FORCE_DIAG,
+                     dense_tail=0):
     """Lists for a chunk from its [Hq, nbq, nbk] score arrays, in the row numbering of the whole sequences: the CSR
     structure has Hq * nbk rows per sequence and the rows of the blocks before the chunk are empty."""
     row_ptr, cols = [0], []
@@ -385,7 +391,9 @@ def block_mask_chunk(scores: list, mode: int, *, keep_num=1, keep_den=1, k=0, th
         off = nbk - nbq
         for h in range(Hq):
             for i in range(nbk):
-                if i >= off:
+                if i >= off and i >= nbk - dense_tail:
+                    cols.extend(range(i + 1))
+                elif i >= off:
                     cols.extend(select_row(S[h, i - off], i, mode, keep_num=keep_num, keep_den=keep_den, k=k,
                                            threshold=threshold, flags=flags))
                 row_ptr.append(len(cols))

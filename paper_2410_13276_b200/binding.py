@@ -46,7 +46,7 @@ class seer_shape(C.Structure):
 
 class seer_mask_params(C.Structure):
     _fields_ = [("mode", C.c_int32), ("keep_num", C.c_int32), ("keep_den", C.c_int32), ("k", C.c_int32),
-                ("threshold", C.c_float), ("flags", C.c_uint32)]
+                ("threshold", C.c_float), ("flags", C.c_uint32), ("dense_tail_blocks", C.c_int32)]
 
 
 class seer_gate_options(C.Structure):
@@ -153,8 +153,8 @@ def make_shape(cu_seqlens: Sequence[int], num_q_heads: int, num_kv_heads: int, *
 
 
 def make_mask_params(mode: int, *, keep_num: int = 1, keep_den: int = 1, k: int = 0, threshold: float = 0.0,
-                     flags: int = SEER_FORCE_DIAG) -> seer_mask_params:
-    return seer_mask_params(mode, keep_num, keep_den, k, threshold, flags)
+                     flags: int = SEER_FORCE_DIAG, dense_tail: int = 0) -> seer_mask_params:
+    return seer_mask_params(mode, keep_num, keep_den, k, threshold, flags, dense_tail)
 
 
 def seer_workspace_bytes(shape: seer_shape) -> int:

@@ -18,6 +18,7 @@ struct RowInfo {
   int i;            // query block index (row has n = i + 1 causal blocks)
   bool valid;
   bool skip;        // chunked prefill: a query block before the chunk, its list is empty
+  int nb;           // blocks of the row's sequence
 };
 
 // Rows [row_lo, row_hi) of the CSR structure whose scores sit at (offset in the full matrix - score_base) in `scores`.
@@ -29,6 +30,7 @@ __device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const RowBand& b
   RowInfo ri;
   ri.valid = r < band.row_hi;
   ri.skip = false;
+  ri.nb = 0;
   if (!ri.valid) { ri.s = nullptr; ri.i = 0; return ri; }
   const int b = find_sequence(m.blk_off, m.batch, (int)(r / m.num_q_heads));
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
@@ -37,6 +39,7 @@ __device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const RowBand& b
   ri.i = (int)(local - (int64_t)h * nb);
   ri.s = scores + (m.score_off[b] + ((int64_t)h * nb + ri.i) * nb - band.score_base);
   ri.skip = m.chunked && ri.i < m.qoff[b];
+  ri.nb = nb;
   return ri;
 }
 
@@ -85,6 +88,8 @@ count_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mas
   int c = 0;
   if (ri.skip) {
     // nothing listed
+  } else if (ri.i >= ri.nb - p.dense_tail_blocks) {
+    c = n;                                             // a dense row at the end of the sequence
   } else if (p.mode == SEER_THRESHOLD) {
     for (int j = lane; j < n; j += 32) c += (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold) ? 1 : 0;
     c = warp_sum(c);
@@ -175,6 +180,10 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   int32_t* __restrict__ out = col_idx + out0;
   const uint32_t lt_mask = (1u << lane) - 1u;
 
+  if (ri.i >= ri.nb - p.dense_tail_blocks) {           // a dense row at the end of the sequence: every causal block
+    for (int j = lane; j < n; j += 32) out[j] = j;
+    return;
+  }
   if (p.mode == SEER_THRESHOLD) {
     int written = 0;
     for (int base = 0; base < n; base += 32) {

@@ -320,6 +320,7 @@ seer_status seer_block_mask(seer_ctx* ctx, const seer_shape* shape, const float*
   if (p->mode != SEER_TOPK_RATIO && p->mode != SEER_TOPK_COUNT && p->mode != SEER_THRESHOLD) return SEER_ERR_INVALID_ARG;
   if (p->mode == SEER_TOPK_RATIO && (p->keep_num < 0 || p->keep_den < 1)) return SEER_ERR_INVALID_ARG;
   if (p->flags & ~(uint32_t)(SEER_FORCE_DIAG | SEER_FORCE_SINK)) return SEER_ERR_INVALID_ARG;
+  if (p->dense_tail_blocks < 0) return SEER_ERR_INVALID_ARG;
   if (t.total_blocks > 0 && !scores) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
@@ -407,6 +408,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
   if (p->mode != SEER_TOPK_RATIO && p->mode != SEER_TOPK_COUNT && p->mode != SEER_THRESHOLD) return SEER_ERR_INVALID_ARG;
   if (p->mode == SEER_TOPK_RATIO && (p->keep_num < 0 || p->keep_den < 1)) return SEER_ERR_INVALID_ARG;
   if (p->flags & ~(uint32_t)(SEER_FORCE_DIAG | SEER_FORCE_SINK)) return SEER_ERR_INVALID_ARG;
+  if (p->dense_tail_blocks < 0) return SEER_ERR_INVALID_ARG;
   if (t.total_blocks > 0 && (!q || !k || !Wq || !Wk)) return SEER_ERR_INVALID_ARG;
   const size_t gate_bytes = gate_workspace_bytes(t, shape);
   if (t.total_blocks > 0 && !ws_ok(ws, ws_bytes, gate_bytes + min_band_bytes(t))) return SEER_ERR_WORKSPACE;

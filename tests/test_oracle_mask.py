@@ -134,3 +134,28 @@ def test_block_mask_csr_layout_and_row_ids():
     assert counts.tolist() == want
     fp, fc = O.full_causal_lists([0, 5, 12], 4, 2)
     assert np.diff(fp).tolist() == [1, 2, 1, 2, 1, 2, 1, 2] and fc[:3].tolist() == [0, 0, 1]
+
+
+def test_dense_tail_keeps_the_last_query_blocks_whole():
+    """Sec. 4: sparsity in the context, dense on the question.  Closed forms: the last `dense_tail` rows of every
+    (sequence, head) list all their causal blocks, the other rows are untouched; a tail as long as the sequence gives
+    the full causal lists; a tail of zero changes nothing."""
+    rng = np.random.default_rng(7)
+    scores = [random_scores(rng, 6, hq=2), random_scores(rng, 2, hq=2), random_scores(rng, 9, hq=2)]
+    base_rp, base_col = O.block_mask(scores, COUNT, k=2, flags=DIAG)
+    rp0, col0 = O.block_mask(scores, COUNT, k=2, flags=DIAG, dense_tail=0)
+    assert np.array_equal(rp0, base_rp) and np.array_equal(col0, base_col)
+    rp, col = O.block_mask(scores, COUNT, k=2, flags=DIAG, dense_tail=3)
+    r = 0
+    for nb in (6, 2, 9):
+        for _h in range(2):
+            for i in range(nb):
+                got = col[rp[r]:rp[r + 1]].tolist()
+                if i >= nb - 3:
+                    assert got == list(range(i + 1))
+                else:
+                    assert got == base_col[base_rp[r]:base_rp[r + 1]].tolist()
+                r += 1
+    frp, fcol = O.block_mask(scores, THR, threshold=2.0, flags=0, dense_tail=9)
+    wrp, wcol = O.full_causal_lists([0, 6 * 4, 8 * 4, 17 * 4], 4, 2)
+    assert np.array_equal(frp, wrp) and np.array_equal(fcol, wcol)

@@ -91,6 +91,8 @@ typedef struct {
  * score rows before the chunk are not written, their CSR rows are empty, and lists given for them are ignored by the
  * attention.  The results are those of the whole problem restricted to the chunk (same kernels, same arithmetic).
  * A score buffer of full size is only needed by the separate gate and mask calls; seer_gate_block_mask needs none.
+ * With no query at all (cu_q[batch] = 0) the gate and attention calls return SEER_OK without work (q, o, scores may be
+ * NULL) and the mask calls write empty rows.
  * Not supported with a chunk (SEER_ERR_UNSUPPORTED): seer_prefill_host, seer_gate_scores_static. */
 
 /* Sizing helpers (pure host arithmetic; return 0 / -1 on an invalid shape). */

@@ -270,7 +270,7 @@ seer_status seer_gate_scores(seer_ctx* ctx, const seer_shape* shape, const void*
   ShapeTotals t;
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
-  if (t.total_blocks == 0) return SEER_OK;
+  if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;   // no score row to write
   if (!q || !k || !Wq || !Wk || !scores) return SEER_ERR_INVALID_ARG;
   if (!ws_ok(ws, ws_bytes, gate_workspace_bytes(t, shape))) return SEER_ERR_WORKSPACE;
   SeqMeta m; int slot;
@@ -294,7 +294,7 @@ seer_status seer_gate_scores_ex(seer_ctx* ctx, const seer_shape* shape, const se
   ShapeTotals t;
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
-  if (t.total_blocks == 0) return SEER_OK;
+  if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;   // no score row to write
   if (!q || !k || !Wq || !Wk || !scores) return SEER_ERR_INVALID_ARG;
   if (!ws_ok(ws, ws_bytes, gate_workspace_bytes(t, shape))) return SEER_ERR_WORKSPACE;
   SeqMeta m; int slot;
@@ -342,7 +342,7 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
   if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;   // 128-token lists go through seer_expand_block_lists first
-  if (t.total_blocks == 0) return SEER_OK;
+  if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;   // no output row
   if (!q || !k || !v || !row_ptr || !o) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
@@ -364,7 +364,7 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
   if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;
-  if (t.total_blocks == 0) return SEER_OK;
+  if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;
   if (!q || !k || !row_ptr || !lse) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
@@ -409,7 +409,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
   if (p->mode == SEER_TOPK_RATIO && (p->keep_num < 0 || p->keep_den < 1)) return SEER_ERR_INVALID_ARG;
   if (p->flags & ~(uint32_t)(SEER_FORCE_DIAG | SEER_FORCE_SINK)) return SEER_ERR_INVALID_ARG;
   if (p->dense_tail_blocks < 0) return SEER_ERR_INVALID_ARG;
-  if (t.total_blocks > 0 && (!q || !k || !Wq || !Wk)) return SEER_ERR_INVALID_ARG;
+  if (t.total_blocks > 0 && ((!q && t.total_q_tokens > 0) || !k || !Wq || !Wk)) return SEER_ERR_INVALID_ARG;
   const size_t gate_bytes = gate_workspace_bytes(t, shape);
   if (t.total_blocks > 0 && !ws_ok(ws, ws_bytes, gate_bytes + min_band_bytes(t))) return SEER_ERR_WORKSPACE;
   SeqMeta m; int slot;

@@ -169,3 +169,59 @@ def test_chunk_shape_validation(rt):
     with pytest.raises(B.SeerError) as e:
         B.seer_gate_scores_static(s, buf, buf, buf, buf, buf)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_chunks_equal_rows_of_the_whole_run(rt, seed):
+    """Seeded random packed batches, chunk starts and mask modes: scores, lists, o and lse of the chunk equal the matching
+    rows of the GPU's whole-problem run exactly (that run is what the other tests hold against the oracle)."""
+    B, Prefill, ctx = rt
+    rng = np.random.default_rng(123_000 + seed)
+    blk = int(rng.choice([64, 64, 128]))
+    nseq = int(rng.integers(1, 4))
+    lens = [int(x) for x in rng.choice([1, 64, 65, 200, 333, 512, 700, 1300], size=nseq)]
+    starts = []
+    for S in lens:
+        nb = (S + blk - 1) // blk
+        c = int(rng.integers(0, nb + 1))                     # nb: the sequence contributes no query
+        starts.append(S if c == nb else c * blk)
+    hkv = int(rng.integers(1, 3)); hq = hkv * int(rng.choice([1, 2, 4]))
+    mode = int(rng.integers(0, 3))
+    params = B.make_mask_params(mode, keep_num=1, keep_den=int(rng.integers(2, 6)), k=int(rng.integers(0, 5)),
+                                threshold=float(rng.choice([0.0, 0.05, 0.3])), flags=int(rng.choice([0, 1, 3])),
+                                dense_tail=int(rng.choice([0, 0, 1])))
+    w = W.make_small(seed=124_000 + seed, seqlens=lens, hq=hq, hkv=hkv, q_gain=2.0, block=blk)
+    qc, cu_q = make_chunk(w, starts)
+    full = Prefill(w.cu_seqlens, hq, hkv, ctx=ctx, want_lse=True, block=blk)
+    full.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    full.run(params)
+    part = Prefill(w.cu_seqlens, hq, hkv, ctx=ctx, want_lse=True, block=blk, cu_seqlens_q=cu_q)
+    if qc.shape[0] == 0:
+        qc = np.zeros((1,) + w.q.shape[1:], np.uint16)       # a buffer to point at; no query is read
+    part.set_inputs(qc, w.k, w.v, w.wq, w.wk)
+    part.o.fill_(float("nan"))
+    part.run(params)
+    assert full.status() == 0 and part.status() == 0, (lens, starts, blk)
+    offs = O.chunk_offsets(cu_q, w.cu_seqlens, blk)
+    rp, col = part.lists_host()
+    rp_f, col_f = full.lists_host()
+    s_full = O.unflatten_scores(full.scores_host(), w.cu_seqlens, blk, hq)
+    s_part = O.unflatten_scores(part.scores_host(), w.cu_seqlens, blk, hq)
+    r = 0
+    for b, S in enumerate(lens):
+        nb = (S + blk - 1) // blk
+        for h in range(hq):
+            for i in range(nb):
+                if i >= int(offs[b]):
+                    assert np.array_equal(s_part[b][h, i, :i + 1], s_full[b][h, i, :i + 1]), (lens, starts, b, h, i)
+                    assert np.array_equal(col[rp[r]:rp[r + 1]], col_f[rp_f[r]:rp_f[r + 1]]), (lens, starts, b, h, i)
+                else:
+                    assert rp[r + 1] == rp[r]
+                r += 1
+    o_part, lse_part = part.o_host(), part.lse_host()
+    o_full, lse_full = full.o_host(), full.lse_host()
+    for b, st in enumerate(starts):
+        k0, k1 = int(w.cu_seqlens[b]), int(w.cu_seqlens[b + 1])
+        q0, q1 = int(cu_q[b]), int(cu_q[b + 1])
+        assert np.array_equal(o_part[q0:q1], o_full[k0 + st:k1]), (lens, starts, blk)
+        assert np.array_equal(lse_part[:, q0:q1], lse_full[:, k0 + st:k1])

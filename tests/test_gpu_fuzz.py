@@ -48,7 +48,7 @@ def draw_case(seed):
     return lens, hkv * group, hkv, kw, gain
 
 
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", range(48))
 def test_random_shape_whole_path(rt, seed):
     B, Prefill, ctx = rt
     lens, hq, hkv, kw, gain = draw_case(seed)

@@ -3,15 +3,19 @@
 //   scan_kernel  : exclusive prefix sum of the counts -> row_ptr, nnz, capacity check
 //   fill_kernel  : one warp per row repeats the selection and writes the ascending list by ballot compaction
 // Selection order in the TopK modes is (score descending, block index ascending): scores become order-preserving
-// 32-bit keys, the key of the last kept candidate is found by a radix select over the row held in shared memory (four
-// 8-bit passes with warp-private histograms; rows too long to stage fall back to a bitwise search that re-reads the
-// scores), and ties at that key are resolved by rank in index order.
+// 32-bit keys, the key of the last kept candidate is found by a radix select over the row held in shared memory (at most
+// four 8-bit passes with warp-private histograms; batches with rows too long to stage re-read the scores in every pass), and ties
+// at that key are resolved by rank in index order.
 #include "seer_internal.cuh"
 
 namespace seer {
 
 constexpr int kMaskWarps = 4;
-constexpr int kMaskSmemRowMax = 8192;   // rows up to this many blocks are staged in shared memory
+// Rows are staged in shared memory when the longest row of the batch has at most this many blocks (16 bytes of shared
+// memory per block and CTA).  Beyond that the staging buffer would cost more in occupancy than it saves in reads
+// (measured: 4096 blocks 4.6 ms staged, 3.1 ms not; 10240 blocks 103 ms against 27 ms), and every pass re-reads the
+// scores, which stay in L1 / L2 between the passes of a row.
+constexpr int kMaskSmemRowMax = 2048;
 
 struct RowInfo {
   const float* s;   // scores of this row
@@ -223,8 +227,8 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
     T = 0u; need_eq = 0;            // every candidate is kept (key >= 1 > 0)
   } else if (take == 0) {
     T = 0xffffffffu; need_eq = 0;   // nothing beyond the forced blocks
-  } else if (staged) {
-    // Radix select, 8 bits per pass from the top: histogram the current digit of the keys that match the prefix found
+  } else {
+    // Radix select, 8 bits per pass from the top (rows too long to stage re-read their scores in every pass): histogram the current digit of the keys that match the prefix found
     // so far (warp-private shared-memory bins), walk the bins from the largest digit down until `remaining` is covered.
     uint32_t* hist = hist_smem + warp * 256;
     // The scores of a row are often close together; the leading bits all candidate keys share need no pass: the passes
@@ -238,7 +242,7 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
       for (int b = lane; b < 256; b += 32) hist[b] = 0u;
       __syncwarp();
       for (int j = lane; j < n; j += 32) {
-        const uint32_t kk = keys[j];
+        const uint32_t kk = key_at(j);
         if (kk != 0u && (kk & prefix_mask) == prefix) atomicAdd(&hist[(kk >> shift) & 255u], 1u);
       }
       __syncwarp();
@@ -274,16 +278,6 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
     }
     T = prefix;                      // the take-th largest key; `remaining` of the keys equal to it are kept
     need_eq = remaining;
-  } else {
-    for (int bit = 31; bit >= 0; --bit) {
-      const uint32_t cand = T | (1u << bit);
-      int cnt = 0;
-      for (int j = lane; j < n; j += 32) cnt += key_at(j) >= cand;
-      if (warp_sum(cnt) >= take) T = cand;
-    }
-    int gt = 0;
-    for (int j = lane; j < n; j += 32) gt += key_at(j) > T;
-    need_eq = take - warp_sum(gt);
   }
   int written = 0, eq_seen = 0;
   for (int base = 0; base < n; base += 32) {
@@ -308,7 +302,7 @@ int launch_mask_band(seer_ctx* ctx, const SeqMeta& m, const float* scores, int64
   const unsigned grid = (unsigned)((row_hi - row_lo + kMaskWarps - 1) / kMaskWarps);
   count_kernel<<<grid, kMaskWarps * 32, 0, stream>>>(m, band, scores, p, row_ptr);
   scan_kernel<<<1, 1024, 0, stream>>>(row_hi - row_lo, row_ptr + row_lo, first ? 1 : 0, col_capacity, nnz_out, ctx->d_status);
-  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // longer rows re-read their scores instead
+  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // long rows re-read their scores instead
   const size_t smem = (size_t)kMaskWarps * (stage_cap + 256) * sizeof(uint32_t);
   fill_kernel<<<grid, kMaskWarps * 32, smem, stream>>>(m, band, scores, p, row_ptr, col_idx, col_capacity, stage_cap);
   cudaError_t e = cudaGetLastError();

@@ -353,3 +353,26 @@ def test_prefill_host_equals_the_three_calls(rt, cfg):
         assert torch.equal(ho.view(torch.bfloat16), o_ref)
         assert torch.equal(hl, lse_ref)
 
+
+
+@pytest.mark.parametrize("mode,kw", [(O.MODE_TOPK_RATIO, dict(keep_num=1, keep_den=7)), (O.MODE_TOPK_COUNT, dict(k=300)),
+                                     (O.MODE_THRESHOLD, dict(threshold=0.5))])
+def test_mask_without_row_staging(rt, mode, kw):
+    """When the longest row of a batch has more than 2048 blocks the mask builder does not stage rows in shared memory:
+    every radix pass re-reads the scores.  Synthetic scores with many exact ties (values on a grid of 1000 levels), lists
+    bit-exact against the oracle's selection on sampled rows, short and long."""
+    B, Prefill, ctx = rt
+    nb = 8300
+    p = Prefill([0, nb * 64], 1, 1, ctx=ctx, want_lse=False, col_capacity=nb * (nb + 1) // 2)
+    rng = np.random.default_rng(4711)
+    scores = (rng.integers(0, 1000, size=(nb, nb)).astype(np.float32) / np.float32(1000.0))
+    p.set_scores(scores.reshape(-1))
+    params = B.make_mask_params(mode, keep_num=kw.get("keep_num", 1), keep_den=kw.get("keep_den", 1), k=kw.get("k", 0),
+                                threshold=kw.get("threshold", 0.0), flags=3)
+    p.mask(params)
+    assert p.status() == 0
+    rp, col = p.lists_host()
+    assert rp[-1] == len(col) == int(p.nnz.item())
+    for i in [0, 1, 299, 300, 301, 4095, 8191, 8192, 8193, 8250, nb - 2, nb - 1]:
+        want = O.select_row(scores[i], i, mode, flags=3, **kw)
+        assert col[rp[i]:rp[i + 1]].tolist() == want, i

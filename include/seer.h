@@ -156,7 +156,11 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
                                 void* stream);
 
 /* Selects the attention kernel used by seer_sparse_attn: 0 = tcgen05 / TMEM / TMA kernel (default),
- * 1 = mma.sync kernel kept as an on-device cross-check.  Returns SEER_ERR_INVALID_ARG for other values. */
+ * 1 = mma.sync kernel (on-device cross-check; also the faster one for very short lists), 2 = chosen per call from
+ * the shape: the persistent tcgen05 kernel pays about 10 us per (head, query block) row whatever its list length, the
+ * mma.sync kernel about 3.5 us plus more per block, so batches whose rows have at most 8 causal blocks on average
+ * (many short sequences) go to the mma.sync kernel and everything else to the tcgen05 kernel (measured crossover:
+ * 8.5 listed blocks per row).  Returns SEER_ERR_INVALID_ARG for other values. */
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);
 
 /* Synchronises `stream`, returns the device status word (SEER_OK if nothing was raised) and clears it. */

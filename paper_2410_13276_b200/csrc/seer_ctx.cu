@@ -347,7 +347,10 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
   if (st != SEER_OK) return st;
-  int n = ctx->attn_impl == 1 ? launch_attn_mma(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
+  // impl 2: by shape.  The lists are at most the causal blocks; rows that short cost the persistent kernel more in
+  // per-row hand-over than the legacy kernel needs for the whole row.
+  const bool legacy = ctx->attn_impl == 1 || (ctx->attn_impl == 2 && t.causal_blocks <= 8 * t.rows);
+  int n = legacy ? launch_attn_mma(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
                               : launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream);
   finish_call(ctx, slot, stream);
   if (n < 0) return SEER_ERR_CUDA;
@@ -521,7 +524,7 @@ seer_status seer_expand_block_lists(seer_ctx* ctx, const seer_shape* shape, cons
 }
 
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl) {
-  if (!ctx || (impl != 0 && impl != 1)) return SEER_ERR_INVALID_ARG;
+  if (!ctx || impl < 0 || impl > 2) return SEER_ERR_INVALID_ARG;
   ctx->attn_impl = impl;
   return SEER_OK;
 }

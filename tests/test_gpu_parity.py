@@ -376,3 +376,30 @@ def test_mask_without_row_staging(rt, mode, kw):
     for i in [0, 1, 299, 300, 301, 4095, 8191, 8192, 8193, 8250, nb - 2, nb - 1]:
         want = O.select_row(scores[i], i, mode, flags=3, **kw)
         assert col[rp[i]:rp[i + 1]].tolist() == want, i
+
+
+def test_attention_kernel_chosen_by_shape(rt):
+    """seer_set_attn_impl(ctx, 2): batches of short sequences (at most 8 causal blocks per row on average) run the
+    mma.sync kernel, everything else the tcgen05 kernel; the output is exactly that of the kernel chosen."""
+    import torch
+    B, Prefill, ctx = rt
+    params = B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=1, flags=1)
+    try:
+        for lens, want in (([200] * 9 + [64, 1], 1), ([1100, 900], 0)):     # avg causal blocks per row 2.4 and 8.7
+            w = W.make_small(seed=31_000 + want, seqlens=lens, hq=4, hkv=2)
+            p = Prefill(w.cu_seqlens, 4, 2, ctx=ctx, want_lse=True)
+            p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+            p.gate(); p.mask(params)
+            outs = {}
+            for impl in (0, 1, 2):
+                B.seer_set_attn_impl(ctx, impl)
+                p.o.fill_(float("nan"))
+                p.attn()
+                assert p.status() == 0
+                outs[impl] = (p.o.clone(), p.lse.clone())
+            assert torch.equal(outs[2][0], outs[want][0]) and torch.equal(outs[2][1], outs[want][1])
+            assert not torch.equal(outs[0][0], outs[1][0])                  # the two kernels round differently
+        with pytest.raises(B.SeerError):
+            B.seer_set_attn_impl(ctx, 3)
+    finally:
+        B.seer_set_attn_impl(ctx, 0)

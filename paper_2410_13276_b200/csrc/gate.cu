@@ -48,7 +48,8 @@ __device__ __forceinline__ void acc_bf16x8(float (&a)[8], const uint4& u) {
 }
 
 // grid.x = total_chunks * (Hq + Hkv); the head varies fastest so that CTAs running together read
-// neighbouring 256-byte segments of the same token rows.
+// neighbouring 256-byte segments of the same token rows.  A chunk is 16 consecutive blocks of the packed batch, whatever
+// sequences they belong to (a chunk per sequence would leave most of a CTA idle on batches of short sequences).
 __global__ void __launch_bounds__(kPoolThreads)
 pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                     const float* __restrict__ Wq, const float* __restrict__ Wk, uint16_t* __restrict__ gq,
@@ -66,23 +67,24 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
   uint16_t* __restrict__ out = is_q ? gq : gk;
   const size_t plane = (size_t)H * m.total_blocks * kGateDim;   // elements between the hi / mid / lo planes
 
-  const int b = find_sequence(m.chunk_off, m.batch, chunk);
-  const int s0 = m.cu_seqlens[b], s1 = m.cu_seqlens[b + 1];
-  const int nb = m.blk_off[b + 1] - m.blk_off[b];
-  const int i0 = (chunk - m.chunk_off[b]) * kPoolChunk;
-  const int nblk = min(kPoolChunk, nb - i0);
+  const int g0 = chunk * kPoolChunk;                            // first block of the chunk, numbered over the batch
+  const int nblk = min(kPoolChunk, m.total_blocks - g0);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int half = lane >> 4, cchunk = lane & 15;
   const size_t row_stride = (size_t)H * kHeadDim;  // elements between consecutive tokens
-  // chunked prefill: q holds the last positions only; query blocks before the chunk are skipped (projected as zeros)
-  const int q_first = (m.chunked && is_q) ? m.qoff[b] : 0;
-  const int q_shift = (m.chunked && is_q) ? m.qdelta[b] : 0;
-  if (i0 + nblk <= q_first) return;
+  bool any = false;
 
   for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
-    const int t0 = s0 + (i0 + bi) * m.block;
-    const int cnt = (i0 + bi < q_first) ? 0 : min(m.block, s1 - t0);
+    const int b = find_sequence(m.blk_off, m.batch, g0 + bi);
+    const int i = g0 + bi - m.blk_off[b];
+    const int s0 = m.cu_seqlens[b], s1 = m.cu_seqlens[b + 1];
+    // chunked prefill: q holds the last positions only; query blocks before the chunk are skipped (projected as zeros)
+    const int q_first = (m.chunked && is_q) ? m.qoff[b] : 0;
+    const int q_shift = (m.chunked && is_q) ? m.qdelta[b] : 0;
+    const int t0 = s0 + i * m.block;
+    const int cnt = (i < q_first) ? 0 : min(m.block, s1 - t0);
+    any |= cnt > 0;
     const uint16_t* base = x + ((ptrdiff_t)t0 + q_shift) * (ptrdiff_t)row_stride + (size_t)h * kHeadDim + cchunk * 8;
     float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
@@ -108,7 +110,7 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
       dst[1] = make_float4(a[4], a[5], a[6], a[7]);
     }
   }
-  __syncthreads();
+  if (!__syncthreads_or(any ? 1 : 0)) return;                   // every block of the chunk lies before its queries
 
   // projection: thread -> output column o, 8 of the 16 blocks
   const int o = threadIdx.x & (kGateDim - 1);
@@ -120,7 +122,7 @@ pool_project_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* _
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = fmaf(pooled[grp * 8 + j][c], w, acc[j]);
   }
-  const size_t obase = ((size_t)h * m.total_blocks + m.blk_off[b] + i0) * kGateDim;
+  const size_t obase = ((size_t)h * m.total_blocks + g0) * kGateDim;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const int bi = grp * 8 + j;
@@ -150,13 +152,13 @@ __device__ __forceinline__ void min_bf16x8(float (&a)[8], const uint4& u) {
   a[6] = fminf(a[6], __uint_as_float(u.w << 16)); a[7] = fminf(a[7], __uint_as_float(u.w & 0xffff0000u));
 }
 
-constexpr int kPoolExSmem = kPoolChunk * 3 * kHeadDim * (int)sizeof(float);   // 24 KB: [16 blocks][up to 3 parts][128]
 
 __global__ void __launch_bounds__(kPoolThreads)
 pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                        const float* __restrict__ Wq, const float* __restrict__ Wk, uint16_t* __restrict__ gq,
                        uint16_t* __restrict__ gk, uint32_t pool_q, uint32_t pool_k, float rope_theta) {
   __shared__ __align__(16) float pooled[kPoolChunk][3 * kHeadDim];
+  __shared__ int block_pos[kPoolChunk];                        // position of each block in its sequence (block RoPE)
 
   const int heads_total = m.num_q_heads + m.num_kv_heads;
   const int chunk = blockIdx.x / heads_total;
@@ -176,23 +178,25 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
   const int off_max = (methods & SEER_POOL_AVG) ? kHeadDim : 0;
   const int off_min = off_max + ((methods & SEER_POOL_MAX) ? kHeadDim : 0);
 
-  const int b = find_sequence(m.chunk_off, m.batch, chunk);
-  const int s0 = m.cu_seqlens[b], s1 = m.cu_seqlens[b + 1];
-  const int nb = m.blk_off[b + 1] - m.blk_off[b];
-  const int i0 = (chunk - m.chunk_off[b]) * kPoolChunk;
-  const int nblk = min(kPoolChunk, nb - i0);
+  const int g0 = chunk * kPoolChunk;                            // first block of the chunk, numbered over the batch
+  const int nblk = min(kPoolChunk, m.total_blocks - g0);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int half = lane >> 4, cchunk = lane & 15;
   const size_t row_stride = (size_t)H * kHeadDim;
-  // chunked prefill: q holds the last positions only; query blocks before the chunk are skipped (projected as zeros)
-  const int q_first = (m.chunked && is_q) ? m.qoff[b] : 0;
-  const int q_shift = (m.chunked && is_q) ? m.qdelta[b] : 0;
-  if (i0 + nblk <= q_first) return;
+  bool any = false;
 
   for (int bi = warp; bi < nblk; bi += kPoolThreads / 32) {
-    const int t0 = s0 + (i0 + bi) * m.block;
-    const int cnt = (i0 + bi < q_first) ? 0 : min(m.block, s1 - t0);
+    const int b = find_sequence(m.blk_off, m.batch, g0 + bi);
+    const int i = g0 + bi - m.blk_off[b];
+    const int s0 = m.cu_seqlens[b], s1 = m.cu_seqlens[b + 1];
+    // chunked prefill: q holds the last positions only; query blocks before the chunk are skipped (projected as zeros)
+    const int q_first = (m.chunked && is_q) ? m.qoff[b] : 0;
+    const int q_shift = (m.chunked && is_q) ? m.qdelta[b] : 0;
+    const int t0 = s0 + i * m.block;
+    const int cnt = (i < q_first) ? 0 : min(m.block, s1 - t0);
+    any |= cnt > 0;
+    if (lane == 0) block_pos[bi] = i;
     const uint16_t* base = x + ((ptrdiff_t)t0 + q_shift) * (ptrdiff_t)row_stride + (size_t)h * kHeadDim + cchunk * 8;
     float a[8], hi[8], lo[8];
 #pragma unroll
@@ -236,7 +240,7 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
       }
     }
   }
-  __syncthreads();
+  if (!__syncthreads_or(any ? 1 : 0)) return;                   // every block of the chunk lies before its queries
 
   // projection: thread -> output column o, 8 of the 16 blocks
   const int o = threadIdx.x & (kGateDim - 1);
@@ -260,14 +264,14 @@ pool_project_ex_kernel(SeqMeta m, const uint16_t* __restrict__ q, const uint16_t
     for (int j = 0; j < 8; ++j) {
       const int bi = grp * 8 + j;
       double sn, cs;
-      sincos((double)(i0 + bi) * freq, &sn, &cs);
+      sincos((double)(bi < nblk ? block_pos[bi] : 0) * freq, &sn, &cs);
       const float partner = pooled[bi][o ^ (kGateDim / 2)];
       // first half: x1 cos - x2 sin; second half: x2 cos + x1 sin
       acc[j] = (o < kGateDim / 2) ? (float)((double)acc[j] * cs - (double)partner * sn)
                                   : (float)((double)acc[j] * cs + (double)partner * sn);
     }
   }
-  const size_t obase = ((size_t)h * m.total_blocks + m.blk_off[b] + i0) * kGateDim;
+  const size_t obase = ((size_t)h * m.total_blocks + g0) * kGateDim;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const int bi = grp * 8 + j;
@@ -311,9 +315,13 @@ __device__ __forceinline__ void gs_load_planes(uint32_t dst, const uint16_t* __r
   }
 }
 
-// grid.x = band.tiles * band.heads (head fastest; tiles are visited from the last rows, the longest, to the first).  The
-// band is a rectangle of (64-row score tile, query head) pairs; the whole problem is the band (0, total_tiles, 0, Hq, 0).
-// Scores of the band are written at their offset in the full matrix minus band.score_base.
+// grid.x = tiles * band.heads (head fastest; tiles are visited from the last rows to the first).  A tile is 64
+// consecutive block rows of the packed batch, counted from band.blk_lo, whatever sequences they belong to (a tile per
+// sequence would leave most of a CTA idle on batches of short sequences): row r of the tile is query block i_r of
+// sequence b_r, its causal columns are that sequence's blocks 0..i_r, i.e. the blocks seq_start_r .. r of the batch.  The
+// CTA walks the column tiles from the sequence start of its first row to its last row; entries of other sequences are
+// masked.  The whole problem is the band (0, total_blocks, 0, Hq, 0).  Scores are written at their offset in the full
+// matrix minus band.score_base.
 __global__ void __launch_bounds__(kScoreThreads)
 gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, const uint16_t* __restrict__ gk,
                    float* __restrict__ scores) {
@@ -323,33 +331,58 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
   float* row_l = row_m + kScoreTile;                                      // [64]
   float* part_m = row_l + kScoreTile;                                     // [2 column halves][64]
   float* part_l = part_m + 2 * kScoreTile;
+  __shared__ int row_start[kScoreTile];        // first block of the row's sequence, numbered over the batch
+  __shared__ int row_last[kScoreTile];         // the row's own block (its last causal column); -1: nothing to compute
+  __shared__ long long row_off[kScoreTile];    // element offset of the row's scores (column 0) in the buffer
 
-  const int tile_g = band.tile_lo + band.tiles - 1 - (int)(blockIdx.x / band.heads);
+  const int tiles = (band.blk_hi - band.blk_lo + kScoreTile - 1) / kScoreTile;
+  const int tile = tiles - 1 - (int)(blockIdx.x / band.heads);
   const int h = band.head_lo + (int)(blockIdx.x % band.heads);
   const int g = h / m.group;
-  const int b = find_sequence(m.tile_off, m.batch, tile_g);
-  const int nb = m.blk_off[b + 1] - m.blk_off[b];
-  const int i0 = (tile_g - m.tile_off[b]) * kScoreTile;
-  const int rows_valid = min(kScoreTile, nb - i0);
-  if (m.chunked && i0 + rows_valid <= m.qoff[b]) return;   // chunked prefill: a tile of query blocks before the chunk
+  const int r0 = band.blk_lo + tile * kScoreTile;                          // first block row of the tile
+  const int rows_valid = min(kScoreTile, band.blk_hi - r0);
+  int live = 0;
+  if (threadIdx.x < kScoreTile) {
+    const int r = threadIdx.x;
+    int start = 0, last = -1;
+    long long off = 0;
+    if (r < rows_valid) {
+      const int gb = r0 + r;
+      const int b = find_sequence(m.blk_off, m.batch, gb);
+      const int nb = m.blk_off[b + 1] - m.blk_off[b];
+      const int i = gb - m.blk_off[b];
+      start = m.blk_off[b];
+      off = m.score_off[b] + ((long long)h * nb + i) * nb - band.score_base;
+      if (!(m.chunked && i < m.qoff[b])) last = gb;                       // chunked prefill: rows before the chunk are skipped
+    }
+    row_start[r] = start; row_last[r] = last; row_off[r] = off;
+    live = last >= 0;
+  }
+  if (!__syncthreads_or(live)) return;                                     // a tile of query blocks before their chunks
   const size_t plane_q = (size_t)m.num_q_heads * m.total_blocks * kGateDim;
   const size_t plane_k = (size_t)m.num_kv_heads * m.total_blocks * kGateDim;
-  const uint16_t* gq_h = gq + ((size_t)h * m.total_blocks + m.blk_off[b]) * kGateDim;
-  const uint16_t* gk_g = gk + ((size_t)g * m.total_blocks + m.blk_off[b]) * kGateDim;
-  const int64_t sc_off = m.score_off[b] + (int64_t)h * nb * nb - band.score_base;
-  float* sc = scores + sc_off;
+  const uint16_t* gq_h = gq + (size_t)h * m.total_blocks * kGateDim;
+  const uint16_t* gk_g = gk + (size_t)g * m.total_blocks * kGateDim;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int wr = warp & 3, wc = warp >> 2;                               // row group, column half
   const int gid = lane >> 2, tig = lane & 3;
   const float scale = rsqrtf((float)kGateDim);
-  const bool vec_ok = (nb & 1) == 0 && (sc_off & 1) == 0;                // 8-byte stores of column pairs
 
-  const int last_col = i0 + rows_valid - 1;
-  gs_load_planes(sA, gq_h, plane_q, i0, rows_valid);
-  gs_load_planes(sB0, gk_g, plane_k, 0, min(kScoreTile, nb));
+  const int first_col = row_start[0];                                     // rows ascend, so do their sequence starts
+  const int last_col = r0 + rows_valid - 1;
+  gs_load_planes(sA, gq_h, plane_q, r0, rows_valid);
+  gs_load_planes(sB0, gk_g, plane_k, first_col, min(kScoreTile, last_col + 1 - first_col));
   asm volatile("cp.async.commit_group;" ::: "memory");
 
+  // the two rows of this thread: r = wr * 16 + gid + 8 e
+  int my_start[2], my_last[2];
+  long long my_off[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const int r = wr * 16 + gid + e * 8;
+    my_start[e] = row_start[r]; my_last[e] = row_last[r]; my_off[e] = row_off[r];
+  }
   float run_m[2] = {-CUDART_INF_F, -CUDART_INF_F}, run_l[2] = {0.f, 0.f};
   // the warp's A fragments (16 rows x 128 k, three planes) stay in registers for the whole row tile
   asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -363,11 +396,12 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
       gs_ldsm_x4(a[ks][pl], sA + (uint32_t)pl * kPlaneTile + gs_tile_off(row, ks * 2 + (lane >> 4)));
     }
   int buf = 0;
-  for (int j0 = 0; j0 <= last_col; j0 += kScoreTile, buf ^= 1) {
+  for (int j0 = first_col; j0 <= last_col; j0 += kScoreTile, buf ^= 1) {
     const uint32_t sB = sB0 + (uint32_t)buf * 3 * kPlaneTile;
     __syncthreads();                                   // the other B buffer's fragments have been read
     if (j0 + kScoreTile <= last_col)
-      gs_load_planes(sB0 + (uint32_t)(buf ^ 1) * 3 * kPlaneTile, gk_g, plane_k, j0 + kScoreTile, min(kScoreTile, nb - j0 - kScoreTile));
+      gs_load_planes(sB0 + (uint32_t)(buf ^ 1) * 3 * kPlaneTile, gk_g, plane_k, j0 + kScoreTile,
+                     min(kScoreTile, last_col + 1 - j0 - kScoreTile));
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 1;" ::: "memory");   // everything but the copy just started has landed
     __syncthreads();
@@ -396,19 +430,18 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
         }
       }
     }
-    // thread holds rows (gid, gid + 8) of the warp's 16 and columns (4 wc + nt) * 8 + 2 * tig + {0, 1}
+    // thread holds rows (gid, gid + 8) of the warp's 16 and columns (4 wc + nt) * 8 + 2 * tig + {0, 1} of the tile
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      const int i = i0 + wr * 16 + gid + e * 8;
-      if (i >= nb) continue;
+      if (my_last[e] < 0) continue;
       float x[4][2];
       float tmax = -CUDART_INF_F;
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          const int j = j0 + (wc * 4 + nt) * 8 + 2 * tig + c;
-          x[nt][c] = j <= i ? acc[nt][2 * e + c] * scale : -CUDART_INF_F;
+          const int j = j0 + (wc * 4 + nt) * 8 + 2 * tig + c;              // block of the batch
+          x[nt][c] = (j >= my_start[e] && j <= my_last[e]) ? acc[nt][2 * e + c] * scale : -CUDART_INF_F;
           tmax = fmaxf(tmax, x[nt][c]);
         }
       if (tmax == -CUDART_INF_F) continue;             // nothing causal for this thread in this tile
@@ -423,12 +456,14 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
         const int j = j0 + (wc * 4 + nt) * 8 + 2 * tig;
-        float* dst = sc + (size_t)i * nb + j;
-        if (vec_ok && j + 1 <= i) {
+        const long long at = my_off[e] + (j - my_start[e]);                // element offset of (row, j)
+        float* dst = scores + at;
+        const bool in0 = j >= my_start[e] && j <= my_last[e], in1 = j + 1 >= my_start[e] && j + 1 <= my_last[e];
+        if (in0 && in1 && (at & 1) == 0) {
           *reinterpret_cast<float2*>(dst) = make_float2(x[nt][0], x[nt][1]);
         } else {
-          if (j <= i) dst[0] = x[nt][0];
-          if (j + 1 <= i) dst[1] = x[nt][1];
+          if (in0) dst[0] = x[nt][0];
+          if (in1) dst[1] = x[nt][1];
         }
       }
     }
@@ -461,22 +496,22 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
   __syncthreads();
   // normalise in place: the logits this CTA just wrote are re-read (L2) and replaced by exp(x - m) / l; a warp per row,
   // four columns per lane and step, so that many independent loads are in flight
-  const bool vec4 = (nb & 3) == 0 && (sc_off & 3) == 0;
   for (int r = warp; r < rows_valid; r += kScoreThreads / 32) {
-    const int i = i0 + r;
+    if (row_last[r] < 0) continue;
+    const int n = row_last[r] - row_start[r] + 1;      // causal columns of the row
     const float mm = row_m[r];
     const float inv = 1.0f / row_l[r];
-    float* dst = sc + (size_t)i * nb;
-    if (vec4) {
-      const int full = (i + 1) & ~3;                   // columns 0 .. full-1 in whole float4s
+    float* dst = scores + row_off[r];
+    if ((row_off[r] & 3) == 0) {
+      const int full = n & ~3;                         // columns 0 .. full-1 in whole float4s
       for (int j = lane * 4; j < full; j += 128) {
         float4 v = *reinterpret_cast<float4*>(dst + j);
         v.x = __expf(v.x - mm) * inv; v.y = __expf(v.y - mm) * inv; v.z = __expf(v.z - mm) * inv; v.w = __expf(v.w - mm) * inv;
         *reinterpret_cast<float4*>(dst + j) = v;
       }
-      for (int j = full + lane; j <= i; j += 32) dst[j] = __expf(dst[j] - mm) * inv;
+      for (int j = full + lane; j < n; j += 32) dst[j] = __expf(dst[j] - mm) * inv;
     } else {
-      for (int j = lane; j <= i; j += 32) dst[j] = __expf(dst[j] - mm) * inv;
+      for (int j = lane; j < n; j += 32) dst[j] = __expf(dst[j] - mm) * inv;
     }
   }
 }
@@ -494,8 +529,8 @@ int launch_gate(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, c
     cudaError_t e0 = cudaGetLastError();
     return e0 == cudaSuccess ? 1 : -(int)e0;
   }
-  const ScoreBand all = {0, m.total_tiles, 0, m.num_q_heads, 0};
-  const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
+  const ScoreBand all = {0, m.total_blocks, 0, m.num_q_heads, 0};
+  const unsigned grid2 = (unsigned)((m.total_blocks + kScoreTile - 1) / kScoreTile) * (unsigned)m.num_q_heads;
   gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, all, gq, gk, scores);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 2 : -(int)e;
@@ -515,8 +550,8 @@ int launch_gate_ex(seer_ctx* ctx, const SeqMeta& m, const seer_gate_options& opt
     cudaError_t e0 = cudaGetLastError();
     return e0 == cudaSuccess ? 1 : -(int)e0;
   }
-  const ScoreBand all = {0, m.total_tiles, 0, m.num_q_heads, 0};
-  const unsigned grid2 = (unsigned)m.total_tiles * (unsigned)m.num_q_heads;
+  const ScoreBand all = {0, m.total_blocks, 0, m.num_q_heads, 0};
+  const unsigned grid2 = (unsigned)((m.total_blocks + kScoreTile - 1) / kScoreTile) * (unsigned)m.num_q_heads;
   gate_scores_kernel<<<grid2, kScoreThreads, kScoreSmem, stream>>>(m, all, gq, gk, scores);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 2 : -(int)e;
@@ -527,7 +562,7 @@ int launch_gate_scores_band(const SeqMeta& m, const ScoreBand& band, const void*
   size_t gq_bytes = ((size_t)m.num_q_heads * m.total_blocks * kGateDim * 6 + 255) / 256 * 256;
   const uint16_t* gq = (const uint16_t*)ws;
   const uint16_t* gk = (const uint16_t*)((const char*)ws + gq_bytes);
-  const unsigned grid = (unsigned)band.tiles * (unsigned)band.heads;
+  const unsigned grid = (unsigned)((band.blk_hi - band.blk_lo + kScoreTile - 1) / kScoreTile) * (unsigned)band.heads;
   if (grid == 0) return 0;
   gate_scores_kernel<<<grid, kScoreThreads, kScoreSmem, stream>>>(m, band, gq, gk, scores);
   cudaError_t e = cudaGetLastError();

@@ -51,7 +51,8 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
   t->total_tokens = cu[s->batch];
   t->total_q_tokens = s->cu_seqlens_q_host ? s->cu_seqlens_q_host[s->batch] : cu[s->batch];
   t->total_blocks = blocks;
-  t->total_chunks = chunks;
+  (void)chunks;
+  t->total_chunks = (blocks + kPoolChunk - 1) / kPoolChunk;   // chunks of the gate's first kernel run over the whole batch
   t->total_tiles = tiles;
   t->rows = blocks * s->num_q_heads;
   t->score_elems = sq * s->num_q_heads;
@@ -433,9 +434,9 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
     if (n < 0) bad = true; else launched += n;
   }
   // One band after the other, in CSR row order: scores of the band -> counts -> row_ptr (continued) -> lists.
-  auto run_band = [&](int tile_lo, int tiles, int head_lo, int heads, int64_t base, int64_t row_lo, int64_t row_hi) {
+  auto run_band = [&](int64_t blk_lo, int64_t blk_hi, int head_lo, int heads, int64_t base, int64_t row_lo, int64_t row_hi) {
     if (bad || row_hi <= row_lo) return;
-    const ScoreBand band = {tile_lo, tiles, head_lo, heads, base & ~(int64_t)3};
+    const ScoreBand band = {(int32_t)blk_lo, (int32_t)blk_hi, head_lo, heads, base & ~(int64_t)3};
     int n = launch_gate_scores_band(m, band, ws, band_buf, stream);
     if (n >= 0) {
       launched += n;
@@ -462,7 +463,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
         elems += (int64_t)Hq * n1 * n1; blocks += n1; tiles += (n1 + kScoreTile - 1) / kScoreTile;
         ++b1;
       }
-      run_band((int)tile_off, (int)tiles, 0, Hq, score_off, Hq * blk_off, Hq * (blk_off + blocks));
+      run_band(blk_off, blk_off + blocks, 0, Hq, score_off, Hq * blk_off, Hq * (blk_off + blocks));
       blk_off += blocks; tile_off += tiles; score_off += elems;
       b = b1;
       continue;
@@ -473,7 +474,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
       const int hb = (int)(cap / (nb * nb));
       for (int h0 = 0; h0 < Hq; h0 += hb) {
         const int h1 = h0 + hb < Hq ? h0 + hb : Hq;
-        run_band((int)tile_off, (int)ntile, h0, h1 - h0, score_off + (int64_t)h0 * nb * nb, Hq * blk_off + (int64_t)h0 * nb,
+        run_band(blk_off, blk_off + nb, h0, h1 - h0, score_off + (int64_t)h0 * nb * nb, Hq * blk_off + (int64_t)h0 * nb,
                  Hq * blk_off + (int64_t)h1 * nb);
       }
     } else {
@@ -483,7 +484,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
         for (int64_t t0 = 0; t0 < ntile; t0 += tb) {
           const int64_t t1 = t0 + tb < ntile ? t0 + tb : ntile;
           const int64_t i0 = t0 * kScoreTile, i1 = t1 * kScoreTile < nb ? t1 * kScoreTile : nb;
-          run_band((int)(tile_off + t0), (int)(t1 - t0), h, 1, score_off + ((int64_t)h * nb + i0) * nb,
+          run_band(blk_off + i0, blk_off + i1, h, 1, score_off + ((int64_t)h * nb + i0) * nb,
                    Hq * blk_off + (int64_t)h * nb + i0, Hq * blk_off + (int64_t)h * nb + i1);
         }
     }

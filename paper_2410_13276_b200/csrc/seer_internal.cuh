@@ -45,11 +45,11 @@ struct SeqMeta {
   int32_t chunked;             // 1 if the shape carries cu_seqlens_q
 };
 
-// A rectangle of (64-row score tile, query head) pairs whose scores are produced and consumed together; tiles are
-// numbered over the whole batch (tile_off).  score_base is the offset, in the full score matrix, of the band's first
-// element: the band's scores live at (full offset - score_base) in whatever buffer the kernels are given.
+// A rectangle of (block row of the packed batch, query head) pairs whose scores are produced and consumed together.
+// score_base is the offset, in the full score matrix, of the band's first element: the band's scores live at
+// (full offset - score_base) in whatever buffer the kernels are given.
 struct ScoreBand {
-  int32_t tile_lo, tiles;
+  int32_t blk_lo, blk_hi;      // block rows [blk_lo, blk_hi), numbered over the batch (blk_off)
   int32_t head_lo, heads;
   int64_t score_base;
 };

@@ -95,10 +95,32 @@ count_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mas
   } else if (ri.i >= ri.nb - p.dense_tail_blocks) {
     c = n;                                             // a dense row at the end of the sequence
   } else if (p.mode == SEER_THRESHOLD) {
-    for (int j = lane; j < n; j += 32) c += (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold) ? 1 : 0;
+    int head = 0;
+    if ((reinterpret_cast<uintptr_t>(ri.s) & 15) == 0) {       // four scores per lane and load where the row is aligned
+      head = n & ~3;
+      for (int j = lane * 4; j < head; j += 128) {
+        const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
+        c += (is_forced(j, ri.i, p.flags) || v.x > p.threshold) ? 1 : 0;
+        c += (is_forced(j + 1, ri.i, p.flags) || v.y > p.threshold) ? 1 : 0;
+        c += (is_forced(j + 2, ri.i, p.flags) || v.z > p.threshold) ? 1 : 0;
+        c += (is_forced(j + 3, ri.i, p.flags) || v.w > p.threshold) ? 1 : 0;
+      }
+    }
+    for (int j = head + lane; j < n; j += 32) c += (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold) ? 1 : 0;
     c = warp_sum(c);
   } else {
-    for (int j = lane; j < n; j += 32) c += (!is_forced(j, ri.i, p.flags) && score_key(ri.s[j]) != 0u) ? 1 : 0;
+    int head = 0;
+    if ((reinterpret_cast<uintptr_t>(ri.s) & 15) == 0) {
+      head = n & ~3;
+      for (int j = lane * 4; j < head; j += 128) {
+        const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
+        c += (!is_forced(j, ri.i, p.flags) && score_key(v.x) != 0u) ? 1 : 0;
+        c += (!is_forced(j + 1, ri.i, p.flags) && score_key(v.y) != 0u) ? 1 : 0;
+        c += (!is_forced(j + 2, ri.i, p.flags) && score_key(v.z) != 0u) ? 1 : 0;
+        c += (!is_forced(j + 3, ri.i, p.flags) && score_key(v.w) != 0u) ? 1 : 0;
+      }
+    }
+    for (int j = head + lane; j < n; j += 32) c += (!is_forced(j, ri.i, p.flags) && score_key(ri.s[j]) != 0u) ? 1 : 0;
     const int ncand = warp_sum(c);
     const int nf = num_forced(ri.i, p.flags);
     const int take = max(keep_count(n, p) - nf, 0);
@@ -190,7 +212,31 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   }
   if (p.mode == SEER_THRESHOLD) {
     int written = 0;
-    for (int base = 0; base < n; base += 32) {
+    int head = 0;
+    if ((reinterpret_cast<uintptr_t>(ri.s) & 15) == 0) {
+      // four consecutive columns per lane: the lane's kept columns follow those of the lanes below it
+      head = n & ~127;
+      for (int base = 0; base < head; base += 128) {
+        const int j = base + 4 * lane;
+        const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
+        const bool k0 = is_forced(j, ri.i, p.flags) || v.x > p.threshold, k1 = is_forced(j + 1, ri.i, p.flags) || v.y > p.threshold;
+        const bool k2 = is_forced(j + 2, ri.i, p.flags) || v.z > p.threshold, k3 = is_forced(j + 3, ri.i, p.flags) || v.w > p.threshold;
+        const int mine = (int)k0 + (int)k1 + (int)k2 + (int)k3;
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int u = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += u;
+        }
+        int at = written + incl - mine;
+        if (k0) out[at++] = j;
+        if (k1) out[at++] = j + 1;
+        if (k2) out[at++] = j + 2;
+        if (k3) out[at++] = j + 3;
+        written += __shfl_sync(0xffffffffu, incl, 31);
+      }
+    }
+    for (int base = head; base < n; base += 32) {
       const int j = base + lane;
       const bool keep = j < n && (is_forced(j, ri.i, p.flags) || ri.s[j] > p.threshold);
       const uint32_t bal = __ballot_sync(0xffffffffu, keep);
@@ -207,12 +253,22 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   const bool staged = n <= stage_cap;
   int c = 0;
   uint32_t k_and = 0xffffffffu, k_or = 0u;     // over the candidates' keys: the bits all of them share are k_and | ~k_or
-  for (int j = lane; j < n; j += 32) {
-    const uint32_t kk = is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]);
+  auto take_key = [&](int j, float sc) {
+    const uint32_t kk = is_forced(j, ri.i, p.flags) ? 0u : score_key(sc);
     if (staged) keys[j] = kk;
     c += kk != 0u;
     if (kk != 0u) { k_and &= kk; k_or |= kk; }
+  };
+  // four scores per lane and load where the row is 16-byte aligned (the loop is bound by the latency of its loads)
+  int head = 0;
+  if ((reinterpret_cast<uintptr_t>(ri.s) & 15) == 0) {
+    head = n & ~3;
+    for (int j = lane * 4; j < head; j += 128) {
+      const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
+      take_key(j, v.x); take_key(j + 1, v.y); take_key(j + 2, v.z); take_key(j + 3, v.w);
+    }
   }
+  for (int j = head + lane; j < n; j += 32) take_key(j, ri.s[j]);
   const int ncand = warp_sum(c);
   k_and = __reduce_and_sync(0xffffffffu, k_and);
   k_or = __reduce_or_sync(0xffffffffu, k_or);

@@ -405,11 +405,13 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 1;" ::: "memory");   // everything but the copy just started has landed
     __syncthreads();
-    float acc[4][4];
+    // two accumulators per 8-column group: the small terms and the large ones are independent MMA chains (the kernel is
+    // bound by the latency of dependent MMAs, eight warps per SM), added once per column tile, small to large
+    float acc[4][4], accs[4][4];
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-      for (int c = 0; c < 4; ++c) acc[nt][c] = 0.f;
+      for (int c = 0; c < 4; ++c) { acc[nt][c] = 0.f; accs[nt][c] = 0.f; }
 #pragma unroll
     for (int kk = 0; kk < 8; kk += 2) {                // two 16-wide k steps per pass (one B ldmatrix.x4 covers both)
 #pragma unroll
@@ -420,16 +422,20 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
           gs_ldsm_x4(bf[pl], sB + (uint32_t)pl * kPlaneTile + gs_tile_off((wc * 4 + nt) * 8 + (lane & 7), kk * 2 + (lane >> 3)));
 #pragma unroll
         for (int s2 = 0; s2 < 2; ++s2) {
-          // smallest terms first: hi*lo, lo*hi, mid*mid, then hi*mid, mid*hi, then hi*hi
-          gs_mma(acc[nt], a[kk + s2][0], bf[2][2 * s2], bf[2][2 * s2 + 1]);
-          gs_mma(acc[nt], a[kk + s2][2], bf[0][2 * s2], bf[0][2 * s2 + 1]);
-          gs_mma(acc[nt], a[kk + s2][1], bf[1][2 * s2], bf[1][2 * s2 + 1]);
+          // small chain: hi*lo, lo*hi, mid*mid; large chain: hi*mid, mid*hi, hi*hi
+          gs_mma(accs[nt], a[kk + s2][0], bf[2][2 * s2], bf[2][2 * s2 + 1]);
           gs_mma(acc[nt], a[kk + s2][0], bf[1][2 * s2], bf[1][2 * s2 + 1]);
+          gs_mma(accs[nt], a[kk + s2][2], bf[0][2 * s2], bf[0][2 * s2 + 1]);
           gs_mma(acc[nt], a[kk + s2][1], bf[0][2 * s2], bf[0][2 * s2 + 1]);
+          gs_mma(accs[nt], a[kk + s2][1], bf[1][2 * s2], bf[1][2 * s2 + 1]);
           gs_mma(acc[nt], a[kk + s2][0], bf[0][2 * s2], bf[0][2 * s2 + 1]);
         }
       }
     }
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[nt][c] += accs[nt][c];
     // thread holds rows (gid, gid + 8) of the warp's 16 and columns (4 wc + nt) * 8 + 2 * tig + {0, 1} of the tile
 #pragma unroll
     for (int e = 0; e < 2; ++e) {

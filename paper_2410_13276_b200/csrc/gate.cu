@@ -623,18 +623,16 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
 
   // per-batch offsets, built on the host stack and copied into the head of the array
   struct HostMeta {
-    int32_t cu[kStaticMaxBatch + 4], blk[kStaticMaxBatch + 4], chunk[kStaticMaxBatch + 4], tile[kStaticMaxBatch + 4];
+    int32_t cu[kStaticMaxBatch + 4], blk[kStaticMaxBatch + 4];
     int64_t score[kStaticMaxBatch + 2];
   } hm;
   static_assert(sizeof(HostMeta) <= kStaticMetaBytes, "metadata region too small");
-  hm.blk[0] = hm.chunk[0] = hm.tile[0] = 0;
+  hm.blk[0] = 0;
   hm.score[0] = 0;
   for (int b = 0; b < shape->batch; ++b) {
     hm.cu[b] = shape->cu_seqlens_host[b];
     const int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + shape->block - 1) / shape->block;
     hm.blk[b + 1] = hm.blk[b] + nb;
-    hm.chunk[b + 1] = hm.chunk[b] + (nb + kPoolChunk - 1) / kPoolChunk;
-    hm.tile[b + 1] = hm.tile[b] + (nb + kScoreTile - 1) / kScoreTile;
     hm.score[b + 1] = hm.score[b] + (int64_t)shape->num_q_heads * nb * nb;
   }
   hm.cu[shape->batch] = shape->cu_seqlens_host[shape->batch];
@@ -644,8 +642,6 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   SeqMeta m;
   m.cu_seqlens = (const int32_t*)(base + offsetof(HostMeta, cu));
   m.blk_off = (const int32_t*)(base + offsetof(HostMeta, blk));
-  m.chunk_off = (const int32_t*)(base + offsetof(HostMeta, chunk));
-  m.tile_off = (const int32_t*)(base + offsetof(HostMeta, tile));
   m.score_off = (const int64_t*)(base + offsetof(HostMeta, score));
   m.batch = shape->batch;
   m.num_q_heads = shape->num_q_heads;
@@ -654,7 +650,6 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   m.total_tokens = (int32_t)t.total_tokens;
   m.total_blocks = (int32_t)t.total_blocks;
   m.total_chunks = (int32_t)t.total_chunks;
-  m.total_tiles = (int32_t)t.total_tiles;
   m.max_nb = t.max_nb;
   m.rows = t.rows;
   m.score_elems = t.score_elems;

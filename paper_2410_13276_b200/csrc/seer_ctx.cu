@@ -10,9 +10,7 @@ static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // Byte offsets of the four arrays inside a metadata slot.
 constexpr size_t kOffCu = 0;
 constexpr size_t kOffBlk = kOffCu + sizeof(int32_t) * (kMaxBatch + 1 + 3);
-constexpr size_t kOffChunk = kOffBlk + sizeof(int32_t) * (kMaxBatch + 1 + 3);
-constexpr size_t kOffTile = kOffChunk + sizeof(int32_t) * (kMaxBatch + 1 + 3);
-constexpr size_t kOffScore = kOffTile + sizeof(int32_t) * (kMaxBatch + 1 + 3);
+constexpr size_t kOffScore = kOffBlk + sizeof(int32_t) * (kMaxBatch + 1 + 3);
 constexpr size_t kOffQoff = kOffScore + sizeof(int64_t) * (kMaxBatch + 1);
 constexpr size_t kOffQdelta = kOffQoff + sizeof(int32_t) * (kMaxBatch + 4);
 constexpr size_t kSlotBytes = kOffQdelta + sizeof(int32_t) * (kMaxBatch + 4);
@@ -36,14 +34,12 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
       if (sq > 0 && (sk - sq) % s->block != 0) return SEER_ERR_UNSUPPORTED;
     }
   }
-  int64_t blocks = 0, chunks = 0, tiles = 0, sq = 0, causal = 0;
+  int64_t blocks = 0, sq = 0, causal = 0;
   int32_t max_nb = 0;
   for (int b = 0; b < s->batch; ++b) {
     if (cu[b + 1] < cu[b]) return SEER_ERR_INVALID_ARG;
     int64_t nb = ((int64_t)cu[b + 1] - cu[b] + s->block - 1) / s->block;
     blocks += nb;
-    chunks += (nb + kPoolChunk - 1) / kPoolChunk;
-    tiles += (nb + kScoreTile - 1) / kScoreTile;
     sq += nb * nb;
     causal += nb * (nb + 1) / 2;
     if (nb > max_nb) max_nb = (int32_t)nb;
@@ -51,9 +47,7 @@ seer_status shape_totals(const seer_shape* s, ShapeTotals* t) {
   t->total_tokens = cu[s->batch];
   t->total_q_tokens = s->cu_seqlens_q_host ? s->cu_seqlens_q_host[s->batch] : cu[s->batch];
   t->total_blocks = blocks;
-  (void)chunks;
   t->total_chunks = (blocks + kPoolChunk - 1) / kPoolChunk;   // chunks of the gate's first kernel run over the whole batch
-  t->total_tiles = tiles;
   t->rows = blocks * s->num_q_heads;
   t->score_elems = sq * s->num_q_heads;
   t->causal_blocks = causal * s->num_q_heads;
@@ -97,18 +91,14 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
     char* h = (char*)s.pinned;
     int32_t* cu = (int32_t*)(h + kOffCu);
     int32_t* blk = (int32_t*)(h + kOffBlk);
-    int32_t* chk = (int32_t*)(h + kOffChunk);
-    int32_t* til = (int32_t*)(h + kOffTile);
     int64_t* sc = (int64_t*)(h + kOffScore);
     int32_t* qo = (int32_t*)(h + kOffQoff);
     int32_t* qd = (int32_t*)(h + kOffQdelta);
-    blk[0] = 0; chk[0] = 0; til[0] = 0; sc[0] = 0;
+    blk[0] = 0; sc[0] = 0;
     for (int b = 0; b < shape->batch; ++b) {
       cu[b] = shape->cu_seqlens_host[b];
       int32_t nb = (shape->cu_seqlens_host[b + 1] - shape->cu_seqlens_host[b] + shape->block - 1) / shape->block;
       blk[b + 1] = blk[b] + nb;
-      chk[b + 1] = chk[b] + (nb + kPoolChunk - 1) / kPoolChunk;
-      til[b + 1] = til[b] + (nb + kScoreTile - 1) / kScoreTile;
       sc[b + 1] = sc[b] + (int64_t)shape->num_q_heads * nb * nb;
       qo[b] = 0; qd[b] = 0;
       if (const int32_t* cq = shape->cu_seqlens_q_host) {
@@ -130,8 +120,6 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   const char* d = (const char*)s.dev;
   m->cu_seqlens = (const int32_t*)(d + kOffCu);
   m->blk_off = (const int32_t*)(d + kOffBlk);
-  m->chunk_off = (const int32_t*)(d + kOffChunk);
-  m->tile_off = (const int32_t*)(d + kOffTile);
   m->score_off = (const int64_t*)(d + kOffScore);
   m->batch = shape->batch;
   m->num_q_heads = shape->num_q_heads;
@@ -140,7 +128,6 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   m->total_tokens = (int32_t)t.total_tokens;
   m->total_blocks = (int32_t)t.total_blocks;
   m->total_chunks = (int32_t)t.total_chunks;
-  m->total_tiles = (int32_t)t.total_tiles;
   m->max_nb = t.max_nb;
   m->rows = t.rows;
   m->score_elems = t.score_elems;
@@ -450,21 +437,21 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
   const int32_t* cu = shape->cu_seqlens_host;
   const int Hq = shape->num_q_heads;
   auto blocks_of = [&](int b) { return ((int64_t)cu[b + 1] - cu[b] + shape->block - 1) / shape->block; };
-  int64_t blk_off = 0, tile_off = 0, score_off = 0;    // of sequence b
+  int64_t blk_off = 0, score_off = 0;                  // of sequence b
   for (int b = 0; b < shape->batch && !bad;) {
     const int64_t nb = blocks_of(b);
     if ((int64_t)Hq * nb * nb <= cap) {
       // whole sequences, as many as fit
       int b1 = b;
-      int64_t blocks = 0, tiles = 0, elems = 0;
+      int64_t blocks = 0, elems = 0;
       while (b1 < shape->batch) {
         const int64_t n1 = blocks_of(b1);
         if (elems + (int64_t)Hq * n1 * n1 > cap) break;
-        elems += (int64_t)Hq * n1 * n1; blocks += n1; tiles += (n1 + kScoreTile - 1) / kScoreTile;
+        elems += (int64_t)Hq * n1 * n1; blocks += n1;
         ++b1;
       }
       run_band(blk_off, blk_off + blocks, 0, Hq, score_off, Hq * blk_off, Hq * (blk_off + blocks));
-      blk_off += blocks; tile_off += tiles; score_off += elems;
+      blk_off += blocks; score_off += elems;
       b = b1;
       continue;
     }
@@ -488,7 +475,7 @@ seer_status seer_gate_block_mask(seer_ctx* ctx, const seer_shape* shape, const s
                    Hq * blk_off + (int64_t)h * nb + i0, Hq * blk_off + (int64_t)h * nb + i1);
         }
     }
-    blk_off += nb; tile_off += ntile; score_off += (int64_t)Hq * nb * nb;
+    blk_off += nb; score_off += (int64_t)Hq * nb * nb;
     ++b;
   }
   finish_call(ctx, slot, stream);

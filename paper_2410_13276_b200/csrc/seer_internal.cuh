@@ -16,15 +16,13 @@ constexpr int kGateDim = 128;
 constexpr int kMaxBatch = 4096;
 constexpr int kMetaSlots = 8;
 constexpr int kPoolChunk = 16;  // blocks pooled and projected by one CTA of the gate's first kernel
-constexpr int kScoreTile = 64;  // score rows handled by one CTA of the gate's second kernel
+constexpr int kScoreTile = 64;  // score rows (blocks of the packed batch) handled by one CTA of the gate's second kernel
 
 // Per-batch metadata the kernels read from device memory.
 struct SeqMeta {
   const int32_t* cu_seqlens;   // [batch+1] token offsets
   const int32_t* blk_off;      // [batch+1] cumulative number of blocks
   const int64_t* score_off;    // [batch+1] Hq * cumulative nb^2
-  const int32_t* chunk_off;    // [batch+1] cumulative ceil(nb / kPoolChunk)
-  const int32_t* tile_off;     // [batch+1] cumulative ceil(nb / kScoreTile)
   int32_t batch;
   int32_t num_q_heads;
   int32_t num_kv_heads;
@@ -32,7 +30,6 @@ struct SeqMeta {
   int32_t total_tokens;
   int32_t total_blocks;
   int32_t total_chunks;
-  int32_t total_tiles;
   int32_t max_nb;
   int64_t rows;                // Hq * total_blocks
   int64_t score_elems;
@@ -90,7 +87,7 @@ void finish_call(seer_ctx* ctx, int slot, cudaStream_t stream);
 
 // Host-only shape arithmetic (no CUDA calls): returns SEER_OK and fills totals.
 struct ShapeTotals {
-  int64_t total_tokens, total_q_tokens, total_blocks, total_chunks, total_tiles, rows, score_elems, causal_blocks;
+  int64_t total_tokens, total_q_tokens, total_blocks, total_chunks, rows, score_elems, causal_blocks;
   int32_t max_nb;
 };
 seer_status shape_totals(const seer_shape* shape, ShapeTotals* t);

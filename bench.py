@@ -150,7 +150,7 @@ def cpu_oracle_sample(w, rp, col, budget_rows=None):
     """Times the oracle's attention on a sample of (head, query-block) rows.  Returns (tflops, seconds, description, cores)."""
     from oracle import seer_oracle as O
     from paper_2410_13276_b200 import workloads as W
-    rows = W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=1234, per_head_random=32)   # ~1150 rows, about 10 s of CPU work
+    rows = W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=1234, per_head_random=56)   # ~1900 rows, about 10 s of CPU work
     if budget_rows:
         rows = rows[:: max(1, len(rows) // budget_rows)]
     blocks = int(sum(int(rp[r + 1] - rp[r]) for r in rows))

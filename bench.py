@@ -468,6 +468,8 @@ def main():
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
                             "kernel": "seer_sparse_attn"},
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
+               # mask builder: every causal score read once, every kept block and row offset written once (algorithmic bytes)
+               "mask_gbs": ((B.seer_causal_blocks(p.shape) + nnz + B.seer_mask_rows(p.shape)) * 4) / (mask_ms * 1e-3) / 1e9,
                "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128, "chunked_prefill": chunked,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:

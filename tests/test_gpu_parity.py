@@ -403,3 +403,53 @@ def test_attention_kernel_chosen_by_shape(rt):
             B.seer_set_attn_impl(ctx, 3)
     finally:
         B.seer_set_attn_impl(ctx, 0)
+
+
+@pytest.mark.parametrize("name", ["c1", "c2s", "c3s", "c4s", "c5s"])
+def test_end_to_end_list_overlap_with_the_oracle(rt, name, record_property):
+    """GPU gate -> GPU mask against oracle gate -> oracle mask on the reduced twins.  Not a bit-exact gate: scores within
+    1e-3 of each other may fall on different sides of the selection boundary.  The Jaccard overlap of the (row, block)
+    pairs is reported and must stay high; every difference must be a near-boundary flip (both scores within 2e-3
+    relative of the row's boundary score)."""
+    B, Prefill, ctx = rt
+    w = W.make_workload(name)
+    spec = w.masks[0]
+    thr = spec.threshold
+    if spec.mode == W.MODE_THRESHOLD and thr is None:
+        import json, os
+        with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "thresholds.json")) as f:
+            thr = float.fromhex(json.load(f)[name]["threshold_hex"])
+    p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx, want_lse=False)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    params = B.make_mask_params(spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k, threshold=thr or 0.0,
+                                flags=spec.flags)
+    p.gate(); p.mask(params)
+    assert p.status() == 0
+    rp, col = p.lists_host()
+    ref_scores = O.gate_scores(w.q, w.k, w.wq, w.wk, w.cu_seqlens, 64)
+    orp, ocol = O.block_mask(ref_scores, spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                             threshold=thr or 0.0, flags=spec.flags)
+    rows = len(rp) - 1
+    g = set(zip(np.repeat(np.arange(rows), np.diff(rp)).tolist(), col.tolist()))
+    o = set(zip(np.repeat(np.arange(rows), np.diff(orp)).tolist(), ocol.tolist()))
+    jac = len(g & o) / max(len(g | o), 1)
+    record_property("jaccard", jac)
+    print(f"{name}: kept {len(g)} (gpu) / {len(o)} (oracle), Jaccard {jac:.6f}")
+    assert jac >= 0.995, (name, jac)
+    # the differing pairs are near-boundary: their oracle score is within 2e-3 relative of the weakest kept score of the row
+    flat = {}
+    base = 0
+    for b, S in enumerate(ref_scores):
+        Hq, nb, _ = S.shape
+        for h in range(Hq):
+            for i in range(nb):
+                flat[base + h * nb + i] = S[h, i]
+        base += Hq * nb
+    for (r, j) in (g ^ o):
+        row = flat[r].astype(np.float64)
+        kept_o = ocol[orp[r]:orp[r + 1]]
+        if spec.mode == W.MODE_THRESHOLD:
+            bound = float(np.float32(thr))
+        else:
+            bound = float(min(row[x] for x in kept_o.tolist()))          # the weakest kept score of the row
+        assert abs(row[j] - bound) <= 2e-3 * abs(bound) + 1e-30, (name, r, j, row[j], bound)

@@ -408,6 +408,24 @@ def main():
                    "attn_tflops": n3 * FLOP_PER_BLOCK / (t[2] * 1e-3) / 1e12, "o_equals_rows_of_whole_run": same}
         del o3
 
+    # list statistics of the bench mask: K/V sharing factor of the lists inside a GQA group (entries / distinct
+    # (KV head, query block, key block) triples) and issued over useful MMA work of the tcgen05 kernel (S^T is computed on
+    # whole 128-key tiles, so the last tile of an odd list is half padding; P V skips that half)
+    list_stats = None
+    if rank == 0 and not args.no_extras and len(w.cu_seqlens) == 2:
+        rp_h = p.row_ptr.cpu().numpy().astype(np.int64)
+        col_h = p.col_idx[:nnz].cpu().numpy().astype(np.int64)
+        nb_h = int(w.num_blocks[0]); G_h = w.num_q_heads // w.num_kv_heads
+        counts = np.diff(rp_h)
+        row_of = np.repeat(np.arange(len(counts), dtype=np.int64), counts)
+        head_of, i_of = row_of // nb_h, row_of % nb_h
+        triple = ((head_of // G_h) * nb_h + i_of) * nb_h + col_h
+        useful = float(counts.sum())
+        issued = float((2 * ((counts + 1) // 2)).sum())
+        list_stats = {"kv_sharing_factor": useful / float(np.unique(triple).size),
+                      "mma_issued_over_useful": (issued + useful) / (2.0 * useful)}
+        del rp_h, col_h, row_of, head_of, i_of, triple
+
     # the max-pooled attention map on the kept blocks (Eq. 2; a side output for distillation / diagnostics), outside the
     # timed region: one attention launch that also writes lse, then the block-max pass
     block_max_ms = None
@@ -470,7 +488,7 @@ def main():
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
                # mask builder: every causal score read once, every kept block and row offset written once (algorithmic bytes)
                "mask_gbs": ((B.seer_causal_blocks(p.shape) + nnz + B.seer_mask_rows(p.shape)) * 4) / (mask_ms * 1e-3) / 1e9,
-               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128, "chunked_prefill": chunked,
+               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128, "chunked_prefill": chunked, "list_stats": list_stats,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:
             dense_blocks = B.seer_causal_blocks(p.shape)

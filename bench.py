@@ -34,8 +34,8 @@ METRIC = "sparse_prefill_attention_effective_tflops_128k_90pct_block_sparsity"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--keep", default="1/10", help="TopK ratio for the c3 workload")
@@ -479,7 +479,7 @@ def main():
                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_desc(w, spec),
                "kept_blocks": nnz, "stage_ms": {"gate": gate_ms, "mask": mask_ms, "attn": attn_ms,
-                                                "attn_min": float(min(attn_all))},
+                                                "attn_min": float(min(attn_all)), "attn_median": float(np.median(attn_all))},
                "attn_kernel": "tcgen05" if args.attn_impl == 0 else "mma.sync",
                "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
                             "frac": achieved / burst, "peak_source": f"bf16 dense burst, of {src}",

@@ -62,14 +62,23 @@ def pick_mask(w, args, need_threshold=True):
     return spec
 
 
+L2_BYTES = 126 << 20
+
+
+def input_bytes(w) -> int:
+    return int(w.total_tokens) * (w.num_q_heads + 2 * w.num_kv_heads) * 256
+
+
 def workload_desc(w, spec):
+    flush = input_bytes(w) <= 2 * L2_BYTES
     return {"workload": f"{w.name}: 1 attention layer, batch {len(w.cu_seqlens) - 1}, tokens {w.total_tokens}, "
                         f"{w.num_q_heads} q heads / {w.num_kv_heads} kv heads, head_dim 128, block 64, causal",
             "mask": ({0: "topk_ratio", 1: "topk_count", 2: "threshold"}[spec.mode]
                      + (f" {spec.keep_num}/{spec.keep_den}" if spec.mode == 0 else
                         f" {spec.threshold!r} (target sparsity {spec.target_sparsity})" if spec.mode == 2 else f" {spec.k}")
                      + f", flags {spec.flags}"),
-            "l2": "inputs larger than L2 (no flush)"}
+            "l2": ("L2 flushed before every timed step (a 256 MB buffer is overwritten; the step time is the sum of the "
+                   "per-step event spans)" if flush else "inputs larger than L2 (no flush)")}
 
 
 def peaks():
@@ -273,8 +282,12 @@ def main():
     if sampler:
         sampler.mark_start()
     t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    # small workloads fit the 126 MB L2: overwrite a buffer twice that size before every step, outside the event spans
+    flush_buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if input_bytes(w) <= 2 * L2_BYTES else None
     t_start.record(stream)
     for s in range(args.steps):
+        if flush_buf is not None:
+            flush_buf.fill_(s & 0xff)
         ev[s][0].record(stream); p.gate()
         ev[s][1].record(stream); p.mask(params)
         ev[s][2].record(stream); p.attn()
@@ -282,6 +295,9 @@ def main():
     t_end.record(stream)
     barrier()
     total_ms = t_start.elapsed_time(t_end)
+    if flush_buf is not None:                                # leave the flushes out: sum of the per-step spans
+        total_ms = float(sum(e[0].elapsed_time(e[3]) for e in ev))
+        del flush_buf
     launches = B.seer_launch_count(p.ctx) - l0
     clocks = None
     if sampler:

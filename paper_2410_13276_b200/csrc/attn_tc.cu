@@ -793,6 +793,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const float cm = fmaxf(fmaxf(lsum[gt], lsum[64 + gt]), fmaxf(lsum[128 + gt], lsum[192 + gt]));
             float nm = fmaxf(old, cm + kRefShift);
             if (nm == -CUDART_INF_F) nm = 0.f;           // nothing visible in this column yet
+            // a query column past the end of a ragged block holds whatever tokens follow in the packed tensor: an
+            // unreachable reference makes its p = 0, so that it can never ask for a rebase (results must not depend on
+            // the neighbours in the batch)
+            if (gt >= it.q_valid) nm = 1.0e30f;
             alpha[gt] = old == -CUDART_INF_F ? 0.f : exp2f(old - nm);
             mref[gt] = nm;
           }

@@ -453,3 +453,34 @@ def test_end_to_end_list_overlap_with_the_oracle(rt, name, record_property):
         else:
             bound = float(min(row[x] for x in kept_o.tolist()))          # the weakest kept score of the row
         assert abs(row[j] - bound) <= 2e-3 * abs(bound) + 1e-30, (name, r, j, row[j], bound)
+
+
+def test_output_does_not_depend_on_the_neighbours_in_the_batch(rt):
+    """A sequence whose last block is ragged: the query columns past its end hold the first tokens of the next sequence
+    in the packed tensor.  They must be inert (they could otherwise ask for a rescaling of the whole tile and change
+    the rounding of the valid columns): attention output and lse of the sequence are bit-identical whether it is
+    followed by nothing, by small tokens or by huge ones, with the same lists."""
+    import torch
+    B, Prefill, ctx = rt
+    S, hq, hkv = 333, 2, 1
+    w = W.make_small(seed=52_000, seqlens=[S], hq=hq, hkv=hkv, q_gain=2.0)
+    rp, col = O.full_causal_lists([0, S], 64, hq)
+    outs = []
+    for tail, gain in ((0, 0.0), (200, 1.0), (200, 60.0)):
+        lens = [S] + ([tail] if tail else [])
+        w2 = W.make_small(seed=52_001, seqlens=lens, hq=hq, hkv=hkv, q_gain=1.0)
+        q, k, v = w2.q.copy(), w2.k.copy(), w2.v.copy()
+        q[:S], k[:S], v[:S] = w.q, w.k, w.v
+        if tail:
+            big = W.f32_to_bf16_bits((np.random.default_rng(5).standard_normal((tail, hq, 128)) * gain).astype(np.float32))
+            q[S:] = big
+            k[S:] = W.f32_to_bf16_bits((np.random.default_rng(6).standard_normal((tail, hkv, 128)) * gain).astype(np.float32))
+        rp2, col2 = O.full_causal_lists(w2.cu_seqlens, 64, hq)
+        p = Prefill(w2.cu_seqlens, hq, hkv, ctx=ctx, want_lse=True)
+        p.set_inputs(q, k, v, w2.wq, w2.wk)
+        p.set_lists(rp2, col2)
+        p.attn()
+        assert p.status() == 0
+        outs.append((p.o[:S].clone(), p.lse[:, :S].clone()))
+    for o2, l2 in outs[1:]:
+        assert torch.equal(o2, outs[0][0]) and torch.equal(l2, outs[0][1])

@@ -85,3 +85,64 @@ def test_random_shape_whole_path(rt, seed):
     assert np.all(np.abs(lg[fin] - lr[fin]) <= 2e-3 + 1e-3 * np.abs(lr[fin])) and np.all(lg[~fin] == lr[~fin])
     bref = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, hq, hkv, 64, 1 / math.sqrt(128))
     assert np.all(np.abs(bmax[: len(col)] - bref) <= 1e-2 * bref + 1e-7), (lens, hq, hkv, kw)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_shape_all_features(rt, seed):
+    """Seeded random combinations of everything the library offers on one problem: block 64 or 128, composed pooling
+    and block RoPE in the gate, every mask mode with random flags and a dense tail, the one-call gate + mask with a random
+    band size, the list expansion for 128-token blocks, attention and (at block 64) the max-pooled map; each against
+    the oracle as in the tests of the single features."""
+    import torch
+    from test_oracle_block128 import expand_reference
+    B, Prefill, ctx = rt
+    rng = np.random.default_rng(777_000 + seed)
+    blk = int(rng.choice([64, 128]))
+    nseq = int(rng.integers(1, 4))
+    lens = [int(x) for x in rng.choice([1, 63, 64, 65, 127, 128, 129, 200, 333, 512, 700, 1000], size=nseq)]
+    hkv = int(rng.integers(1, 3))
+    hq = hkv * int(rng.choice([1, 2, 4, 5]))
+    mode = int(rng.integers(0, 3))
+    kw = dict(keep_num=int(rng.integers(1, 3)), keep_den=int(rng.integers(2, 7)), k=int(rng.integers(0, 6)),
+              threshold=float(rng.choice([0.0, 0.02, 0.1, 0.5])), flags=int(rng.choice([0, 1, 2, 3])))
+    tail = int(rng.choice([0, 0, 1, 2]))
+    pq, pk = int(rng.choice([1, 3, 7])), int(rng.choice([1, 6, 7]))
+    theta = float(rng.choice([0.0, 10000.0, 500000.0]))
+    w = W.make_small(seed=778_000 + seed, seqlens=lens, hq=hq, hkv=hkv, q_gain=float(rng.choice([1.0, 3.0])), block=blk)
+    wq = W.make_gate_weights(seed, hq, bin(pq).count("1") * 128)
+    wk = W.make_gate_weights(seed + 1, hkv, bin(pk).count("1") * 128)
+    wq_d, wk_d = torch.from_numpy(wq).cuda(), torch.from_numpy(wk).cuda()
+    opt = B.seer_gate_options(pq, pk, theta)
+    params = B.make_mask_params(mode, dense_tail=tail, **kw)
+    what = (blk, lens, hq, hkv, mode, kw, tail, pq, pk, theta)
+    p = Prefill(w.cu_seqlens, hq, hkv, ctx=ctx, want_lse=True, block=blk)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    p.o.fill_(float("nan"))
+    p.gate_ex(opt, wq_d, wk_d); p.mask(params); p.attn()
+    assert p.status() == 0, what
+    got = O.unflatten_scores(p.scores_host(), w.cu_seqlens, blk, hq)
+    ref = O.gate_scores_ex(w.q, w.k, wq, wk, w.cu_seqlens, blk, pool_q=pq, pool_k=pk, rope_theta=theta)
+    for g, r in zip(got, ref):
+        il = np.tril_indices(r.shape[-1])
+        gg, rr = g[:, il[0], il[1]].astype(np.float64), r[:, il[0], il[1]].astype(np.float64)
+        assert np.all(np.abs(gg - rr) <= np.where(rr < 1e-30, 1e-33, 1e-3 * rr)), what
+    rp, col = p.lists_host()
+    orp, ocol = O.block_mask(got, mode, dense_tail=tail, **kw)
+    assert np.array_equal(rp, orp) and np.array_equal(col, ocol), what
+    if blk == 128:
+        rp64, col64 = p.lists64_host()
+        erp, ecol = expand_reference(w.cu_seqlens, hq, rp, col)
+        assert np.array_equal(rp64, erp) and np.array_equal(col64, ecol), what
+    o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, hq, hkv, blk, 1 / math.sqrt(128))
+    x = p.o_host().astype(np.float64)
+    assert np.all(np.abs(x - o_ref) <= 2e-2 + 1e-2 * np.abs(o_ref)), what
+    lg, fin = p.lse_host().astype(np.float64), np.isfinite(lse_ref)
+    assert np.all(np.abs(lg[fin] - lse_ref[fin]) <= 2e-3 + 1e-3 * np.abs(lse_ref[fin])) and np.all(np.isneginf(lg[~fin])), what
+    p.row_ptr.fill_(-1)
+    p.gate_mask(params, band_bytes=int(rng.choice([0, 20000, 1 << 20])), options=opt, wq=wq_d, wk=wk_d)
+    rp2, col2 = p.lists_host()
+    assert p.status() == 0 and np.array_equal(rp2, rp) and np.array_equal(col2, col), what
+    if blk == 64:
+        bm = p.block_max().cpu().numpy()[:len(col)]
+        bref = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, hq, hkv, 64, 1 / math.sqrt(128))
+        assert np.all(np.abs(bm - bref) <= 1e-2 * np.abs(bref) + 1e-30), what

@@ -146,3 +146,53 @@ def test_random_shape_all_features(rt, seed):
         bm = p.block_max().cpu().numpy()[:len(col)]
         bref = O.maxpool_listed_blocks(w.q, w.k, w.cu_seqlens, rp, col, hq, hkv, 64, 1 / math.sqrt(128))
         assert np.all(np.abs(bm - bref) <= 1e-2 * np.abs(bref) + 1e-30), what
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_lists_on_data_that_moves_the_softmax_references(rt, seed):
+    """Random lists (odd lengths, rows without their diagonal block, empty rows) on inputs built to exceed the running
+    softmax references again and again: key norms that grow along the sequence, a few huge outlier keys, queries of very
+    different scales, strongly negative logits followed by a late positive block.  Both attention kernels against the
+    oracle."""
+    B, Prefill, ctx = rt
+    rng = np.random.default_rng(555_000 + seed)
+    lens = [int(rng.integers(300, 2500)) for _ in range(int(rng.integers(1, 3)))]
+    hq = int(rng.choice([1, 2]))
+    w = W.make_small(seed=556_000 + seed, seqlens=lens, hq=hq, hkv=1)
+    T = int(w.cu_seqlens[-1])
+    kf, qf = W.bf16_bits_to_f32(w.k).copy(), W.bf16_bits_to_f32(w.q).copy()
+    kind = int(rng.integers(0, 4))
+    if kind == 0:
+        kf *= np.linspace(0.2, float(rng.choice([8.0, 20.0])), T, dtype=np.float32)[:, None, None]
+    elif kind == 1:
+        kf[rng.choice(T, size=8, replace=False)] *= 40.0
+    elif kind == 2:
+        qf *= np.exp(rng.normal(0, 1.5, size=(T, 1, 1))).astype(np.float32)
+    else:
+        kf[:] = -np.abs(kf); qf[:] = np.abs(qf); kf[T - 70:] = np.abs(kf[T - 70:]) * 3
+    k, q = W.f32_to_bf16_bits(kf), W.f32_to_bf16_bits(qf)
+    rp, col = [0], []
+    for S in lens:
+        for _h in range(hq):
+            for i in range((S + 63) // 64):
+                keep = {i} if rng.random() < 0.9 else set()
+                keep |= {int(j) for j in range(i + 1) if rng.random() < 0.5}
+                col.extend(sorted(keep)); rp.append(len(col))
+    rp, col = np.asarray(rp, np.int64), np.asarray(col, np.int32)
+    p = Prefill(w.cu_seqlens, hq, 1, ctx=ctx, want_lse=True)
+    p.set_inputs(q, k, w.v, w.wq, w.wk)
+    p.set_lists(rp, col)
+    o_ref, lse_ref = O.sparse_attention(q, k, w.v, w.cu_seqlens, rp, col, hq, 1, 64, 1 / math.sqrt(128))
+    fin = np.isfinite(lse_ref)
+    try:
+        for impl in (0, 1):
+            B.seer_set_attn_impl(ctx, impl)
+            p.o.fill_(float("nan"))
+            p.attn()
+            assert p.status() == 0, (seed, impl)
+            x, lg = p.o_host().astype(np.float64), p.lse_host().astype(np.float64)
+            assert np.all(np.abs(x - o_ref) <= 2e-2 + 1e-2 * np.abs(o_ref)), (seed, impl, kind)
+            assert np.all(np.abs(lg[fin] - lse_ref[fin]) <= 2e-3 + 1e-3 * np.abs(lse_ref[fin])), (seed, impl, kind)
+            assert np.all(np.isneginf(lg[~fin]))
+    finally:
+        B.seer_set_attn_impl(ctx, 0)

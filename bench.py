@@ -40,7 +40,7 @@ def parse():
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--keep", default="1/10", help="TopK ratio for the c3 workload")
     ap.add_argument("--seq", type=int, default=None, help="override the sequence length (profiling on a smaller case)")
-    ap.add_argument("--attn-impl", type=int, default=0, help="0 tcgen05 kernel, 1 mma.sync kernel, 2 chosen per call from the shape")
+    ap.add_argument("--attn-impl", type=int, default=0, help="0 tcgen05 kernel, 1 mma.sync kernel, 2 chosen per call from the shape, 3 tcgen05 kernel split by query columns")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-list run of the attention kernel")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true")
@@ -496,7 +496,7 @@ def main():
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_desc(w, spec),
                "kept_blocks": nnz, "stage_ms": {"gate": gate_ms, "mask": mask_ms, "attn": attn_ms,
                                                 "attn_min": float(min(attn_all)), "attn_median": float(np.median(attn_all))},
-               "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape"}[args.attn_impl],
+               "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape", 3: "tcgen05, softmax split by query columns"}[args.attn_impl],
                "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
                             "frac": achieved / burst, "peak_source": f"bf16 dense burst, of {src}",
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,

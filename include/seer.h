@@ -160,7 +160,11 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
  * the shape: the persistent tcgen05 kernel pays about 10 us per (head, query block) row whatever its list length, the
  * mma.sync kernel about 3.5 us plus more per block, so batches whose rows have at most 8 causal blocks on average
  * (many short sequences) go to the mma.sync kernel and everything else to the tcgen05 kernel (measured crossover:
- * 8.5 listed blocks per row).  Returns SEER_ERR_INVALID_ARG for other values. */
+ * 8.5 listed blocks per row); 3 = the tcgen05 kernel with the softmax work split by query columns instead of by
+ * tiles (both softmax groups on every tile, 32 columns each, nothing merged per row: about half the per-row cost,
+ * slightly more per tile — faster where most lists are short, e.g. threshold masks: 7.2 against 8.9 ms at 65 536
+ * tokens and 92 % sparsity; 3 % slower at 131 072 tokens with TopK 1/10).  Returns SEER_ERR_INVALID_ARG for other
+ * values. */
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);
 
 /* Synchronises `stream`, returns the device status word (SEER_OK if nothing was raised) and clears it. */

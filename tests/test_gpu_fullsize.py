@@ -130,8 +130,9 @@ def test_threshold_workloads_full_size(rt, name, heads):
     check_workload(rt, name, [spec], sample_heads=heads, rows_per_head=2)
 
 
-def test_c3_bench_configuration_all_rows_cross_check(rt):
-    """Every output row of the bench workload, not a sample: the tcgen05 kernel against the independent mma.sync kernel
+@pytest.mark.parametrize("impl", [0, 3])
+def test_c3_bench_configuration_all_rows_cross_check(rt, impl):
+    """Every output row of the bench workload, not a sample: each tcgen05 kernel against the independent mma.sync kernel
     (different tiling, layout and softmax scheme; itself checked against the oracle on the small cases) on the same
     lists.  Both round P and o to bf16, so the bound is the attention tolerance between two results of that kind."""
     import torch
@@ -139,7 +140,11 @@ def test_c3_bench_configuration_all_rows_cross_check(rt):
     w = W.make_workload("c3")
     p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx)
     p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
-    p.run(B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=10, flags=3))
+    B.seer_set_attn_impl(ctx, impl)
+    try:
+        p.run(B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=10, flags=3))
+    finally:
+        B.seer_set_attn_impl(ctx, 0)
     assert p.status() == 0
     o_tc = p.o.float().clone()
     lse_tc = p.lse.clone()

@@ -118,7 +118,11 @@ def test_random_shape_all_features(rt, seed):
     p = Prefill(w.cu_seqlens, hq, hkv, ctx=ctx, want_lse=True, block=blk)
     p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
     p.o.fill_(float("nan"))
-    p.gate_ex(opt, wq_d, wk_d); p.mask(params); p.attn()
+    B.seer_set_attn_impl(ctx, 3 if seed % 2 else 0)      # the two tcgen05 kernels take turns
+    try:
+        p.gate_ex(opt, wq_d, wk_d); p.mask(params); p.attn()
+    finally:
+        B.seer_set_attn_impl(ctx, 0)
     assert p.status() == 0, what
     got = O.unflatten_scores(p.scores_host(), w.cu_seqlens, blk, hq)
     ref = O.gate_scores_ex(w.q, w.k, wq, wk, w.cu_seqlens, blk, pool_q=pq, pool_k=pk, rope_theta=theta)
@@ -152,8 +156,8 @@ def test_random_shape_all_features(rt, seed):
 def test_random_lists_on_data_that_moves_the_softmax_references(rt, seed):
     """Random lists (odd lengths, rows without their diagonal block, empty rows) on inputs built to exceed the running
     softmax references again and again: key norms that grow along the sequence, a few huge outlier keys, queries of very
-    different scales, strongly negative logits followed by a late positive block.  Both attention kernels against the
-    oracle."""
+    different scales, strongly negative logits followed by a late positive block.  All three attention kernels against
+    the oracle."""
     B, Prefill, ctx = rt
     rng = np.random.default_rng(555_000 + seed)
     lens = [int(rng.integers(300, 2500)) for _ in range(int(rng.integers(1, 3)))]
@@ -185,7 +189,7 @@ def test_random_lists_on_data_that_moves_the_softmax_references(rt, seed):
     o_ref, lse_ref = O.sparse_attention(q, k, w.v, w.cu_seqlens, rp, col, hq, 1, 64, 1 / math.sqrt(128))
     fin = np.isfinite(lse_ref)
     try:
-        for impl in (0, 1):
+        for impl in (0, 1, 3):
             B.seer_set_attn_impl(ctx, impl)
             p.o.fill_(float("nan"))
             p.attn()

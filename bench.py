@@ -496,7 +496,7 @@ def main():
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_desc(w, spec),
                "kept_blocks": nnz, "stage_ms": {"gate": gate_ms, "mask": mask_ms, "attn": attn_ms,
                                                 "attn_min": float(min(attn_all)), "attn_median": float(np.median(attn_all))},
-               "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape", 3: "tcgen05, softmax split by query columns"}[args.attn_impl],
+               "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape", 3: "tcgen05, softmax split by query columns", 4: "tcgen05, previous arrangement"}[args.attn_impl],
                "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
                             "frac": achieved / burst, "peak_source": f"bf16 dense burst, of {src}",
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,

@@ -198,7 +198,7 @@ seer_status seer_create(seer_ctx** out, int device) {
          cudaEventCreateWithFlags(&ctx->ev_comp[i], cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&ctx->ev_d2h[i], cudaEventDisableTiming) == cudaSuccess;
   if (ok) ok = init_gate(ctx) == SEER_OK && init_mask(ctx) == SEER_OK && init_attn_mma(ctx) == SEER_OK &&
-              init_attn_tc(ctx) == SEER_OK && init_attn_tc2(ctx) == SEER_OK;
+              init_attn_tc(ctx) == SEER_OK && init_attn_tc2(ctx) == SEER_OK && init_attn_tcs(ctx) == SEER_OK;
   if (!ok) { seer_destroy(ctx); return SEER_ERR_CUDA; }
   *out = ctx;
   return SEER_OK;
@@ -340,7 +340,8 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   const bool legacy = ctx->attn_impl == 1 || (ctx->attn_impl == 2 && t.causal_blocks <= 8 * t.rows);
   int n = legacy ? launch_attn_mma(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
           : ctx->attn_impl == 3 ? launch_attn_tc2(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
-                                : launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream);
+          : ctx->attn_impl == 4 ? launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
+                                : launch_attn_tcs(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream);
   finish_call(ctx, slot, stream);
   if (n < 0) return SEER_ERR_CUDA;
   ctx->launches += n;
@@ -513,7 +514,7 @@ seer_status seer_expand_block_lists(seer_ctx* ctx, const seer_shape* shape, cons
 }
 
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl) {
-  if (!ctx || impl < 0 || impl > 3) return SEER_ERR_INVALID_ARG;
+  if (!ctx || impl < 0 || impl > 4) return SEER_ERR_INVALID_ARG;
   ctx->attn_impl = impl;
   return SEER_OK;
 }

@@ -124,6 +124,9 @@ int launch_attn_tc2(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* 
                     const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
 seer_status init_attn_tc(seer_ctx* ctx);
 seer_status init_attn_tc2(seer_ctx* ctx);
+int launch_attn_tcs(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
+                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
+seer_status init_attn_tcs(seer_ctx* ctx);
 
 // Sequence that owns global block index gb: largest b with blk_off[b] <= gb (empty sequences are skipped).
 __device__ __forceinline__ int find_sequence(const int32_t* __restrict__ off, int batch, int x) {

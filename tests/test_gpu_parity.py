@@ -400,7 +400,7 @@ def test_attention_kernel_chosen_by_shape(rt):
             assert torch.equal(outs[2][0], outs[want][0]) and torch.equal(outs[2][1], outs[want][1])
             assert not torch.equal(outs[0][0], outs[1][0])                  # the two kernels round differently
         with pytest.raises(B.SeerError):
-            B.seer_set_attn_impl(ctx, 4)
+            B.seer_set_attn_impl(ctx, 9)
     finally:
         B.seer_set_attn_impl(ctx, 0)
 

@@ -43,6 +43,11 @@ constexpr float kFirstShift = 12.f; // ... and this far above the score of the s
 constexpr float kNoRef = -32768.f; // reference of a column that has not seen a key yet: the first visible score overflows it
 constexpr int kHelperRegs = 56, kSoftmaxRegs = 200;   // (2 * 56 + 2 * 200) * 128 = 65536
 constexpr int kGroupThreads = 128;
+// a helper thread that polls a barrier shares its scheduler with two softmax warps: it sleeps between polls
+constexpr int kProducerSleepNs = 128, kIssuerSleepNs = 0;
+// of every eight column pairs of a pass this many take their exponentials on the FMA pipe, the others on the
+// special-function unit (measured optimum of the pass alone: 3)
+constexpr int kPolyPairsOf8 = 3;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
 constexpr uint32_t kQBytes = 2 * kHalfQ;         // 16 KB
@@ -82,6 +87,13 @@ __device__ __forceinline__ uint64_t make_desc_ns(uint32_t saddr, uint32_t lbo_by
   return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46);
 }
 
+__device__ __forceinline__ bool mbar_test(uint32_t addr, uint32_t parity) {
+  uint32_t done;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+  return done != 0;
+}
+
 // The smallest bf16 number >= v (v finite), as a float.
 __device__ __forceinline__ float bf16_ceil(float v) {
   uint32_t b = __float_as_uint(v);
@@ -109,7 +121,7 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
 }
 
 // One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(sl2 * x), x = s - R[c] as the MMA left it.
-// Of every four columns two exponentials go to the special-function unit and two to the FMA pipe.
+// kPolyPairsOf8 of every eight column pairs take their exponentials on the FMA pipe, the others on the special-function unit.
 //   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the OR of the packed words: bit 14 or 30
 //                      set means some p >= 2, i.e. a score 2^(kRefShift + 1) above the maximum its reference was taken
 //                      from, or an infinity / NaN.
@@ -117,30 +129,28 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
 // MASKED applies the causal mask of a diagonal block, drops a dead row and the query columns past a ragged block.
 template <bool MASKED, bool SUBTRACT>
 __device__ __forceinline__ uint32_t tile_pass(uint32_t s_addr, float sl2, bool row_live, bool diag,
-                                              int key_local, int q_valid, float (&l)[64], uint32_t (&pk)[32], long long* dbg = nullptr) {
+                                              int key_local, int q_valid, float (&l)[64], uint32_t (&pk)[32], uint32_t early_bar = 0u,
+                                              uint32_t early_parity = 0u, bool* early_done = nullptr) {
   uint32_t ored = 0u;
   const float2 sl22 = make_float2(sl2, sl2);
-  long long dbg0 = 0;
-  if (dbg) dbg0 = clock64();
   // two TMEM round trips per pass: the second half is requested before the first is worked on
   uint32_t sv[2][32];
   tc_ld32(s_addr, sv[0]);
 #pragma unroll
   for (int ch = 0; ch < 2; ++ch) {
     tc_wait_ld32(sv[ch]);
-    if (dbg) { const long long n_ = clock64(); dbg[ch] += n_ - dbg0; dbg0 = n_; }
     if (ch == 0) tc_ld32(s_addr + 32, sv[1]);
+    // a barrier the caller needs after the pass is looked at here, so that the answer has arrived by then
+    if (ch == 1 && early_done != nullptr) *early_done = mbar_test(early_bar, early_parity);
     // stage by stage over the 32 columns, each stage a run of independent instructions, in place
     float2 v[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __fmul2_rn(make_float2(__uint_as_float(sv[ch][2 * i]), __uint_as_float(sv[ch][2 * i + 1])), sl22);
-#ifndef SEER_NO_EXP
 #pragma unroll
-    for (int i = 0; i < 16; i += 2) {
-      v[i] = make_float2(ex2f(v[i].x), ex2f(v[i].y));
-      v[i + 1] = exp2_poly2(v[i + 1]);
+    for (int i = 0; i < 16; ++i) {
+      if ((i & 7) < kPolyPairsOf8) v[i] = exp2_poly2(v[i]);
+      else v[i] = make_float2(ex2f(v[i].x), ex2f(v[i].y));
     }
-#endif
     if (MASKED) {
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
@@ -197,7 +207,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       mbar_init(sh.bar(b + V_EMPTY), 1);
       mbar_init(sh.bar(b + S_FULL), 1);
       mbar_init(sh.bar(b + S_FULL + 1), 1);
-      mbar_init(sh.bar(b + P_FULL), kGroupThreads / 32);      // one arrival per softmax warp
+      mbar_init(sh.bar(b + P_FULL), 1);                       // one arrival, after the softmax group has met
       mbar_init(sh.bar(b + PV_DONE), 1);
       mbar_init(sh.bar(b + FIXED), 1);
     }
@@ -245,7 +255,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const Item it = decode_item<kChunk>(m, row_ptr, w);
           if (it.ntiles == 0) continue;
           if (!is_v) {
-            if (!mbar_wait(sh, bb + Q_EMPTY, (nitem & 1u) ^ 1u, status)) break;
+            if (!mbar_wait<kProducerSleepNs>(sh, bb + Q_EMPTY, (nitem & 1u) ^ 1u, status)) break;
             mbar_expect_tx(sh.bar(bb + Q_FULL), kQBytes);
             const int tq = it.s0 + it.i * kBlock + (kChunk ? it.dq : 0);
             tma_load_3d(sbase + kStQ, &map_q, sh.bar(bb + Q_FULL), 0, it.h, tq);
@@ -257,7 +267,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
             if (!is_v && (ja == -2 || jb == -2)) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
             tr.sample(cnt); tr.ev(1, cnt);
-            if (!mbar_wait(sh, empty, (cnt & 1u) ^ 1u, status)) { ok = false; break; }
+            if (!mbar_wait<kProducerSleepNs>(sh, empty, (cnt & 1u) ^ 1u, status)) { ok = false; break; }
             tr.ev(2, cnt);
             const bool has_b = jb != -1;
             const int xa = ja < 0 ? 0 : ja, xb = jb < 0 ? 0 : jb;   // a rejected entry: any valid block, masked out in the softmax
@@ -294,7 +304,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         bool ok = true;
         // S^T of the next tile of the stream (ordinal cs) into buffer cs & 1: eight K-steps over d, a ninth that
         // subtracts the softmax references
-        auto issue_s = [&](bool last_of_item) -> bool {
+        auto issue_s = [&](bool last_of_item, bool with_refs) -> bool {
           tr.ev(10, cs);
           if (!mbar_wait(sh, bb + K_FULL, cs & 1u, status)) return false;
           tr.ev(11, cs);
@@ -306,7 +316,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int kk = 0; kk < 8; ++kk)
             tc_mma(d, desc_hi_k | (uint64_t)(klo + (uint32_t)((kk >> 2) * (kHalfKV >> 4) + (kk & 3) * 2)),
                    desc_hi_k | (uint64_t)(qlo + (uint32_t)((kk >> 2) * (kHalfQ >> 4) + (kk & 3) * 2)), kIdescS, kk > 0);
-          tc_mma(d, ones_d, qext_d, kIdescS, 1u);
+          if (with_refs) tc_mma(d, ones_d, qext_d, kIdescS, 1u);
           tc_commit(sh.bar(bb + S_FULL + (int)(cs & 1u)));
           tc_commit(sh.bar(bb + K_EMPTY));
           if (last_of_item) tc_commit(sh.bar(bb + Q_EMPTY));   // last S^T of the item: Q may be replaced
@@ -320,15 +330,18 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tr.sample(cs);
           if (!mbar_wait(sh, bb + Q_FULL, nitem & 1u, status)) break;
           ++nitem;
-          if (!issue_s(it.ntiles == 1)) break;
-          if (it.ntiles > 1 && !issue_s(it.ntiles == 2)) break;
+          // the first two tiles of an item are computed without references (the row still holds those of the previous
+          // item, and a result must not depend on which item came before): the group subtracts its first references
+          // from them in place
+          if (!issue_s(it.ntiles == 1, false)) break;
+          if (it.ntiles > 1 && !issue_s(it.ntiles == 2, false)) break;
           for (int t = 0; t < it.ntiles; ++t, ++cp) {
             tr.sample(cp); tr.ev(13, cp);
             if (!mbar_wait(sh, bb + V_FULL, cp & 1u, status)) { ok = false; break; }
             tr.ev(14, cp);
             // P^T of tile t is complete; the group has also finished with S^T buffer cp & 1 (and, at t = 0, with the
             // O^T accumulator of the previous item)
-            if (!mbar_wait(sh, bb + P_FULL, cp & 1u, status)) { ok = false; break; }
+            if (!mbar_wait<kIssuerSleepNs>(sh, bb + P_FULL, cp & 1u, status)) { ok = false; break; }
             tr.ev(15, cp);
             tc_fence_after();
             // 16 keys (2048 bytes of 128-byte rows) per step; an odd list leaves the second block of its last tile out
@@ -345,7 +358,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tc_commit(sh.bar(bb + V_EMPTY));
             tc_commit(sh.bar(bb + PV_DONE));
             tr.ev(16, cp);
-            if (t + 2 < it.ntiles && !issue_s(t + 3 == it.ntiles)) { ok = false; break; }
+            if (t + 2 < it.ntiles && !issue_s(t + 3 == it.ntiles, true)) { ok = false; break; }
           }
         }
         tr.flush();
@@ -406,10 +419,12 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
       int nja = list_block(it, col_idx, 0), njb = list_block(it, col_idx, 1);
       tr.ev(29, 0);
+      bool s_seen = false;                                  // S_FULL of the coming tile was already seen complete
       for (int t = 0; t < it.ntiles; ++t, ++cnt) {
         const uint32_t sbuf = cnt & 1u;
         if constexpr (kTrace) { seg_last = clock64(); ++seg_n; }
-        bool fail = !mbar_wait(sh, bb + S_FULL + (int)sbuf, (cnt >> 1) & 1u, status);
+        bool fail = false;
+        if (!s_seen) fail = !mbar_wait(sh, bb + S_FULL + (int)sbuf, (cnt >> 1) & 1u, status);
         SEG(0);
         tc_fence_after();
         const int ja = nja, jb = njb;
@@ -446,8 +461,8 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tc_fence_before();
           if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
           if (gt < 64) {
-            const float old = rcur[gt];
-            float nr = bf16_ceil(lsum[gt] + old + kFirstShift / sl2);
+            const float old = 0.f;                       // the first two S^T tiles of an item hold the raw scores
+            float nr = bf16_ceil(lsum[gt] + kFirstShift / sl2);
             if (gt >= it.q_valid || !(fabsf(nr) < 3.0e38f)) nr = old;   // not a column of this block / not a finite score
             const float d = old - nr;
             rcur[gt] = nr;
@@ -473,16 +488,34 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         // without references (the first key of the first tile is not a valid entry) the tile goes straight to the rebase
         uint32_t over = 0x40004000u;
+        bool pv_seen = t == 0;                           // the P V of the previous tile has finished: the P^T buffer is free, O^T at rest
         if (!fail && have_ref)
           over = masked ? tile_pass<true, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk)
-                        : tile_pass<false, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk, kTrace ? &seg[8] : nullptr);
+                        : tile_pass<false, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk,
+                                                  sh.bar(bb + PV_DONE), (cnt - 1) & 1u, t >= 1 ? &pv_seen : nullptr);
         SEG(1);
         nja = list_check(it, 2 * t + 2, raw_a); njb = list_check(it, 2 * t + 3, raw_b);
         SEG(2);
-        // the P^T buffer is free (and O^T at rest) when the P V of the previous tile has finished
-        if (!fail && t >= 1) fail = !mbar_wait(sh, bb + PV_DONE, (cnt - 1) & 1u, status);
+        if (!fail && !pv_seen) fail = !mbar_wait(sh, bb + PV_DONE, (cnt - 1) & 1u, status);
         SEG(3);
-        // one vote per tile: does any entry reach 2^(kRefShift + 1) times its reference maximum (or has a wait been lost)?
+        // P^T is stored at once; the vote on the tile (does any entry reach 2^(kRefShift + 1) times its reference
+        // maximum, or has a wait been lost?) comes after the stores, where the group has to meet anyway, and the
+        // issuer is told only after it
+        auto store_p = [&]() {
+          const uint32_t prow = p_base + (uint32_t)r * 128u;
+#pragma unroll
+          for (int ck = 0; ck < 8; ++ck) {
+            const uint32_t a = prow + (uint32_t)((ck ^ (r & 7)) << 4);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(pk[ck * 4]), "r"(pk[ck * 4 + 1]),
+                         "r"(pk[ck * 4 + 2]), "r"(pk[ck * 4 + 3]) : "memory");
+          }
+        };
+        store_p();
+        SEG(6);
+        // the next tile's S^T: asked now, looked at when the next tile starts
+        s_seen = t + 1 < it.ntiles && mbar_test(sh.bar(bb + S_FULL + (int)(sbuf ^ 1u)), ((cnt + 1) >> 1) & 1u);
+        fence_async_smem();
+        tc_fence_before();
         const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
         SEG(4);
         if (slow) {
@@ -520,7 +553,7 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tc_fence_before();                             // this thread's reads of the S^T buffer are done
           named_bar_sync(bar_sync, kGroupThreads);
           if (gt < 64) {
-            const float old = rcur[gt];
+            const float old = have_ref ? rcur[gt] : 0.f;   // (an item's first tiles hold the raw scores)
             // largest raw score of the column in this tile
             const float cm = fmaxf(fmaxf(lsum[gt], lsum[64 + gt]), fmaxf(lsum[128 + gt], lsum[192 + gt])) + old;
             float nr;
@@ -585,25 +618,16 @@ attn_tcs_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tc_fence_after();
           if (masked) tile_pass<true, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk);
           else tile_pass<false, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk);
+          store_p();
+          fence_async_smem();
+          tc_fence_before();
+          named_bar_sync(bar_sync, kGroupThreads);
+          s_seen = false;
           SEG(14);
         }
         SEG(5);
-        // P^T row r (128-byte swizzle)
-        {
-          const uint32_t prow = p_base + (uint32_t)r * 128u;
-#pragma unroll
-          for (int ck = 0; ck < 8; ++ck) {
-            const uint32_t a = prow + (uint32_t)((ck ^ (r & 7)) << 4);
-            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(pk[ck * 4]), "r"(pk[ck * 4 + 1]),
-                         "r"(pk[ck * 4 + 2]), "r"(pk[ck * 4 + 3]) : "memory");
-          }
-        }
-        SEG(6);
-        fence_async_smem();
-        // one arrival per warp (128 would serialise on the barrier word); it also hands the S^T buffer back
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sh.bar(bb + P_FULL));
+        // every thread's stores are visible to the MMA: one arrival hands P^T over and the S^T buffer back
+        if (gt == 0) mbar_arrive(sh.bar(bb + P_FULL));
         SEG(7);
       }
       if (!ok) break;

@@ -10,7 +10,8 @@ blocks (90 % block sparsity), diagonal and sink forced.  Prints ONE JSON line on
 value  = kept-block attention FLOPs (4 * 64 * 64 * 128 per kept block) of all ranks / step time, inputs resident in HBM.
 e2e    = same, through seer_prefill_host: pinned host buffers in, pinned host buffer out, copies inside the timed region.
 roofline = the attention kernel alone (CUDA events around its launch) against the measured bf16 dense peak.
-cpu_baseline = the fp64 CPU oracle's attention on a sample of rows of the same workload, on this machine's host cores.
+cpu_baseline = the fp64 CPU oracle on this machine's host cores: gate and mask in full, attention on a sample of rows of
+               the same workload (measured, and extrapolated to all kept blocks).
 """
 from __future__ import annotations
 
@@ -28,6 +29,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 FLOP_PER_BLOCK = 4 * 64 * 64 * 128
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of the default command, and the capture it is from
+TRAFFIC_C3_KEEP10 = (None, "not captured yet")
 METRIC = "sparse_prefill_attention_effective_tflops_128k_90pct_block_sparsity"
 
 
@@ -40,7 +43,11 @@ def parse():
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--keep", default="1/10", help="TopK ratio for the c3 workload")
     ap.add_argument("--seq", type=int, default=None, help="override the sequence length (profiling on a smaller case)")
-    ap.add_argument("--attn-impl", type=int, default=0, help="0 tcgen05 kernel, 1 mma.sync kernel, 2 chosen per call from the shape, 3 tcgen05 kernel split by query columns")
+    ap.add_argument("--attn-impl", type=int, default=0, choices=[0, 1, 2], help="0 tcgen05 kernel, 1 mma.sync kernel, 2 chosen per call from the shape")
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="also time the other four workloads (and the other TopK ratios of c3) and add the table as `all_workloads`")
+    ap.add_argument("--timeline", action="store_true",
+                    help="one extra attention launch of the instrumented kernel; adds `timeline` (per role: clocks per tile in each step of its loop, CTA 0) to the line")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-list run of the attention kernel")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true")
@@ -155,8 +162,9 @@ class ClockSampler:
                 "load_extended_for_sampling": self.extended}
 
 
-def cpu_oracle_sample(w, rp, col, budget_rows=None):
-    """Times the oracle's attention on a sample of (head, query-block) rows.  Returns (tflops, seconds, description, cores)."""
+def cpu_oracle_sample(w, spec, rp, col, budget_rows=None):
+    """Times the oracle as it stands: gate and mask in full, attention on a sample of (head, query-block) rows.
+    Returns the `cpu_baseline` object."""
     from oracle import seer_oracle as O
     from paper_2410_13276_b200 import workloads as W
     rows = W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=1234, per_head_random=56)   # ~1900 rows, about 10 s of CPU work
@@ -166,8 +174,93 @@ def cpu_oracle_sample(w, rp, col, budget_rows=None):
     t0 = time.perf_counter()
     O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64, w.softmax_scale, rows=rows)
     dt = time.perf_counter() - t0
+    total = int(rp[-1])
+    t0 = time.perf_counter()
+    sc = O.gate_scores(w.q, w.k, w.wq, w.wk, w.cu_seqlens, 64)
+    gate_s = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    O.block_mask(sc, spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                 threshold=spec.threshold or 0.0, flags=spec.flags)
+    mask_s = time.perf_counter() - t0
+    del sc
     cores = len(os.sched_getaffinity(0))
-    return blocks * FLOP_PER_BLOCK / dt / 1e12, dt, f"oracle attention on {len(rows)} sampled (head, query-block) rows = {blocks} kept blocks; gate and mask oracle not included", cores
+    return {"value": blocks * FLOP_PER_BLOCK / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+            "sample": f"oracle attention on {len(rows)} sampled (head, query-block) rows = {blocks} of {total} kept blocks; "
+                      "gate and mask oracle in full",
+            "seconds": dt, "attn_ms_extrapolated": 1e3 * dt * total / max(blocks, 1), "gate_ms": 1e3 * gate_s,
+            "mask_ms": 1e3 * mask_s}
+
+
+TIMELINE_TAGS = {1: "loop", 2: "wait for an empty K / V buffer", 10: "before S^T", 11: "wait K_FULL", 12: "S^T MMAs + commits",
+                 13: "before P V", 14: "wait V_FULL", 15: "wait P_FULL", 16: "P V MMAs + commits",
+                 29: "item start (decode, first list entries)", 30: "tile loop of an item (all tiles)", 31: "epilogue",
+                 32: "wait S_FULL", 33: "softmax pass (incl. first-tile references)", 34: "next list entries",
+                 35: "wait PV_DONE", 36: "fence + vote", 37: "(branch)", 38: "P^T stores", 39: "arrive P_FULL",
+                 40: "rebase: wait next S^T + vote", 41: "rebase: TMEM reads", 42: "rebase: column maxima (shuffles)",
+                 43: "rebase: new references", 44: "rebase: fix MMAs, rescale", 45: "rebase: wait FIXED", 46: "rebase: pass + stores"}
+TIMELINE_ROLES = ["producer K+Q, stream 0", "issuer, stream 0", "producer V, stream 0", "issuer, stream 1",
+                  "softmax group, stream 0", "softmax group, stream 1"]
+
+
+def attention_timeline(p, B, torch):
+    """One attention launch with the trace buffer set: the instrumented instantiation accumulates, for CTA 0, the
+    clocks each role spends in each step of its loop (softmax groups: every tile; helpers: every eighth tile)."""
+    buf = torch.zeros(7 * 8192, dtype=torch.int64, device="cuda")
+    B.seer_set_trace_buffer(p.ctx, buf)
+    try:
+        p.attn(); torch.cuda.synchronize()
+    finally:
+        B.seer_set_trace_buffer(p.ctx, None)
+    t = buf.cpu().numpy().astype(np.uint64)
+    roles = {}
+    for r, name in enumerate(TIMELINE_ROLES):
+        a = t[r * 8192: r * 8192 + 96].reshape(48, 2).astype(np.int64)
+        roles[name] = {TIMELINE_TAGS.get(tag, str(tag)): {"events": int(a[tag, 1]), "clocks_per_event": float(a[tag, 0]) / float(a[tag, 1])}
+                       for tag in range(48) if a[tag, 1]}
+    n = int((t[6 * 8192 + 256: 6 * 8192 + 512] != 0).sum())
+    clk = t[6 * 8192 + 256: 6 * 8192 + 256 + n].astype(np.int64)
+    return {"cta0_roles": roles, "cta_wall_clocks": {"ctas": n, "min": int(clk.min()), "median": int(np.median(clk)), "max": int(clk.max())}}
+
+
+def time_workload(name, keep, args, local, B, W, Prefill, torch, burst):
+    """gate / mask / attention / dense-list attention of one workload (3 warm-ups, 8 timed steps, medians)."""
+    w = W.make_workload(name)
+    a2 = argparse.Namespace(**vars(args)); a2.keep = keep or "1/10"
+    spec = pick_mask(w, a2)
+    p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, device=local, want_lse=False)
+    B.seer_set_attn_impl(p.ctx, args.attn_impl)
+    p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
+    params = B.make_mask_params(spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
+                                threshold=spec.threshold or 0.0, flags=spec.flags)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda") if input_bytes(w) <= 2 * L2_BYTES else None
+    for _ in range(3):
+        p.run(params)
+    torch.cuda.synchronize()
+    nnz = int(p.nnz.item())
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(8)]
+    for s in range(8):
+        if flush is not None:
+            flush.fill_(s)
+        ev[s][0].record(stream); p.gate(); ev[s][1].record(stream); p.mask(params); ev[s][2].record(stream); p.attn(); ev[s][3].record(stream)
+    torch.cuda.synchronize()
+    g, mk, at = (float(np.median([e[i].elapsed_time(e[i + 1]) for e in ev])) for i in range(3))
+    dparams = B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=1, flags=B.SEER_FORCE_DIAG)
+    p.mask(dparams); p.attn(); torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if flush is not None:
+        flush.fill_(1)
+    a.record(stream); p.attn(); b.record(stream); torch.cuda.synchronize()
+    dense_ms = a.elapsed_time(b)
+    dense_blocks = B.seer_causal_blocks(p.shape)
+    status = p.status()
+    out = {"workload": name, "mask": workload_desc(w, spec)["mask"], "tokens": int(w.total_tokens), "kept_blocks": nnz,
+           "gate_ms": g, "mask_ms": mk, "attn_ms": at, "attn_tflops": nnz * FLOP_PER_BLOCK / (at * 1e-3) / 1e12,
+           "attn_frac_of_burst_peak": nnz * FLOP_PER_BLOCK / (at * 1e-3) / 1e12 / burst,
+           "dense_attn_ms": dense_ms, "dense_tflops": dense_blocks * FLOP_PER_BLOCK / (dense_ms * 1e-3) / 1e12,
+           "speedup_over_dense": dense_ms / at, "l2_flushed": flush is not None, "device_status": status}
+    p.ctx.close()
+    return out
 
 
 def seeded_lists_for_rows(w, spec, rows, seed=99):
@@ -315,6 +408,19 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         total_ms = float(t.item())
     ms_step = total_ms / args.steps
+    # the gate's bandwidth-bound first kernel (pooling + projection) on its own, outside the timed region
+    gate_pool_ms = None
+    if rank == 0:
+        for _ in range(3):
+            p.gate_project()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(10):
+            p.gate_project()
+        b.record(stream); torch.cuda.synchronize()
+        gate_pool_ms = a.elapsed_time(b) / 10
+        p.gate(); p.mask(params)
     gate_ms = float(np.median([e[0].elapsed_time(e[1]) for e in ev]))
     mask_ms = float(np.median([e[1].elapsed_time(e[2]) for e in ev]))
     attn_all = [e[2].elapsed_time(e[3]) for e in ev]
@@ -453,6 +559,20 @@ def main():
         block_max_ms = a.elapsed_time(b)
         p.lse = None; p.bmax = None
 
+    # the kernel's own timeline: one launch of the instrumented instantiation (CTA 0; clocks per tile by role and step)
+    timeline = None
+    if rank == 0 and args.timeline:
+        timeline = attention_timeline(p, B, torch)
+
+    # the other workloads (and the other TopK ratios of c3), outside the timed region: gate, mask, attention, dense lists
+    all_wl = None
+    if rank == 0 and args.all_workloads:
+        all_wl = []
+        burst = peaks()[0]
+        for name, keep in (("c1", None), ("c2", None), ("c3", "1/2"), ("c3", "1/4"), ("c3", "1/10"), ("c3", "1/20"),
+                           ("c4", None), ("c5", None)):
+            all_wl.append(time_workload(name, keep, args, local, B, W, Prefill, torch, burst))
+
     # end to end through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
@@ -486,25 +606,31 @@ def main():
     if rank == 0:
         burst, sustained, hbm, src = peaks()
         achieved = flops / (attn_ms * 1e-3) / 1e12
+        gate_pool_bytes = (w.num_q_heads + w.num_kv_heads) * (w.total_tokens * 256 + int(sum(w.num_blocks)) * 768)
+        mask_bytes = (B.seer_causal_blocks(p.shape) + nnz + B.seer_mask_rows(p.shape)) * 4
         # DRAM bytes of one attention launch from an ncu capture of this very command
         # (profiles/attn_tc_kernel_c3_seq131072_keep10_dram.md); other workloads have no capture
-        traffic = None
+        traffic, traffic_source = None, "no ncu capture for this command"
         if w.name == "c3" and args.seq is None and (spec.keep_num, spec.keep_den) == (1, 10) and args.attn_impl == 0:
-            traffic = 5.16e9
+            traffic, traffic_source = TRAFFIC_C3_KEEP10
         out = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_desc(w, spec),
                "kept_blocks": nnz, "stage_ms": {"gate": gate_ms, "mask": mask_ms, "attn": attn_ms,
                                                 "attn_min": float(min(attn_all)), "attn_median": float(np.median(attn_all))},
-               "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape", 3: "tcgen05, softmax split by query columns", 4: "tcgen05, previous arrangement"}[args.attn_impl],
+               "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape"}[args.attn_impl],
                "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
                             "frac": achieved / burst, "peak_source": f"bf16 dense burst, of {src}",
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,
-                            "kernel": "seer_sparse_attn"},
+                            "traffic_source": traffic_source, "kernel": "seer_sparse_attn"},
                "gate_gbs": ((w.num_q_heads + w.num_kv_heads) * w.total_tokens * 256) / (gate_ms * 1e-3) / 1e9,
+               # pooling + projection alone: Q and K read once, 768 bytes written per (head, block); against the measured copy bandwidth
+               "gate_pool_ms": gate_pool_ms,
+               "gate_pool_gbs": gate_pool_bytes / (gate_pool_ms * 1e-3) / 1e9,
+               "gate_pool_frac": gate_pool_bytes / (gate_pool_ms * 1e-3) / 1e9 / hbm,
                # mask builder: every causal score read once, every kept block and row offset written once (algorithmic bytes)
-               "mask_gbs": ((B.seer_causal_blocks(p.shape) + nnz + B.seer_mask_rows(p.shape)) * 4) / (mask_ms * 1e-3) / 1e9,
-               "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128, "chunked_prefill": chunked, "list_stats": list_stats,
+               "mask_gbs": mask_bytes / (mask_ms * 1e-3) / 1e9, "mask_frac": mask_bytes / (mask_ms * 1e-3) / 1e9 / hbm,
+               "all_workloads": all_wl, "timeline": timeline, "gate_variant": gate_var, "block_max_ms": block_max_ms, "fused_gate_mask": fused, "block128": block128, "chunked_prefill": chunked, "list_stats": list_stats,
                "gpu_launches": int(launches), "clocks": clocks, "e2e": e2e}
         if dense_ms:
             dense_blocks = B.seer_causal_blocks(p.shape)
@@ -512,9 +638,7 @@ def main():
                             "speedup_sparse_over_dense": dense_ms / attn_ms}
         if not args.no_cpu:
             rp, col = p.lists_host()
-            v, dt, desc, cores = cpu_oracle_sample(w, rp, col)
-            out["cpu_baseline"] = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc,
-                                   "seconds": dt}
+            out["cpu_baseline"] = cpu_oracle_sample(w, spec, rp, col)
         print(json.dumps(out))
     if world > 1:
         dist.barrier()

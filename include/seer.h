@@ -10,8 +10,15 @@
  *    enqueued by the call has completed on `stream`.  `cu_seqlens_host` and the parameter structs are
  *    HOST memory and are consumed before the call returns.
  *  - Calls enqueue kernels on `stream` (a cudaStream_t passed as void*; NULL = default stream) and return
- *    without synchronising.  The library allocates device memory only in seer_create; per-call scratch
- *    comes from the caller's workspace `ws` (>= seer_workspace_bytes(shape), 256-byte aligned).
+ *    without synchronising, with one exception: the context keeps the batch metadata (sequence offsets) of the
+ *    8 most recent shapes on the device; a call with a ninth shape reuses the least recently used entry whose
+ *    work has finished, and only if all 8 are still in flight does it wait on the host for the oldest one.
+ *    The library allocates device memory only in seer_create; per-call scratch comes from the caller's
+ *    workspace `ws` (>= seer_workspace_bytes(shape), 256-byte aligned).
+ *  - The tcgen05 attention kernel takes all 512 tensor-memory columns and 215 KB of shared memory of an SM, so
+ *    one CTA is resident per SM and its tensor-memory allocation cannot wait on another CTA of this library.  A
+ *    kernel of ANOTHER library that holds tensor memory on the same device at the same time (another stream or
+ *    process) can make that allocation wait; it is the one wait in the kernel the library cannot bound.
  *  - Nothing throws across the ABI.  Host-detectable errors are returned at once and enqueue nothing.
  *    Errors only the device can see (list capacity exceeded, a list entry out of range, a bounded wait
  *    that ran out) are recorded in a status word owned by the context; the offending work is skipped and
@@ -104,10 +111,18 @@ int64_t seer_causal_blocks(const seer_shape* shape);  /* num_q_heads * sum_b nb_
 /* 1. AttnGate (Sec. 3.1, Eq. 1): score = softmax((Pq(Q) Wq)(Pk(K) Wk)^T / sqrt(gate_dim)).
  *    Pq, Pk: average pooling over non-overlapping blocks of `block` tokens (a ragged last block averages the
  *    tokens it has).  The softmax of row i runs over the causal blocks j <= i, so each row sums to 1.
- *    All gate arithmetic is fp32.  Writes `scores` (layout above). */
+ *    Pooling, projection and the softmax are fp32; the logits are fp32-grade products of the projected vectors
+ *    (each split into three bf16 terms, six tensor-core products accumulated in fp32: what is dropped is below
+ *    2^-24 of the product).  Writes `scores` (layout above). */
 seer_status seer_gate_scores(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k,
                              const float* Wq, const float* Wk, float* scores, void* ws, size_t ws_bytes,
                              void* stream);
+
+/* The first half of call 1 alone (Sec. 3.1, Eq. 1: the pooling P(.) and the linear layers W): pools Q and K per block
+ * and projects the pooled vectors; the result stays in `ws` (>= seer_workspace_bytes) in the library's internal
+ * layout.  The bandwidth-bound stage of the gate, exported so that it can be timed on its own. */
+seer_status seer_gate_project(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k,
+                              const float* Wq, const float* Wk, void* ws, size_t ws_bytes, void* stream);
 
 enum { SEER_TOPK_RATIO = 0, SEER_TOPK_COUNT = 1, SEER_THRESHOLD = 2 };
 enum { SEER_FORCE_DIAG = 1u, SEER_FORCE_SINK = 2u };
@@ -157,15 +172,19 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
 
 /* Selects the attention kernel used by seer_sparse_attn: 0 = tcgen05 / TMEM / TMA kernel (default),
  * 1 = mma.sync kernel (on-device cross-check; also the faster one for very short lists), 2 = chosen per call from
- * the shape: the persistent tcgen05 kernel pays about 10 us per (head, query block) row whatever its list length, the
- * mma.sync kernel about 3.5 us plus more per block, so batches whose rows have at most 8 causal blocks on average
- * (many short sequences) go to the mma.sync kernel and everything else to the tcgen05 kernel (measured crossover:
- * 8.5 listed blocks per row); 3 = the tcgen05 kernel with the softmax work split by query columns instead of by
- * tiles (both softmax groups on every tile, 32 columns each, nothing merged per row: about half the per-row cost,
- * slightly more per tile — faster where most lists are short, e.g. threshold masks: 7.2 against 8.9 ms at 65 536
- * tokens and 92 % sparsity; 3 % slower at 131 072 tokens with TopK 1/10).  Returns SEER_ERR_INVALID_ARG for other
- * values. */
+ * the shape: the persistent tcgen05 kernel pays a few microseconds per (head, query block) row whatever its list
+ * length, so batches whose rows have at most 8 causal blocks on average (many short sequences) go to the mma.sync
+ * kernel and everything else to the tcgen05 kernel.  Returns SEER_ERR_INVALID_ARG for other values. */
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl);
+
+/* Test hook for the bounded waits of the tcgen05 attention kernel (no counterpart in the paper).  Every barrier
+ * wait in that kernel gives up after wait_limit_us microseconds (default 2 000 000): the thread raises
+ * SEER_ERR_TIMEOUT on the device status, sets a flag that every other role of its CTA polls, the CTA lets the copies
+ * and MMAs in flight land, frees its tensor memory and returns; rows it had not finished are not written.
+ * lose_v_copy_of_tile >= 0 makes exactly one wait run out: the first stream of CTA 0 never issues the V copy of its
+ * tile with that ordinal (counted over the CTA's work items from 0), so the MMA issuer's wait for it expires;
+ * nothing faults and the context stays usable.  -1 switches the hook off.  wait_limit_us = 0 is rejected. */
+seer_status seer_debug_lost_wait(seer_ctx* ctx, uint32_t wait_limit_us, int32_t lose_v_copy_of_tile);
 
 /* Synchronises `stream`, returns the device status word (SEER_OK if nothing was raised) and clears it. */
 seer_status seer_poll_device_status(seer_ctx* ctx, void* stream);

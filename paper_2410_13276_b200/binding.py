@@ -25,7 +25,7 @@ STATUS_NAMES = ["SEER_OK", "SEER_ERR_INVALID_ARG", "SEER_ERR_UNSUPPORTED", "SEER
 # every symbol include/seer.h declares
 EXPORTS = ["seer_create", "seer_destroy", "seer_status_string", "seer_workspace_bytes", "seer_scores_elems",
            "seer_mask_rows", "seer_causal_blocks", "seer_gate_scores", "seer_block_mask", "seer_sparse_attn",
-           "seer_set_attn_impl", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
+           "seer_gate_project", "seer_set_attn_impl", "seer_debug_lost_wait", "seer_poll_device_status", "seer_launch_count", "seer_prefill_host_arena_bytes",
            "seer_prefill_host", "seer_set_trace_buffer", "seer_gate_scores_static", "seer_gate_scores_ex",
            "seer_attn_block_max", "seer_gate_mask_workspace_bytes", "seer_gate_block_mask",
            "seer_expand_block_lists"]
@@ -83,12 +83,16 @@ def load_library() -> C.CDLL:
     lib.seer_causal_blocks.restype = i64
     lib.seer_gate_scores.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.seer_gate_scores.restype = C.c_int
+    lib.seer_gate_project.argtypes = [vp, shp, vp, vp, vp, vp, vp, sz, vp]
+    lib.seer_gate_project.restype = C.c_int
     lib.seer_block_mask.argtypes = [vp, shp, vp, C.POINTER(seer_mask_params), vp, vp, i64, vp, vp, sz, vp]
     lib.seer_block_mask.restype = C.c_int
     lib.seer_sparse_attn.argtypes = [vp, shp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.seer_sparse_attn.restype = C.c_int
     lib.seer_set_attn_impl.argtypes = [vp, C.c_int]
     lib.seer_set_attn_impl.restype = C.c_int
+    lib.seer_debug_lost_wait.argtypes = [vp, C.c_uint32, C.c_int32]
+    lib.seer_debug_lost_wait.restype = C.c_int
     lib.seer_poll_device_status.argtypes = [vp, vp]
     lib.seer_poll_device_status.restype = C.c_int
     lib.seer_launch_count.argtypes = [vp]
@@ -208,6 +212,12 @@ def seer_gate_scores(ctx: Context, shape: seer_shape, q, k, wq, wk, scores, ws, 
                                      _ptr(ws), ws_bytes, _stream(stream)), "seer_gate_scores")
 
 
+def seer_gate_project(ctx: Context, shape: seer_shape, q, k, wq, wk, ws, stream=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(ctx._lib.seer_gate_project(ctx.handle, C.byref(shape), _ptr(q), _ptr(k), _ptr(wq), _ptr(wk), _ptr(ws), ws_bytes,
+                                      _stream(stream)), "seer_gate_project")
+
+
 def seer_gate_scores_ex(ctx: Context, shape: seer_shape, options: seer_gate_options, q, k, wq, wk, scores, ws,
                         stream=None) -> None:
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
@@ -266,6 +276,10 @@ def seer_sparse_attn(ctx: Context, shape: seer_shape, q, k, v, row_ptr, col_idx,
 
 def seer_set_attn_impl(ctx: Context, impl: int) -> None:
     _check(ctx._lib.seer_set_attn_impl(ctx.handle, impl), "seer_set_attn_impl")
+
+
+def seer_debug_lost_wait(ctx: Context, wait_limit_us: int = 2_000_000, lose_v_copy_of_tile: int = -1) -> None:
+    _check(ctx._lib.seer_debug_lost_wait(ctx.handle, wait_limit_us, lose_v_copy_of_tile), "seer_debug_lost_wait")
 
 
 def seer_poll_device_status(ctx: Context, stream=None) -> int:

@@ -1,452 +1,179 @@
-// Block-sparse causal GQA attention (Sec. 3.3) on the Blackwell tensor path: tcgen05.mma with TMEM accumulators,
-// TMA gathers of the listed K/V blocks, warp-specialised roles.
+// Block-sparse causal GQA attention (Sec. 3.3) on the Blackwell tensor path, two work items in flight per CTA.
 //
-// Orientation.  A query block is 64 rows but the full-rate MMA shape is M = 128, and every (head, query block) has its
-// own list, so rows of different work items cannot share an MMA.  The kernel therefore computes the transposed
-// problem: two listed KV blocks (128 keys) form the M dimension and the 64 queries the N dimension,
+// Orientation (as in every tcgen05 kernel of this library): a query block is 64 rows but the full-rate MMA shape is
+// M = 128, and every (head, query block) has its own list, so the kernel computes the transposed problem: two listed KV
+// blocks (128 keys) form the M dimension and the 64 queries the N dimension,
 //     S^T[128 keys x 64 q] = K_tile[128 x 128 d] * Q^T          (A, B K-major in shared memory)
 //     O^T[128 d x 64 q]   += V_tile^T[128 d x 128 keys] * P^T    (A, B MN-major in shared memory)
-// so every MMA row is useful for arbitrary lists (an odd list pads half a tile once).
 //
-// Softmax in this orientation: a thread owns one key row of S^T (64 query columns).  The per-query running reference
-// m[c] is only a scaling reference, not the exact maximum: p = 2^(s - m[c]); it sits 2^7 above the column maximum it was
-// taken from, and every lane keeps a copy of the 64 references in TMEM (a shared-memory read in the inner loop would
-// queue behind the tensor pipe's operand traffic).  As long as no entry of a tile reaches 2^8 times its reference
-// maximum -- seen as "some p >= 2" on the packed bf16 words -- the tile needs no cross-thread reduction at all;
-// otherwise the group computes exact column maxima (warp shuffles, then four values per column through shared memory),
-// moves the references, rescales its partial sums and the O accumulator, and recomputes the tile.  Row sums are
-// per-thread partials combined once per work item.
+// Softmax references ride in the MMA.  A thread owns a key row of S^T (64 query columns) and would need all 64
+// per-query references in every pass.  Instead the reference of column c, R[c] (a bf16 number in units of raw scores),
+// is subtracted by the tensor core: a ninth K-step multiplies a column of ones (A) by a row holding -R[c] (B, 2 KB,
+// written by the softmax group), so the accumulator holds s - R[c] and a pass is p = 2^(scale * x) with no per-column
+// operand: half the TMEM reads of a pass and no reference registers.  R[c] sits 2^7 above the largest score its column
+// had when it was taken; a tile whose entries all stay below 2 (seen on the packed bf16 words) needs no cross-thread
+// reduction.  Otherwise, and on the first tile of a work item, the group rebases: exact column maxima, new R, row sums
+// and O^T rescaled, the -R row rewritten.  The (at most two) S^T tiles already computed with the old row are corrected in
+// place by one more MMA each, issued by a thread of the group: ones x (R_old - R_new), the difference split into three
+// bf16 terms so that it is exact.
 //
-// Roles (512 threads): warp 0 = TMA producer for Q and K, warp 1 = TMEM owner + issuer of the S^T MMAs, warp 3 = issuer
-// of the P V MMAs (one thread can start a tcgen05.mma only every 64 clocks, so the two products are issued from two
-// threads), warps 4-7 and 8-11 = two softmax groups, warps 12-15 = cp.async producers for V (a warp keeps only ~14 KB of
-// cp.async in flight, so four share a tile).  After the dispatch the helper warpgroups shrink to 56 registers per thread
-// and the softmax warpgroups grow to 200 (setmaxnreg).  The tiles of a work item alternate between the groups (even
-// tiles -> A, odd -> B); each group keeps its own two S^T buffers, two P^T buffers, O^T accumulator, references and row
-// sums, and the epilogue merges the two partial results through their references.  One persistent CTA per SM walks the
-// work items (longest rows first within each KV head).  Every wait is bounded; a wait that runs out raises
-// SEER_ERR_TIMEOUT and the CTA drains and exits.
+// Arrangement.  A CTA runs two independent streams; a stream owns a whole work item (head, query block) from its first
+// tile to its stores: Q tile, K tile, V tile, P^T buffer, two S^T accumulators and one O^T accumulator in TMEM, its own
+// producer threads (K and Q; V), MMA-issuing thread and softmax warpgroup.  The streams never meet at a barrier: while
+// one sits in the first-tile rebase or the epilogue of its item, the other keeps the tensor pipe busy.  The issuing
+// thread of a stream starts S^T of tile t + 2 right after P V of tile t.  Roles (512 threads): warps 0 / 2 = TMA
+// producer of Q and K for stream 0 / 1, warps 1 / 3 = MMA issuer of stream 0 / 1 (warp 1 owns TMEM), warps 4-7 / 8-11
+// = softmax group of stream 0 / 1, warps 12 / 13 = TMA producer of V for stream 0 / 1.  K and V have producers of their
+// own because a copy takes ~700 clocks to land and each buffer is refilled as soon as its product has been read: one
+// producer thread per stream would hold the K copy back behind the wait for the V buffer.  Every wait is bounded; a
+// wait that runs out raises SEER_ERR_TIMEOUT and the CTA drains and exits.
 #include <cuda.h>
 #include <math_constants.h>
 
-#include <map>
-
-#include "seer_internal.cuh"
+#include "attn_tc_common.cuh"
 
 namespace seer {
 namespace tc {
 
-constexpr int kThreads = 512;               // warps 0-3: K(+Q) producer, S^T issuer, -, P V issuer; 4-7 / 8-11: softmax groups A / B; 12-15: V producers
-constexpr int kVProducerWarps = 4;
+using namespace tcc;
+
+constexpr int kThreads = 512;
 constexpr float kRefShift = 7.f;   // softmax references are kept this far (log2) above the column maxima they were taken from
-constexpr int kHelperRegs = 56, kSoftmaxRegs = 200;   // register split after the role dispatch: (2 * 56 + 2 * 200) * 128 = 65536
+constexpr float kFirstShift = 12.f; // ... and this far above the score of the single key an item's first references are taken from
+constexpr float kNoRef = -32768.f; // reference of a column that has not seen a key yet: the first visible score overflows it
+constexpr int kHelperRegs = 56, kSoftmaxRegs = 200;   // (2 * 56 + 2 * 200) * 128 = 65536
 constexpr int kGroupThreads = 128;
+// a helper thread that polls a barrier shares its scheduler with two softmax warps: it sleeps between polls
+constexpr int kProducerSleepNs = 128, kIssuerSleepNs = 0;
+// of every eight column pairs of a pass this many take their exponentials on the FMA pipe, the others on the
+// special-function unit (measured optimum of the pass alone: 3)
+constexpr int kPolyPairsOf8 = 3;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
 constexpr uint32_t kQBytes = 2 * kHalfQ;         // 16 KB
 constexpr uint32_t kKVBytes = 2 * kHalfKV;       // 32 KB (K or V tile of 128 keys)
-constexpr uint32_t kPBytes = 128 * 128;          // 16 KB  P^T [128 keys][64 q] bf16
-// shared memory map (offsets from a 1024-byte aligned base)
-constexpr int kKSlots = 2, kVSlots = 2;
-constexpr uint32_t kOffQ = 0;                                     // 16 KB
-constexpr uint32_t kOffK = kOffQ + kQBytes;                       // kKSlots x 32 KB ring
-constexpr uint32_t kOffV = kOffK + kKSlots * kKVBytes;            // kVSlots x 32 KB ring
-constexpr uint32_t kOffP = kOffV + kVSlots * kKVBytes;            // 4 x 16 KB: two per softmax group (the first also epilogue staging)
-constexpr uint32_t kOffGrp = kOffP + 4 * kPBytes;                 // per-group small arrays
-constexpr uint32_t kGrpMref = 0, kGrpAlpha = 256, kGrpColmax = 512, kGrpLfin = 768, kGrpLsum = 1024;   // lsum: 4 x 64 floats
+constexpr uint32_t kPBytes = 128 * 128;          // 16 KB  P^T [128 keys][64 q] bf16 (also the epilogue's staging)
+// shared memory map (offsets from a 1024-byte aligned base); the big buffers of a stream are contiguous
+constexpr uint32_t kStQ = 0, kStK = kQBytes, kStV = kStK + kKVBytes, kStP = kStV + kKVBytes;
+constexpr uint32_t kStreamBytes = kStP + kPBytes;                 // 96 KB
+constexpr uint32_t kOffOnes = 2 * kStreamBytes;                   // [128 x 16] bf16, columns 0..2 = 1 (no swizzle): 4 KB
+constexpr uint32_t kOffQext = kOffOnes + 4096;                    // per stream [64 x 16] bf16, column 0 = -R[c]: 2 KB
+constexpr uint32_t kOffQfix = kOffQext + 2 * 2048;                // per stream [64 x 16] bf16, columns 0..2 = R_old - R_new in three terms
+constexpr uint32_t kOffGrp = kOffQfix + 2 * 2048;                 // per-group small arrays
+constexpr uint32_t kGrpRcur = 0, kGrpAlpha = 256, kGrpLsum = 1024;   // lsum: 4 x 64 floats
 constexpr uint32_t kGrpBytes = 2048;
-constexpr uint32_t kOffW = kOffGrp + 2 * kGrpBytes;               // merge weights wA[64], wB[64]
-constexpr uint32_t kOffBar = kOffW + 512;                         // mbarriers
-constexpr uint32_t kNumBars = 28;
+constexpr uint32_t kOffBar = kOffGrp + 2 * kGrpBytes;             // mbarriers
+constexpr int kBarsPerStream = 12;
+constexpr uint32_t kNumBars = 2 * kBarsPerStream;
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag
 constexpr uint32_t kOffTrace = kOffMisc + 64;                     // diagnostics: 6 roles x 48 tags x (sum, count)
 constexpr uint32_t kSmemBytes = kOffTrace + 6 * 48 * 16 + 1024;   // + alignment slack
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
-enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2 /* + slot */, K_EMPTY = 5, V_FULL = 8, V_EMPTY = 10,
-           S_FULL = 12 /* + 2*group + buf */, S_EMPTY = 16, P_FULL = 20 /* + 2*group + buf */, PV_DONE = 24 /* + 2*group + buf */ };
+enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2, K_EMPTY = 3, V_FULL = 4, V_EMPTY = 5, S_FULL = 6 /* + buf */, P_FULL = 8,
+           PV_DONE = 9, FIXED = 10 };
 
 constexpr uint32_t kTmemCols = 512;
-__device__ __forceinline__ uint32_t col_s(int group, uint32_t buf) { return (uint32_t)group * 192u + buf * 64u; }
-__device__ __forceinline__ uint32_t col_o(int group) { return (uint32_t)group * 192u + 128u; }
-// the softmax references of a group, replicated in every lane (a shared-memory read in the inner loop queues behind the
-// operand traffic of the tensor pipe; a TMEM read does not)
-__device__ __forceinline__ uint32_t col_m(int group) { return 384u + (uint32_t)group * 64u; }
+// TMEM columns of a stream: two S^T accumulators, O^T
+__device__ __forceinline__ uint32_t col_s(int s, uint32_t buf) { return (uint32_t)s * 256u + buf * 64u; }
+__device__ __forceinline__ uint32_t col_o(int s) { return (uint32_t)s * 256u + 128u; }
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is declared lost
-
-// ------------------------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-
-struct Shared {
-  uint32_t base;         // 1024-aligned shared address
-  __device__ __forceinline__ uint32_t bar(int i) const { return base + kOffBar + 8u * (uint32_t)i; }
-  __device__ __forceinline__ uint32_t abort_flag() const { return base + kOffMisc + 8; }
-};
-
-__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t a) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_shared_u32(uint32_t a, uint32_t v) {
-  asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false after the limit (or when another role has already given up); the caller drains.
-template <int kSleepNs = 0>
-__device__ __forceinline__ bool mbar_wait(const Shared& sh, int bar, uint32_t parity, int* status) {
-  const uint32_t addr = sh.bar(bar);
-  {
-    uint32_t done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-    if (done) return true;
-  }
-  if (mbar_try(addr, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try(addr, parity)) return true;
-    if (kSleepNs > 0) __nanosleep(kSleepNs);   // a waiting helper must not take issue slots from the softmax warps of its scheduler
-    if ((it & 255u) == 0u) {
-      if (ld_shared_u32(sh.abort_flag()) != 0u) return false;
-      if (global_ns() - t0 > kWaitLimitNs) break;
-    }
-  }
-  st_shared_u32(sh.abort_flag(), 1u);
-  atomicCAS(status, 0, (int)SEER_ERR_TIMEOUT);
-  return false;
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-               : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr) : "memory");
-}
-// Waits for the loads of this thread; the loaded registers are in/out operands so that no use of them moves above it.
-__device__ __forceinline__ void tc_wait_ld8(uint32_t (&a)[8], uint32_t (&b)[8]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
-                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7])
-               :: "memory");
-}
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Same wait, with the loaded registers as in/out operands so that no use of them can be scheduled above it.
-__device__ __forceinline__ void tc_wait_ld(uint32_t (&r)[16]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :: "memory");
-}
-// No instruction: makes the registers of a load issued before the last wait depend on that wait.
-__device__ __forceinline__ void tc_tie(uint32_t (&r)[16]) {
-  asm volatile(""
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :: "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void named_bar_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-// CTA-subset OR reduction of a predicate over `threads` threads on barrier `id`
-__device__ __forceinline__ bool named_bar_or(int id, int threads, bool pred) {
-  uint32_t r;
-  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %3, 0;\n\tbar.red.or.pred q, %1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
-               : "=r"(r) : "r"(id), "r"(threads), "r"((uint32_t)pred) : "memory");
-  return r != 0;
-}
-
-// Shared-memory matrix descriptors (128-byte swizzle, descriptor version 1)
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 64
-constexpr uint32_t make_idesc(bool a_mn_major, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((64u >> 3) << 17) | ((128u >> 4) << 24);
-}
 constexpr uint32_t kIdescS = make_idesc(false, false);
 constexpr uint32_t kIdescPV = make_idesc(true, true);
 
+// shared-memory matrix descriptor without swizzle (K-major: 8 x 16-byte core matrices; lbo = distance between the two
+// 16-byte K chunks, sbo = distance between 8-row groups)
+__device__ __forceinline__ uint64_t make_desc_ns(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46);
+}
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+__device__ __forceinline__ bool mbar_test(uint32_t addr, uint32_t parity) {
+  uint32_t done;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+  return done != 0;
+}
+
+// The smallest bf16 number >= v (v finite), as a float.
+__device__ __forceinline__ float bf16_ceil(float v) {
+  uint32_t b = __float_as_uint(v);
+  if ((b & 0xffffu) != 0u) b = v >= 0.f ? ((b + 0x10000u) & 0xffff0000u) : (b & 0xffff0000u);
+  return __uint_as_float(b);
+}
+
+// 2^x for two values at once on the FMA pipe (the special-function unit does 16 exponentials per clock and SM, a
+// quarter of what the pass would need): x = n + f with n = round(x), 2^f by a cubic (relative error 7.5e-5, far below
+// the bf16 rounding of P), 2^n by adding n to the exponent field.  x is clamped to [-125, 128] so that the exponent
+// field stays in 1..254: below gives ~2^-125, above ~2^128 (finite in fp32, an infinity as bf16, which the caller's
+// overflow test sees).
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  x.x = fminf(fmaxf(x.x, -125.f), 128.f); x.y = fminf(fmaxf(x.y, -125.f), 128.f);
+  const float2 magic = make_float2(12582912.f, 12582912.f);        // 1.5 * 2^23: the sum's low mantissa bits are round(x)
+  const float2 t = __fadd2_rn(x, magic);
+  const float2 n = __fadd2_rn(t, make_float2(-12582912.f, -12582912.f));
+  const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));         // in [-0.5, 0.5]
+  float2 r = __ffma2_rn(make_float2(0.05517168343067169f, 0.05517168343067169f), f, make_float2(0.2426111251115799f, 0.2426111251115799f));
+  r = __ffma2_rn(r, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+  r = __ffma2_rn(r, f, make_float2(0.9999280571937561f, 0.9999280571937561f));
+  r.x = __int_as_float(__float_as_int(r.x) + (__float_as_int(t.x) << 23));
+  r.y = __int_as_float(__float_as_int(r.y) + (__float_as_int(t.y) << 23));
   return r;
 }
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
-struct Item {
-  int b, h, g, i, nb, s0, slen, l0, nlist, ntiles, q_valid, dq;
-  int64_t row;
-};
-
-// kChunk: chunked prefill.  q / o / lse hold the last positions of each sequence only: their token index is the k / v
-// token index plus dq, and query blocks before the chunk have nothing to do whatever their lists say.
-template <bool kChunk>
-__device__ __forceinline__ Item decode_item(const SeqMeta& m, const int32_t* __restrict__ row_ptr, int64_t w) {
-  Item it;
-  it.b = find_sequence(m.blk_off, m.batch, (int)(w / m.num_q_heads));
-  it.nb = m.blk_off[it.b + 1] - m.blk_off[it.b];
-  const int local = (int)(w - (int64_t)m.num_q_heads * m.blk_off[it.b]);
-  it.g = local / (it.nb * m.group);
-  const int rem = local - it.g * it.nb * m.group;
-  it.i = it.nb - 1 - rem / m.group;
-  it.h = it.g * m.group + rem % m.group;
-  it.row = (int64_t)m.num_q_heads * m.blk_off[it.b] + (int64_t)it.h * it.nb + it.i;
-  it.s0 = m.cu_seqlens[it.b];
-  it.slen = m.cu_seqlens[it.b + 1] - it.s0;
-  it.q_valid = min(kBlock, it.slen - it.i * kBlock);
-  it.l0 = row_ptr[it.row];
-  it.nlist = row_ptr[it.row + 1] - it.l0;
-  it.dq = 0;
-  if (kChunk) {
-    it.dq = m.qdelta[it.b];
-    if (it.i < m.qoff[it.b]) { it.nlist = 0; it.q_valid = 0; }   // no tiles, and no row of o / lse is written
-  }
-  it.ntiles = (it.nlist + 1) >> 1;
-  return it;
-}
-
-// Block index of list position p of an item: -1 past the end of the list, -2 for an entry outside [0, i].
-__device__ __forceinline__ int list_block(const Item& it, const int32_t* __restrict__ col_idx, int p) {
-  if (p >= it.nlist) return -1;
-  const int j = col_idx[it.l0 + p];
-  return (j < 0 || j > it.i) ? -2 : j;
-}
-
-// The same in two steps, so that the load can be issued long before its result is looked at.
-__device__ __forceinline__ int list_fetch(const Item& it, const int32_t* __restrict__ col_idx, int p) {
-  return p < it.nlist ? __ldg(col_idx + it.l0 + p) : -1;
-}
-__device__ __forceinline__ int list_check(const Item& it, int p, int raw) {
-  if (p >= it.nlist) return -1;
-  return (raw < 0 || raw > it.i) ? -2 : raw;
-}
-
-// Maximum of each of 16 columns over the 32 lanes of a warp; lanes l and l ^ 1 end with column l >> 1.
-__device__ __forceinline__ float warp_colmax16(const float (&x)[16], int lane) {
-  float a[8], b[4], c[2];
-  {
-    const bool up = (lane & 16) != 0;
+// One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(sl2 * x), x = s - R[c] as the MMA left it.
+// kPolyPairsOf8 of every eight column pairs take their exponentials on the FMA pipe, the others on the special-function unit.
+//   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the OR of the packed words: bit 14 or 30
+//                      set means some p >= 2, i.e. a score 2^(kRefShift + 1) above the maximum its reference was taken
+//                      from, or an infinity / NaN.
+//   SUBTRACT == true : removes p from l[c] again (used before a rebase; pk is not touched).
+// MASKED applies the causal mask of a diagonal block, drops a dead row and the query columns past a ragged block.
+template <bool MASKED, bool SUBTRACT>
+__device__ __forceinline__ uint32_t tile_pass(uint32_t s_addr, float sl2, bool row_live, bool diag,
+                                              int key_local, int q_valid, float (&l)[64], uint32_t (&pk)[32], uint32_t early_bar = 0u,
+                                              uint32_t early_parity = 0u, bool* early_done = nullptr) {
+  uint32_t ored = 0u;
+  const float2 sl22 = make_float2(sl2, sl2);
+  // two TMEM round trips per pass: the second half is requested before the first is worked on
+  uint32_t sv[2][32];
+  tc_ld32(s_addr, sv[0]);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) a[i] = fmaxf(up ? x[i + 8] : x[i], __shfl_xor_sync(0xffffffffu, up ? x[i] : x[i + 8], 16));
-  }
-  {
-    const bool up = (lane & 8) != 0;
+  for (int ch = 0; ch < 2; ++ch) {
+    tc_wait_ld32(sv[ch]);
+    if (ch == 0) tc_ld32(s_addr + 32, sv[1]);
+    // a barrier the caller needs after the pass is looked at here, so that the answer has arrived by then
+    if (ch == 1 && early_done != nullptr) *early_done = mbar_test(early_bar, early_parity);
+    // stage by stage over the 32 columns, each stage a run of independent instructions, in place
+    float2 v[16];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) b[i] = fmaxf(up ? a[i + 4] : a[i], __shfl_xor_sync(0xffffffffu, up ? a[i] : a[i + 4], 8));
-  }
-  {
-    const bool up = (lane & 4) != 0;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) c[i] = fmaxf(up ? b[i + 2] : b[i], __shfl_xor_sync(0xffffffffu, up ? b[i] : b[i + 2], 4));
-  }
-  const bool up = (lane & 2) != 0;
-  const float d = fmaxf(up ? c[1] : c[0], __shfl_xor_sync(0xffffffffu, up ? c[0] : c[1], 2));
-  return fmaxf(d, __shfl_xor_sync(0xffffffffu, d, 1));
-}
-
-// Sums l[0..63] over the 32 lanes of a warp; lane ends with the totals of columns (2*bitrev-ish) base, base+1
-// where base = 32*b4 + 16*b3 + 8*b2 + 4*b1 + 2*b0 (b_i = bit i of the lane id).
-__device__ __forceinline__ void warp_colsum(float (&l)[64], int lane, float& out0, float& out1, int& base) {
-  float a[32];
-  {
-    const bool up = (lane & 16) != 0;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const float send = up ? l[i] : l[i + 32];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
-      a[i] = (up ? l[i + 32] : l[i]) + recv;
-    }
-  }
-  float b[16];
-  {
-    const bool up = (lane & 8) != 0;
+    for (int i = 0; i < 16; ++i) v[i] = __fmul2_rn(make_float2(__uint_as_float(sv[ch][2 * i]), __uint_as_float(sv[ch][2 * i + 1])), sl22);
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      const float send = up ? a[i] : a[i + 16];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, 8);
-      b[i] = (up ? a[i + 16] : a[i]) + recv;
+      if ((i & 7) < kPolyPairsOf8) v[i] = exp2_poly2(v[i]);
+      else v[i] = make_float2(ex2f(v[i].x), ex2f(v[i].y));
     }
-  }
-  float c[8];
-  {
-    const bool up = (lane & 4) != 0;
+    if (MASKED) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float send = up ? b[i] : b[i + 8];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, 4);
-      c[i] = (up ? b[i + 8] : b[i]) + recv;
-    }
-  }
-  float d[4];
-  {
-    const bool up = (lane & 2) != 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float send = up ? c[i] : c[i + 4];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, 2);
-      d[i] = (up ? c[i + 4] : c[i]) + recv;
-    }
-  }
-  {
-    const bool up = (lane & 1) != 0;
-    const float s0 = up ? d[0] : d[2], s1 = up ? d[1] : d[3];
-    const float r0 = __shfl_xor_sync(0xffffffffu, s0, 1), r1 = __shfl_xor_sync(0xffffffffu, s1, 1);
-    out0 = (up ? d[2] : d[0]) + r0;
-    out1 = (up ? d[3] : d[1]) + r1;
-  }
-  base = ((lane >> 4) & 1) * 32 + ((lane >> 3) & 1) * 16 + ((lane >> 2) & 1) * 8 + ((lane >> 1) & 1) * 4 + (lane & 1) * 2;
-}
-
-// Optional cycle accounting of CTA 0 (diagnostics): every role attributes the clocks between two consecutive marks to the
-// tag of the later mark, accumulates per tag in shared memory, and writes the sums and mark counts to
-// trace[role * 8192 + tag * 2 ...] when it ends.
-constexpr int kTraceTags = 48;
-template <bool ON>
-struct Tracer {
-  unsigned long long* p;      // global destination (nullptr: off)
-  unsigned long long* acc;    // shared accumulators of this role: [tag][sum, count]
-  long long last;
-  bool on;
-  // Only every 8th tile is timed: the bookkeeping of a timed tile (~100 clocks per event) would otherwise slow the
-  // traced CTA by a quarter and distort what it measures.
-  __device__ __forceinline__ void sample(uint32_t ordinal) {
-    const bool was = on;
-    on = p != nullptr && (ordinal & 7u) == 0u;
-    if (on && !was) last = clock64();
-  }
-  __device__ __forceinline__ void init(unsigned long long* base, int role, unsigned char* smem_trace) {
-    p = (base != nullptr && blockIdx.x == 0) ? base + (size_t)role * 8192 : nullptr;
-    acc = reinterpret_cast<unsigned long long*>(smem_trace) + role * kTraceTags * 2;
-    if (p != nullptr) {
-      for (int i = 0; i < kTraceTags * 2; ++i) acc[i] = 0;
-      last = clock64();
-    }
-    on = false;
-  }
-  __device__ __forceinline__ void ev(uint32_t tag, uint32_t) {
-    if (on) {
-      const long long now = clock64();
-      acc[2 * tag] += (unsigned long long)(now - last);
-      acc[2 * tag + 1] += 1;
-      last = clock64();
-    }
-  }
-  __device__ __forceinline__ void flush() {
-    if (p != nullptr)
-      for (int i = 0; i < kTraceTags * 2; ++i) p[i] = acc[i];
-  }
-};
-template <>
-struct Tracer<false> {   // the production instantiation carries no state and no code
-  __device__ __forceinline__ void sample(uint32_t) {}
-  __device__ __forceinline__ void init(unsigned long long*, int, unsigned char*) {}
-  __device__ __forceinline__ void ev(uint32_t, uint32_t) {}
-  __device__ __forceinline__ void flush() {}
-};
-
-// One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]).
-//   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the OR of the packed words: bit 14 or 30
-//                      set means some p >= 2 (the references sit kRefShift above the column maxima, so that is a score
-//                      2^(kRefShift + 1) above its reference maximum, or an infinity / NaN).
-//   SUBTRACT == true : removes p from l[c] again (used before a rebase; pk is not touched).
-// MASKED applies the causal mask of a diagonal block / drops a dead row.
-template <bool MASKED, bool SUBTRACT, class TR = Tracer<false>>
-__device__ __forceinline__ uint32_t softmax_pass(uint32_t s_addr, uint32_t m_addr, float sl2, bool row_live,
-                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32], TR* tr = nullptr) {
-  uint32_t ored = 0u;
-  uint32_t sv[2][8], mv[2][8];
-  tc_ld8(s_addr, sv[0]);
-  tc_ld8(m_addr, mv[0]);
-#pragma unroll
-  for (int ch = 0; ch < 8; ++ch) {
-    tc_wait_ld8(sv[ch & 1], mv[ch & 1]);
-    if (tr) tr->ev(40 + (ch >> 1), 0);
-    if (ch < 7) {
-      tc_ld8(s_addr + (ch + 1) * 8, sv[(ch + 1) & 1]);
-      tc_ld8(m_addr + (ch + 1) * 8, mv[(ch + 1) & 1]);
-    }
-#pragma unroll
-    for (int e = 0; e < 8; e += 4) {
-      const int c = ch * 8 + e;
-      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -__uint_as_float(mv[ch & 1][e]));
-      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -__uint_as_float(mv[ch & 1][e + 1]));
-      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -__uint_as_float(mv[ch & 1][e + 2]));
-      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -__uint_as_float(mv[ch & 1][e + 3]));
-      if (MASKED) {
-        if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 2)) x2 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 3)) x3 = -CUDART_INF_F;
+      for (int i = 0; i < 16; ++i) {
+        const int c = ch * 32 + 2 * i;
+        if (!row_live || (diag && key_local > c) || c >= q_valid) v[i].x = 0.f;
+        if (!row_live || (diag && key_local > c + 1) || c + 1 >= q_valid) v[i].y = 0.f;
       }
-      const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
-      if (SUBTRACT) {
-        l[c] -= p0; l[c + 1] -= p1; l[c + 2] -= p2; l[c + 3] -= p3;
-      } else {
-        l[c] += p0; l[c + 1] += p1; l[c + 2] += p2; l[c + 3] += p3;
-        pk[c >> 1] = pack_bf16(p0, p1);
-        pk[(c >> 1) + 1] = pack_bf16(p2, p3);
-        ored |= pk[c >> 1] | pk[(c >> 1) + 1];
+    }
+    if (!SUBTRACT) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        pk[ch * 16 + i] = pack_bf16(v[i].x, v[i].y);
+        ored |= pk[ch * 16 + i];
       }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) { v[i].x = -v[i].x; v[i].y = -v[i].y; }
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int c = ch * 32 + 2 * i;
+      const float2 la = __fadd2_rn(make_float2(l[c], l[c + 1]), v[i]);
+      l[c] = la.x; l[c + 1] = la.y;
     }
   }
   return ored;
@@ -456,37 +183,45 @@ __device__ __forceinline__ uint32_t softmax_pass(uint32_t s_addr, uint32_t m_add
 template <bool kTrace, bool kChunk>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-               const __grid_constant__ CUtensorMap map_v, SeqMeta m, const int32_t* __restrict__ row_ptr,
-               const int32_t* __restrict__ col_idx, const void* __restrict__ k_ptr, const void* __restrict__ v_ptr,
-               uint16_t* __restrict__ o,
-               float* __restrict__ lse, int* __restrict__ status, unsigned long long* __restrict__ trace) {
+                const __grid_constant__ CUtensorMap map_v, SeqMeta m,
+                const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                uint16_t* __restrict__ o, float* __restrict__ lse, int* __restrict__ status,
+                unsigned long long* __restrict__ trace) {
   extern __shared__ unsigned char smem_raw[];
   Shared sh;
   sh.base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  sh.bar0 = sh.base + kOffBar;
+  sh.abort_addr = sh.base + kOffMisc + 8;
+  sh.limit_ns = (unsigned long long)m.wait_limit_us * 1000ull;
   unsigned char* smem = smem_raw + (sh.base - smem_u32(smem_raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kOffMisc);
 
   if (threadIdx.x == 0) {
-    mbar_init(sh.bar(Q_FULL), 1);
-    mbar_init(sh.bar(Q_EMPTY), 1);
-    for (int i = 0; i < kKSlots; ++i) {
-      mbar_init(sh.bar(K_FULL + i), 1);
-      mbar_init(sh.bar(K_EMPTY + i), 1);
-    }
-    for (int i = 0; i < kVSlots; ++i) {
-      mbar_init(sh.bar(V_FULL + i), 32 * kVProducerWarps);   // one arrival per producer lane, when its copies have landed
-      mbar_init(sh.bar(V_EMPTY + i), 1);
-    }
-    for (int i = 0; i < 4; ++i) {
-      mbar_init(sh.bar(P_FULL + i), kGroupThreads / 32);   // one arrival per softmax warp
-      mbar_init(sh.bar(PV_DONE + i), 1);
-      mbar_init(sh.bar(S_FULL + i), 1);
-      mbar_init(sh.bar(S_EMPTY + i), 1);                   // passed on by the P V issuer when it has seen P_FULL
+    for (int s = 0; s < 2; ++s) {
+      const int b = s * kBarsPerStream;
+      mbar_init(sh.bar(b + Q_FULL), 1);
+      mbar_init(sh.bar(b + Q_EMPTY), 1);
+      mbar_init(sh.bar(b + K_FULL), 1);
+      mbar_init(sh.bar(b + K_EMPTY), 1);
+      mbar_init(sh.bar(b + V_FULL), 1);
+      mbar_init(sh.bar(b + V_EMPTY), 1);
+      mbar_init(sh.bar(b + S_FULL), 1);
+      mbar_init(sh.bar(b + S_FULL + 1), 1);
+      mbar_init(sh.bar(b + P_FULL), 1);                       // one arrival, after the softmax group has met
+      mbar_init(sh.bar(b + PV_DONE), 1);
+      mbar_init(sh.bar(b + FIXED), 1);
     }
     st_shared_u32(sh.abort_flag(), 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // the column of ones, the two -R rows (R = 0) and the per-group arrays that must start defined
+  for (uint32_t i = threadIdx.x; i < (4096u + 4u * 2048u) / 4u; i += kThreads) {
+    const uint32_t off = i * 4u;   // rows of the first K chunk are 16 bytes apart: elements 0, 1 | 2, 3 | ...
+    reinterpret_cast<uint32_t*>(smem + kOffOnes)[i] = off >= 2048u ? 0u : (off & 15u) == 0u ? 0x3f803f80u : (off & 15u) == 4u ? 0x3f80u : 0u;
+  }
+  for (uint32_t i = threadIdx.x; i < 2u * kGrpBytes / 4u; i += kThreads) reinterpret_cast<uint32_t*>(smem + kOffGrp)[i] = 0u;
+  fence_async_smem();
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sh.base + kOffMisc), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -498,368 +233,412 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const unsigned long long cta_t0 = kTrace ? global_ns() : 0ull;
   const long long cta_c0 = kTrace ? clock64() : 0ll;
 
-  // Ordinals shared by all roles: k = non-empty items seen by this CTA, g = tiles seen, cnt_a / cnt_b = tiles handed to
-  // softmax group A / B.  Every role walks the same items and tiles, so the counters agree without communication.
+  // Every role of stream s walks the same items w = 2 * blockIdx.x + s, + 2 * gridDim.x, ... and the same tiles, so
+  // their ordinals (items seen, tiles seen) agree without communication.
+  const int64_t w_step = 2 * (int64_t)gridDim.x;
 
-  // Register split: the two helper warpgroups (warps 0-3, 12-15) give registers up, the softmax warpgroups take them.
   if (warp < 4 || warp >= 12) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
-  // ============================================================================================ K (+Q) producer (TMA)
-  if (warp == 0) {
-    if (lane == 0) {
-      Tracer<kTrace> tr; tr.init(trace, 0, smem + kOffTrace);
-      uint32_t k = 0, g = 0, slot = 0, use = 0;
-      bool ok = true;
-      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item<kChunk>(m, row_ptr, w);
-        if (it.ntiles == 0) continue;
-        if (!mbar_wait(sh, Q_EMPTY, (k & 1u) ^ 1u, status)) break;
-        mbar_expect_tx(sh.bar(Q_FULL), kQBytes);
-        const int tq = it.s0 + it.i * kBlock + (kChunk ? it.dq : 0);
-        tma_load_3d(sh.base + kOffQ, &map_q, sh.bar(Q_FULL), 0, it.h, tq);
-        tma_load_3d(sh.base + kOffQ + kHalfQ, &map_q, sh.bar(Q_FULL), 64, it.h, tq);
-        ++k;
-        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
-        for (int t = 0; t < it.ntiles; ++t, ++g) {
-          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
-          if (ja == -2 || jb == -2) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
-          tr.sample(g); tr.ev(1, g);
-          if (!mbar_wait(sh, K_EMPTY + (int)slot, (use & 1u) ^ 1u, status)) { ok = false; break; }
-          tr.ev(2, g);
-          const bool has_b = jb != -1;
-          const int xa = ja < 0 ? 0 : ja, xb = jb < 0 ? 0 : jb;   // a rejected entry: any valid block, masked out in the softmax
-          const uint32_t fb = sh.bar(K_FULL + (int)slot), dst = sh.base + kOffK + slot * kKVBytes;
-          mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
-          const int ta = it.s0 + xa * kBlock, tb = it.s0 + xb * kBlock;
-          tma_load_3d(dst, &map_k, fb, 0, it.g, ta);
-          tma_load_3d(dst + kHalfKV, &map_k, fb, 64, it.g, ta);
-          if (has_b) {
-            tma_load_3d(dst + kHalfQ, &map_k, fb, 0, it.g, tb);
-            tma_load_3d(dst + kHalfKV + kHalfQ, &map_k, fb, 64, it.g, tb);
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
+    // ========================================================================================== producers (TMA)
+    // warps 0 / 2: Q and K of stream 0 / 1; warps 12 / 13: V of stream 0 / 1
+    if (warp == 0 || warp == 2 || warp == 12 || warp == 13) {
+      if (lane == 0) {
+        const bool is_v = warp >= 12;
+        const int s = is_v ? warp - 12 : warp >> 1, bb = s * kBarsPerStream;
+        const uint32_t sbase = sh.base + (uint32_t)s * kStreamBytes;
+        Tracer<kTrace> tr; tr.init(s == 0 ? trace : nullptr, is_v ? 2 : 0, smem + kOffTrace);
+        const CUtensorMap* map = is_v ? &map_v : &map_k;
+        const int full = bb + (is_v ? V_FULL : K_FULL), empty = bb + (is_v ? V_EMPTY : K_EMPTY);
+        const uint32_t dst = sbase + (is_v ? kStV : kStK);
+        uint32_t nitem = 0, cnt = 0;
+        bool ok = true;
+        for (int64_t w = 2 * (int64_t)blockIdx.x + s; ok && w < m.rows; w += w_step) {
+          const Item it = decode_item<kChunk>(m, row_ptr, w);
+          if (it.ntiles == 0) continue;
+          if (!is_v) {
+            if (!mbar_wait<kProducerSleepNs>(sh, bb + Q_EMPTY, (nitem & 1u) ^ 1u, status)) break;
+            mbar_expect_tx(sh.bar(bb + Q_FULL), kQBytes);
+            const int tq = it.s0 + it.i * kBlock + (kChunk ? it.dq : 0);
+            tma_load_3d(sbase + kStQ, &map_q, sh.bar(bb + Q_FULL), 0, it.h, tq);
+            tma_load_3d(sbase + kStQ + kHalfQ, &map_q, sh.bar(bb + Q_FULL), 64, it.h, tq);
+            ++nitem;
           }
-          if (++slot == (uint32_t)kKSlots) { slot = 0; ++use; }
-          ja = na; jb = nb2;
-        }
-      }
-      tr.flush();
-    }
-  }
-  // ============================================================================================ V producers (cp.async)
-  // V tiles come through the LSU path (cp.async, 16 bytes per request).  Measured on this part: TMA box gathers of
-  // 128-byte rows sustain ~41 B/clk per SM, cp.async ~80, both together ~85 (the SM's fill limit) and neither slows the
-  // MMAs, so K goes by TMA and V by cp.async.  Producer warp pw copies rows 16 pw .. 16 pw + 15 of each block of the tile;
-  // each lane writes the 128-byte-swizzled layout the MMA descriptor expects (rows past the end of the sequence are
-  // zero-filled: 0 * x must be 0); completion is asynchronous: every lane's copies arrive on the slot's mbarrier when they
-  // have landed.
-  else if (warp >= 12) {
-    const int pw = warp - 12;
-    Tracer<kTrace> tr; tr.init(lane == 0 && pw == 0 ? trace : nullptr, 2, smem + kOffTrace);
-    const unsigned char* __restrict__ xg = reinterpret_cast<const unsigned char*>(v_ptr);
-    const size_t row_bytes = (size_t)m.num_kv_heads * kHeadDim * 2;      // bytes between consecutive tokens
-    const int chunk = lane & 15, rsub = lane >> 4;
-    const int row0 = pw * (kBlock / kVProducerWarps);                    // first row of this warp's share of a block
-    constexpr int kIters = kBlock / kVProducerWarps / 2;                 // 2 rows per warp instruction
-    // destination offset of (row0 + 2 * itc + rsub, this lane's chunk) inside a block half, for itc mod 4 = 0..3
-    uint32_t doff[4];
-#pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-      const int row = 2 * q4 + rsub;
-      doff[q4] = (uint32_t)(chunk >> 3) * kHalfKV + (uint32_t)(row0 + row) * 128u + (uint32_t)(((chunk & 7) ^ (row & 7)) << 4);
-    }
-    uint32_t g = 0;
-    bool ok = true;
-    for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-      const Item it = decode_item<kChunk>(m, row_ptr, w);
-      if (it.ntiles == 0) continue;
-      int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
-      const unsigned char* seq_base = xg + ((size_t)it.s0 * m.num_kv_heads + it.g) * (kHeadDim * 2) + (size_t)chunk * 16 +
-                                      (size_t)(row0 + rsub) * row_bytes;
-      for (int t = 0; t < it.ntiles; ++t, ++g) {
-        const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
-        const uint32_t st = g & 1u;
-        tr.sample(g); tr.ev(3, g);
-        if (!mbar_wait(sh, V_EMPTY + (int)st, ((g >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
-        tr.ev(4, g);
-        const uint32_t dst0 = sh.base + kOffV + st * kKVBytes;
-#pragma unroll 1
-        for (int half_tile = 0; half_tile < 2; ++half_tile) {
-          int j = half_tile ? jb : ja;
-          if (j == -1) continue;                       // odd list: no second block
-          if (j < 0) j = 0;                            // rejected entry: any valid block, masked out in the softmax
-          const int rows_valid = it.slen - j * kBlock - row0 - rsub;   // this lane's rows 2 * itc below this are real
-          const unsigned char* src = seq_base + (size_t)j * kBlock * row_bytes;
-          const uint32_t dst = dst0 + (uint32_t)half_tile * 8192u;
-#pragma unroll
-          for (int itc = 0; itc < kIters; ++itc) {
-            const bool valid = 2 * itc < rows_valid;
-            const int sz = valid ? 16 : 0;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + doff[itc & 3] + (uint32_t)(itc >> 2) * 1024u),
-                         "l"(valid ? src + (size_t)(2 * itc) * row_bytes : seq_base), "r"(sz) : "memory");
+          int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
+          for (int t = 0; t < it.ntiles; ++t, ++cnt) {
+            const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);   // next pair
+            if (!is_v && (ja == -2 || jb == -2)) atomicCAS(status, 0, (int)SEER_ERR_INVALID_INDEX);
+            tr.sample(cnt); tr.ev(1, cnt);
+            if (!mbar_wait<kProducerSleepNs>(sh, empty, (cnt & 1u) ^ 1u, status)) { ok = false; break; }
+            tr.ev(2, cnt);
+            const bool has_b = jb != -1;
+            const int xa = ja < 0 ? 0 : ja, xb = jb < 0 ? 0 : jb;   // a rejected entry: any valid block, masked out in the softmax
+            // test hook: one V copy that is never issued, so that the issuer's wait for it runs out
+            if (is_v && s == 0 && blockIdx.x == 0 && m.lose_v_copy >= 0 && cnt == (uint32_t)m.lose_v_copy) { ja = na; jb = nb2; continue; }
+            const uint32_t fb = sh.bar(full);
+            mbar_expect_tx(fb, has_b ? kKVBytes : kKVBytes / 2);
+            const int ta = it.s0 + xa * kBlock, tb = it.s0 + xb * kBlock;
+            tma_load_3d(dst, map, fb, 0, it.g, ta);
+            tma_load_3d(dst + kHalfKV, map, fb, 64, it.g, ta);
+            if (has_b) {
+              tma_load_3d(dst + kHalfQ, map, fb, 0, it.g, tb);
+              tma_load_3d(dst + kHalfKV + kHalfQ, map, fb, 64, it.g, tb);
+            }
+            ja = na; jb = nb2;
           }
         }
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sh.bar(V_FULL + (int)st)) : "memory");
-        ja = na; jb = nb2;
+        tr.flush();
       }
     }
-    asm volatile("cp.async.wait_all;" ::: "memory");   // nothing of this warp is in flight when the CTA ends
-    tr.flush();
-  }
-  // ============================================================================================ S^T issuer
-  else if (warp == 1) {
-    if (lane == 0) {
-      Tracer<kTrace> tr; tr.init(trace, 1, smem + kOffTrace);
-      uint32_t k = 0, g = 0, cnt_a = 0, cnt_b = 0, slot = 0, use = 0;
-      // descriptor bases; per K-step the start address advances by 32 bytes inside a 64-element swizzle atom and by
-      // one d-half (16 KB / 8 KB) between atoms
-      const uint64_t kd0 = make_desc(sh.base + kOffK, 16, 1024);
-      const uint64_t qd = make_desc(sh.base + kOffQ, 16, 1024);
-      bool ok = true;
-      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item<kChunk>(m, row_ptr, w);
-        if (it.ntiles == 0) continue;
-        if (!mbar_wait(sh, Q_FULL, k & 1u, status)) break;
-        for (int t = 0; t < it.ntiles; ++t, ++g) {
-          const int grp = t & 1;
-          const uint32_t cn = grp ? cnt_b : cnt_a, buf = cn & 1u;
-          tr.sample(g); tr.ev(10, g);
-          if (!mbar_wait(sh, K_FULL + (int)slot, use & 1u, status)) { ok = false; break; }
-          tr.ev(11, g);
-          if (!mbar_wait(sh, S_EMPTY + 2 * grp + buf, ((cn >> 1) & 1u) ^ 1u, status)) { ok = false; break; }
-          tr.ev(12, g);
+    // ========================================================================================== MMA issuer of a stream
+    else if (warp == 1 || warp == 3) {
+      if (lane == 0) {
+        const int s = warp >> 1, bb = s * kBarsPerStream;
+        const uint32_t sbase = sh.base + (uint32_t)s * kStreamBytes;
+        Tracer<kTrace> tr; tr.init(trace, s == 0 ? 1 : 3, smem + kOffTrace);
+        // (the low word of a descriptor holds the start address and the leading-dimension offset, the high word is constant)
+        const uint64_t desc_hi_k = make_desc(0, 16, 1024) & 0xffffffff00000000ull;
+        const uint64_t desc_hi_v = make_desc(0, kHalfKV, 1024) & 0xffffffff00000000ull;
+        const uint32_t kd_lo = (uint32_t)make_desc(sbase + kStK, 16, 1024), qd_lo = (uint32_t)make_desc(sbase + kStQ, 16, 1024);
+        const uint32_t vd_lo = (uint32_t)make_desc(sbase + kStV, kHalfKV, 1024), pd_lo = (uint32_t)make_desc(sbase + kStP, kHalfKV, 1024);
+        const uint64_t ones_d = make_desc_ns(sh.base + kOffOnes, 2048, 128);
+        const uint64_t qext_d = make_desc_ns(sh.base + kOffQext + (uint32_t)s * 2048u, 1024, 128);
+        const uint32_t d_o = tmem + col_o(s);
+        uint32_t nitem = 0, cs = 0, cp = 0;   // items, S^T tiles issued, P V tiles issued (of this stream)
+        bool ok = true;
+        // S^T of the next tile of the stream (ordinal cs) into buffer cs & 1: eight K-steps over d, a ninth that
+        // subtracts the softmax references
+        auto issue_s = [&](bool last_of_item, bool with_refs) -> bool {
+          tr.ev(10, cs);
+          if (!mbar_wait(sh, bb + K_FULL, cs & 1u, status)) return false;
+          tr.ev(11, cs);
           tc_fence_after();
-          const uint64_t kd = kd0 + (uint64_t)(slot * (kKVBytes >> 4));
-          const uint32_t d = tmem + col_s(grp, buf);
+          const uint32_t d = tmem + col_s(s, cs & 1u);
+          uint32_t klo = kd_lo, qlo = qd_lo;
+          asm volatile("" : "+r"(klo), "+r"(qlo));   // the descriptors are formed here, not kept in registers across the loop
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
-            tc_mma(d, kd + (uint64_t)((kk >> 2) * (kHalfKV >> 4) + (kk & 3) * 2),
-                   qd + (uint64_t)((kk >> 2) * (kHalfQ >> 4) + (kk & 3) * 2), kIdescS, kk > 0);
-          tc_commit(sh.bar(S_FULL + 2 * grp + buf));
-          tc_commit(sh.bar(K_EMPTY + (int)slot));
-          if (t == it.ntiles - 1) tc_commit(sh.bar(Q_EMPTY));   // last S^T of the item: Q may be replaced
-          tr.ev(17, g);
-          if (grp) ++cnt_b; else ++cnt_a;
-          if (++slot == (uint32_t)kKSlots) { slot = 0; ++use; }
-        }
-        ++k;
-      }
-      tr.flush();
-    }
-  }
-  // ============================================================================================ P V issuer
-  else if (warp == 3) {
-    if (lane == 0) {
-      Tracer<kTrace> tr; tr.init(trace, 3, smem + kOffTrace);
-      uint32_t g = 0, cnt_a = 0, cnt_b = 0;
-      const uint64_t vd0 = make_desc(sh.base + kOffV, kHalfKV, 1024), vd1 = make_desc(sh.base + kOffV + kKVBytes, kHalfKV, 1024);
-      const uint64_t pd0 = make_desc(sh.base + kOffP, kHalfKV, 1024);   // P^T buffer (group, buf) lies 2 * group + buf buffers on
-      bool ok = true;
-      for (int64_t w = blockIdx.x; ok && w < m.rows; w += gridDim.x) {
-        const Item it = decode_item<kChunk>(m, row_ptr, w);
-        for (int t = 0; t < it.ntiles; ++t, ++g) {
-          const int grp = t & 1;
-          const uint32_t cn = grp ? cnt_b : cnt_a, st = g & 1u;
-          tr.sample(g); tr.ev(13, g);
-          if (!mbar_wait(sh, V_FULL + st, (g >> 1) & 1u, status)) { ok = false; break; }
-          tr.ev(14, g);
-          const uint32_t pb = 2u * (uint32_t)grp + (cn & 1u);
-          if (!mbar_wait(sh, P_FULL + (int)pb, (cn >> 1) & 1u, status)) { ok = false; break; }
-          // the softmax group has finished with S^T buffer cn & 1 as well (it read it before it wrote P^T): tell the S^T issuer
-          mbar_arrive(sh.bar(S_EMPTY + (int)pb));
-          tr.ev(15, g);
-          fence_async_smem();     // V was written through the generic proxy (cp.async); the MMA reads through the async proxy
-          tc_fence_after();
-          const uint64_t vd = st ? vd1 : vd0, pd = pd0 + (uint64_t)(pb * (kPBytes >> 4));
-          const uint32_t d = tmem + col_o(grp);
-          const uint32_t acc0 = t >= 2 ? 1u : 0u;                  // first tile of this group in the item starts O^T afresh
-          // 16 keys (2048 bytes of 128-byte rows) per step; an odd list leaves the second block of its last tile out
+            tc_mma(d, desc_hi_k | (uint64_t)(klo + (uint32_t)((kk >> 2) * (kHalfKV >> 4) + (kk & 3) * 2)),
+                   desc_hi_k | (uint64_t)(qlo + (uint32_t)((kk >> 2) * (kHalfQ >> 4) + (kk & 3) * 2)), kIdescS, kk > 0);
+          if (with_refs) tc_mma(d, ones_d, qext_d, kIdescS, 1u);
+          tc_commit(sh.bar(bb + S_FULL + (int)(cs & 1u)));
+          tc_commit(sh.bar(bb + K_EMPTY));
+          if (last_of_item) tc_commit(sh.bar(bb + Q_EMPTY));   // last S^T of the item: Q may be replaced
+          tr.ev(12, cs);
+          ++cs;
+          return true;
+        };
+        for (int64_t w = 2 * (int64_t)blockIdx.x + s; ok && w < m.rows; w += w_step) {
+          const Item it = decode_item<kChunk>(m, row_ptr, w);
+          if (it.ntiles == 0) continue;
+          tr.sample(cs);
+          if (!mbar_wait(sh, bb + Q_FULL, nitem & 1u, status)) break;
+          ++nitem;
+          // the first two tiles of an item are computed without references (the row still holds those of the previous
+          // item, and a result must not depend on which item came before): the group subtracts its first references
+          // from them in place
+          if (!issue_s(it.ntiles == 1, false)) break;
+          if (it.ntiles > 1 && !issue_s(it.ntiles == 2, false)) break;
+          for (int t = 0; t < it.ntiles; ++t, ++cp) {
+            tr.sample(cp); tr.ev(13, cp);
+            if (!mbar_wait(sh, bb + V_FULL, cp & 1u, status)) { ok = false; break; }
+            tr.ev(14, cp);
+            // P^T of tile t is complete; the group has also finished with S^T buffer cp & 1 (and, at t = 0, with the
+            // O^T accumulator of the previous item)
+            if (!mbar_wait<kIssuerSleepNs>(sh, bb + P_FULL, cp & 1u, status)) { ok = false; break; }
+            tr.ev(15, cp);
+            tc_fence_after();
+            // 16 keys (2048 bytes of 128-byte rows) per step; an odd list leaves the second block of its last tile out
+            uint32_t vlo = vd_lo, plo = pd_lo;
+            asm volatile("" : "+r"(vlo), "+r"(plo));
 #pragma unroll
-          for (int kk = 0; kk < 4; ++kk) tc_mma(d, vd + (uint64_t)(kk * 128), pd + (uint64_t)(kk * 128), kIdescPV, kk > 0 ? 1u : acc0);
-          if (2 * t + 1 < it.nlist) {
+            for (int kk = 0; kk < 4; ++kk)
+              tc_mma(d_o, desc_hi_v | (uint64_t)(vlo + (uint32_t)(kk * 128)), desc_hi_v | (uint64_t)(plo + (uint32_t)(kk * 128)), kIdescPV, (kk > 0 || t > 0) ? 1u : 0u);
+            if (2 * t + 1 < it.nlist) {
 #pragma unroll
-            for (int kk = 4; kk < 8; ++kk) tc_mma(d, vd + (uint64_t)(kk * 128), pd + (uint64_t)(kk * 128), kIdescPV, 1u);
+              for (int kk = 4; kk < 8; ++kk)
+                tc_mma(d_o, desc_hi_v | (uint64_t)(vlo + (uint32_t)(kk * 128)), desc_hi_v | (uint64_t)(plo + (uint32_t)(kk * 128)), kIdescPV, 1u);
+            }
+            tc_commit(sh.bar(bb + V_EMPTY));
+            tc_commit(sh.bar(bb + PV_DONE));
+            tr.ev(16, cp);
+            if (t + 2 < it.ntiles && !issue_s(t + 3 == it.ntiles, true)) { ok = false; break; }
           }
-          tc_commit(sh.bar(V_EMPTY + st));
-          tc_commit(sh.bar(PV_DONE + (int)pb));
-          tr.ev(19, g);
-          if (grp) ++cnt_b; else ++cnt_a;
         }
+        tr.flush();
       }
-      tr.flush();
     }
-  }
   }   // helper warpgroups
   // ============================================================================================ softmax groups
   else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-    const int grp = (warp - 4) >> 2;                     // 0 = A (even tiles), 1 = B (odd tiles)
-    const int gt = threadIdx.x - 128 - grp * kGroupThreads;   // 0..127 within the group
-    const int gw = (warp - 4) & 3;                       // warp within the group
-    const int quad = warp & 3;                           // TMEM lane quadrant this warp may access
-    const int r = quad * 32 + lane;                      // key row of S^T / d row of O^T owned by this thread
+    const int s = (warp - 4) >> 2, bb = s * kBarsPerStream;
+    const int gt = threadIdx.x - 128 - s * kGroupThreads;   // 0..127 within the group
+    const int gw = (warp - 4) & 3;                          // warp within the group
+    const int quad = warp & 3;                              // TMEM lane quadrant this warp may access
+    const int r = quad * 32 + lane;                         // key row of S^T / d row of O^T owned by this thread
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    unsigned char* gsm = smem + kOffGrp + grp * kGrpBytes;
-    float* mref = reinterpret_cast<float*>(gsm + kGrpMref);
+    unsigned char* gsm = smem + kOffGrp + s * kGrpBytes;
+    float* rcur = reinterpret_cast<float*>(gsm + kGrpRcur);   // R[c], in units of raw scores (always a bf16 number)
     float* alpha = reinterpret_cast<float*>(gsm + kGrpAlpha);
-    float* lfin = reinterpret_cast<float*>(gsm + kGrpLfin);
     float* lsum = reinterpret_cast<float*>(gsm + kGrpLsum);
-    float* w_a = reinterpret_cast<float*>(smem + kOffW);
-    float* w_b = w_a + 64;
-    const float* mref_a = reinterpret_cast<const float*>(smem + kOffGrp + kGrpMref);
-    const float* mref_b = reinterpret_cast<const float*>(smem + kOffGrp + kGrpBytes + kGrpMref);
-    const float* lfin_a = reinterpret_cast<const float*>(smem + kOffGrp + kGrpLfin);
-    const float* lfin_b = reinterpret_cast<const float*>(smem + kOffGrp + kGrpBytes + kGrpLfin);
-    const int bar_sync = 1 + grp, bar_vote = 3 + grp;
+    uint16_t* qext = reinterpret_cast<uint16_t*>(smem + kOffQext + s * 2048);
+    uint16_t* qfix = reinterpret_cast<uint16_t*>(smem + kOffQfix + s * 2048);
+    const uint64_t ones_d = make_desc_ns(sh.base + kOffOnes, 2048, 128);
+    const uint64_t qfix_d = make_desc_ns(sh.base + kOffQfix + (uint32_t)s * 2048u, 1024, 128);
+    uint32_t nfix = 0;                                      // rebases of this stream so far
+    const int bar_sync = 1 + s, bar_vote = 3 + s;
     const float sl2 = m.softmax_scale * 1.4426950408889634f;
+    const float shift_raw = kRefShift / sl2;
     const int key_local = r & 63;
-    Tracer<kTrace> tr; tr.init(gt == 0 ? trace : nullptr, 4 + grp, smem + kOffTrace);
-    uint32_t cnt = 0;                                    // tiles this group has processed
-    uint32_t gbase = 0;                                  // tiles of this CTA before the current item
+    const uint32_t p_base = sh.base + (uint32_t)s * kStreamBytes + kStP;
+    unsigned char* p_gen = smem + (size_t)s * kStreamBytes + kStP;
+    const uint32_t o_addr = tmem + lane_addr + col_o(s);
+    Tracer<kTrace> tr; tr.init(gt == 0 ? trace : nullptr, 4 + s, smem + kOffTrace);
+    uint32_t cnt = 0;                                       // tiles this stream has processed
     bool ok = true;
+    // diagnostics (traced build): clocks of every steady-state tile by segment, kept in registers
+    long long seg[15] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, seg_last = 0;
+    unsigned seg_n = 0, nreb = 0;
+#define SEG(k) do { if constexpr (kTrace) { const long long now_ = clock64(); seg[k] += now_ - seg_last; seg_last = now_; } } while (0)
 
-    for (int64_t w = blockIdx.x; w < m.rows; w += gridDim.x) {
+    for (int64_t w = 2 * (int64_t)blockIdx.x + s; w < m.rows; w += w_step) {
       tr.sample(0);
       const Item it = decode_item<kChunk>(m, row_ptr, w);
       const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock + (kChunk ? it.dq : 0);   // first row of the item in q / o / lse
-      const int tiles_a = (it.ntiles + 1) >> 1, tiles_b = it.ntiles >> 1;
-      const int my_tiles = grp == 0 ? tiles_a : tiles_b;
+      if (it.ntiles == 0) {                                 // no visible key: o = 0, lse = -inf
+        for (int idx = gt; idx < 64 * 16; idx += kGroupThreads) {
+          const int qrow = idx >> 4, chunk = idx & 15;
+          if (qrow < it.q_valid)
+            *reinterpret_cast<uint4*>(o + ((tok0 + qrow) * m.num_q_heads + it.h) * kHeadDim + chunk * 8) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (lse != nullptr && gt < it.q_valid)
+          lse[(int64_t)it.h * (kChunk ? m.total_q_tokens : m.total_tokens) + tok0 + gt] = -CUDART_INF_F;
+        continue;
+      }
       float l_part[64];
 #pragma unroll
       for (int c = 0; c < 64; ++c) l_part[c] = 0.f;
-      if (gt < 64) mref[gt] = -CUDART_INF_F;
-      named_bar_sync(bar_sync, kGroupThreads);
+      const bool ragged_q = it.q_valid < kBlock;
 
-      int nja = list_block(it, col_idx, 2 * grp), njb = list_block(it, col_idx, 2 * grp + 1);
+      int nja = list_block(it, col_idx, 0), njb = list_block(it, col_idx, 1);
       tr.ev(29, 0);
-      for (int t = grp; t < it.ntiles; t += 2, ++cnt) {
+      bool s_seen = false;                                  // S_FULL of the coming tile was already seen complete
+      for (int t = 0; t < it.ntiles; ++t, ++cnt) {
         const uint32_t sbuf = cnt & 1u;
-        tr.sample(cnt); tr.ev(20, gbase + t);
-        bool fail = !mbar_wait(sh, S_FULL + 2 * grp + sbuf, (cnt >> 1) & 1u, status);
-        tr.ev(21, gbase + t);
+        if constexpr (kTrace) { seg_last = clock64(); ++seg_n; }
+        bool fail = false;
+        if (!s_seen) fail = !mbar_wait(sh, bb + S_FULL + (int)sbuf, (cnt >> 1) & 1u, status);
+        SEG(0);
         tc_fence_after();
         const int ja = nja, jb = njb;
-        // this group's next tile: the loads are issued here and looked at after the pass
-        const int raw_a = list_fetch(it, col_idx, 2 * t + 4), raw_b = list_fetch(it, col_idx, 2 * t + 5);
+        // the next tile's list entries: the loads are issued here and looked at after the pass
+        const int raw_a = list_fetch(it, col_idx, 2 * t + 2), raw_b = list_fetch(it, col_idx, 2 * t + 3);
         const int my_j = r < 64 ? ja : jb;
         const bool row_live = my_j >= 0;                 // absent / rejected blocks contribute nothing
         const bool diag = my_j == it.i;
-        const bool masked = !row_live || diag;           // uniform per warp (a warp lies in one block half)
-        const uint32_t s_addr = tmem + lane_addr + col_s(grp, sbuf);
-        const uint32_t m_addr = tmem + lane_addr + col_m(grp);
+        const bool masked = !row_live || diag || ragged_q;   // uniform per warp (a warp lies in one block half)
+        const uint32_t s_addr = tmem + lane_addr + col_s(s, sbuf);
         uint32_t pk[32];
-        // the first tile of a group in an item has no references yet: it goes straight to the rebase path
-        uint32_t over = 0x40004000u;
-        if (!fail && t >= 2) over = masked ? softmax_pass<true, false, Tracer<kTrace>>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk, &tr)
-                                 : softmax_pass<false, false, Tracer<kTrace>>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk, &tr);
-        nja = list_check(it, 2 * t + 4, raw_a); njb = list_check(it, 2 * t + 5, raw_b);
-        tr.ev(23, gbase + t);
-        // P^T goes to buffer cnt & 1 of the group; the P V that read that buffer two tiles ago has normally long finished
-        if (!fail && cnt >= 2) fail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)sbuf, ((cnt >> 1) - 1) & 1u, status);
-        tr.ev(22, gbase + t);
-        // one vote per tile: does any entry reach 2^(kRefShift + 1) times its reference maximum (or has a wait been lost)?
-        const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
-        tr.ev(24, gbase + t);
-        if (slow) {
-          // the O^T accumulator is rescaled below: the previous P V of this group must have finished
-          if (!fail && t >= 2) fail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)(sbuf ^ 1u), ((cnt - 1) >> 1) & 1u, status);
+        // First tile of an item: the references are still those of another item.  Column c takes the score of the
+        // tile's first key (visible to every query of the block: it is the first key of a block not later than the
+        // query block) plus kFirstShift as its reference: no reduction over the keys.  A reference taken from a key of
+        // the column itself can never be too high (what it would flush to zero is negligible next to that key), and
+        // if it is too low the pass below says so and the group rebases on exact maxima.
+        bool have_ref = t >= 1;
+        if (t == 0 && ja >= 0) {
+          if (!fail && it.ntiles > 1) fail = !mbar_wait(sh, bb + S_FULL + (int)(sbuf ^ 1u), ((cnt + 1) >> 1) & 1u, status);
           tc_fence_after();
-          if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
-          // ---- rebase: take this tile's contribution out of the row sums again, find the exact column maxima, move
-          // the references, rescale the row sums and O^T, and recompute the tile
-          if (t >= 2) {
-            if (masked) softmax_pass<true, true>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
-            else softmax_pass<false, true>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
-          }
-          // column maxima of the tile: over the lanes of each warp by shuffles (16 columns at a time: lane pair l, l ^ 1
-          // ends with column l >> 1 of the chunk), over the four warps through shared memory
-#pragma unroll 2
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t sv[16];
-            tc_ld16(s_addr + ch * 16, sv);
-            tc_wait_ld(sv);
-            float xv[16];
+          if (!fail && gw == 0) {                         // (the TMEM load is a warp-wide instruction; lane 0 holds key row 0)
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const int c = ch * 16 + e;
-              float x = __uint_as_float(sv[e]) * sl2;
-              if (!row_live || (diag && key_local > c)) x = -CUDART_INF_F;
-              xv[e] = x;
-            }
-            const float cm = warp_colmax16(xv, lane);
-            if ((lane & 1) == 0) lsum[gw * 64 + ch * 16 + (lane >> 1)] = cm;
-          }
-          named_bar_sync(bar_sync, kGroupThreads);
-          if (gt < 64) {
-            const float old = mref[gt];
-            const float cm = fmaxf(fmaxf(lsum[gt], lsum[64 + gt]), fmaxf(lsum[128 + gt], lsum[192 + gt]));
-            float nm = fmaxf(old, cm + kRefShift);
-            if (nm == -CUDART_INF_F) nm = 0.f;           // nothing visible in this column yet
-            // a query column past the end of a ragged block holds whatever tokens follow in the packed tensor: an
-            // unreachable reference makes its p = 0, so that it can never ask for a rebase (results must not depend on
-            // the neighbours in the batch)
-            if (gt >= it.q_valid) nm = 1.0e30f;
-            alpha[gt] = old == -CUDART_INF_F ? 0.f : exp2f(old - nm);
-            mref[gt] = nm;
-          }
-          named_bar_sync(bar_sync, kGroupThreads);
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {                // this lane's copy of the new references
-            uint32_t mv[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) mv[e] = __float_as_uint(mref[ch * 16 + e]);
-            tc_st16(m_addr + ch * 16, mv);
-          }
-          tc_wait_st();
-          // a reference that moved by more than 2^30 makes everything accumulated so far negligible (and the value
-          // taken out above may not have been finite): start the column afresh
-#pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            const float a = alpha[c];
-            l_part[c] = (t < 2 || a < 9.3e-10f) ? 0.f : l_part[c] * a;
-          }
-          if (t >= 2) {                                  // this group already accumulated into O^T for this item
-#pragma unroll 1
             for (int ch = 0; ch < 4; ++ch) {
-              uint32_t ov[16];
-              tc_ld16(tmem + lane_addr + col_o(grp) + ch * 16, ov);
-              tc_wait_ld(ov);
+              uint32_t sv[16];
+              tc_ld16(s_addr + ch * 16, sv);
+              tc_wait_ld(sv);
+              if (lane == 0) {
 #pragma unroll
-              for (int e = 0; e < 16; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha[ch * 16 + e]);
-              tc_st16(tmem + lane_addr + col_o(grp) + ch * 16, ov);
+                for (int e = 0; e < 16; e += 4)
+                  *reinterpret_cast<uint4*>(&lsum[ch * 16 + e]) = make_uint4(sv[e], sv[e + 1], sv[e + 2], sv[e + 3]);
+              }
             }
-            tc_wait_st();
           }
-          if (masked) softmax_pass<true, false>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
-          else softmax_pass<false, false>(s_addr, m_addr, sl2, row_live, diag, key_local, l_part, pk);
+          tc_fence_before();
+          if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
+          if (gt < 64) {
+            const float old = 0.f;                       // the first two S^T tiles of an item hold the raw scores
+            float nr = bf16_ceil(lsum[gt] + kFirstShift / sl2);
+            if (gt >= it.q_valid || !(fabsf(nr) < 3.0e38f)) nr = old;   // not a column of this block / not a finite score
+            const float d = old - nr;
+            rcur[gt] = nr;
+            qext[gt * 8] = (uint16_t)((__float_as_uint(nr) >> 16) ^ 0x8000u);
+            const uint32_t hi = __float_as_uint(d) & 0xffff0000u;
+            const float r1 = d - __uint_as_float(hi);
+            const uint32_t mid = __float_as_uint(r1) & 0xffff0000u;
+            const uint32_t lo = __float_as_uint(r1 - __uint_as_float(mid)) & 0xffff0000u;
+            *reinterpret_cast<uint2*>(qfix + gt * 8) = make_uint2((hi >> 16) | mid, lo >> 16);
+            fence_async_smem();
+          }
+          named_bar_sync(bar_sync, kGroupThreads);
+          if (gt == 0) {
+            tc_fence_after();
+            tc_mma(tmem + col_s(s, sbuf), ones_d, qfix_d, kIdescS, 1u);
+            if (it.ntiles > 1) tc_mma(tmem + col_s(s, sbuf ^ 1u), ones_d, qfix_d, kIdescS, 1u);
+            tc_commit(sh.bar(bb + FIXED));
+          }
+          if (named_bar_or(bar_vote, kGroupThreads, !mbar_wait(sh, bb + FIXED, nfix & 1u, status))) { ok = false; break; }
+          ++nfix;
+          tc_fence_after();
+          have_ref = true;
         }
-        tr.ev(26, 0);
-        // P^T row r -> buffer cnt & 1 of the group (128-byte swizzle)
-        {
-          const uint32_t prow = sh.base + kOffP + (2u * (uint32_t)grp + sbuf) * kPBytes + (uint32_t)r * 128u;
+        // without references (the first key of the first tile is not a valid entry) the tile goes straight to the rebase
+        uint32_t over = 0x40004000u;
+        bool pv_seen = t == 0;                           // the P V of the previous tile has finished: the P^T buffer is free, O^T at rest
+        if (!fail && have_ref)
+          over = masked ? tile_pass<true, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk)
+                        : tile_pass<false, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk,
+                                                  sh.bar(bb + PV_DONE), (cnt - 1) & 1u, t >= 1 ? &pv_seen : nullptr);
+        SEG(1);
+        nja = list_check(it, 2 * t + 2, raw_a); njb = list_check(it, 2 * t + 3, raw_b);
+        SEG(2);
+        if (!fail && !pv_seen) fail = !mbar_wait(sh, bb + PV_DONE, (cnt - 1) & 1u, status);
+        SEG(3);
+        // P^T is stored at once; the vote on the tile (does any entry reach 2^(kRefShift + 1) times its reference
+        // maximum, or has a wait been lost?) comes after the stores, where the group has to meet anyway, and the
+        // issuer is told only after it
+        auto store_p = [&]() {
+          const uint32_t prow = p_base + (uint32_t)r * 128u;
 #pragma unroll
           for (int ck = 0; ck < 8; ++ck) {
             const uint32_t a = prow + (uint32_t)((ck ^ (r & 7)) << 4);
             asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(pk[ck * 4]), "r"(pk[ck * 4 + 1]),
                          "r"(pk[ck * 4 + 2]), "r"(pk[ck * 4 + 3]) : "memory");
           }
-        }
-        tr.ev(27, 0);
+        };
+        store_p();
+        SEG(6);
+        // the next tile's S^T: asked now, looked at when the next tile starts
+        s_seen = t + 1 < it.ntiles && mbar_test(sh.bar(bb + S_FULL + (int)(sbuf ^ 1u)), ((cnt + 1) >> 1) & 1u);
         fence_async_smem();
-        tr.ev(28, 0);
-        // one arrival per warp (128 would serialise on the barrier word); it also hands the S^T buffer back
         tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(sh.bar(P_FULL + 2 * grp + (int)sbuf));
-        tr.ev(25, gbase + t);
+        const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
+        SEG(4);
+        if (slow) {
+          // the -R row may only change when the S^T of the next tile, issued with the old row, has been computed
+          if (!fail && t + 1 < it.ntiles) fail = !mbar_wait(sh, bb + S_FULL + (int)(sbuf ^ 1u), ((cnt + 1) >> 1) & 1u, status);
+          tc_fence_after();
+          if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
+          SEG(8);
+          if constexpr (kTrace) ++nreb;
+          // ---- rebase: take this tile's contribution out of the row sums again, find the exact column maxima, move
+          // the references, rescale the row sums and O^T, and recompute the tile
+          if (have_ref) {
+            if (masked) tile_pass<true, true>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk);
+            else tile_pass<false, true>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk);
+          }
+          // column maxima of the accumulator (s - R of the buffer): over the lanes of each warp by shuffles (16 columns
+          // at a time: lane pair l, l ^ 1 ends with column l >> 1 of the chunk), over the four warps through shared memory
+#pragma unroll 2
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t sv[16];
+            tc_ld16(s_addr + ch * 16, sv);
+            tc_wait_ld(sv);
+            SEG(9);
+            float xv[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const int c = ch * 16 + e;
+              float x = __uint_as_float(sv[e]);
+              if (!row_live || (diag && key_local > c)) x = -CUDART_INF_F;
+              xv[e] = x;
+            }
+            const float cm = warp_colmax16(xv, lane);
+            if ((lane & 1) == 0) lsum[gw * 64 + ch * 16 + (lane >> 1)] = cm;
+            SEG(10);
+          }
+          tc_fence_before();                             // this thread's reads of the S^T buffer are done
+          named_bar_sync(bar_sync, kGroupThreads);
+          if (gt < 64) {
+            const float old = have_ref ? rcur[gt] : 0.f;   // (an item's first tiles hold the raw scores)
+            // largest raw score of the column in this tile
+            const float cm = fmaxf(fmaxf(lsum[gt], lsum[64 + gt]), fmaxf(lsum[128 + gt], lsum[192 + gt])) + old;
+            float nr;
+            if (!have_ref) nr = cm == -CUDART_INF_F ? kNoRef : bf16_ceil(cm + shift_raw);
+            else nr = cm == -CUDART_INF_F ? old : fmaxf(old, bf16_ceil(cm + shift_raw));
+            // a query column past the end of a ragged block holds whatever tokens follow in the packed tensor; the
+            // masked pass drops it, and it never moves a reference (results must not depend on the neighbours in the batch)
+            if (gt >= it.q_valid) nr = old;
+            const float d = old - nr;
+            alpha[gt] = have_ref ? exp2f(d * sl2) : 0.f;
+            rcur[gt] = nr;
+            qext[gt * 8] = (uint16_t)((__float_as_uint(nr) >> 16) ^ 0x8000u);   // -R[c] as bf16, column 0 of row c
+            // d = R_old - R_new in three bf16 terms (truncations, so every remainder is exact), columns 0..2 of row c
+            const uint32_t hi = __float_as_uint(d) & 0xffff0000u;
+            const float r1 = d - __uint_as_float(hi);
+            const uint32_t mid = __float_as_uint(r1) & 0xffff0000u;
+            const uint32_t lo = __float_as_uint(r1 - __uint_as_float(mid)) & 0xffff0000u;
+            *reinterpret_cast<uint2*>(qfix + gt * 8) = make_uint2((hi >> 16) | mid, lo >> 16);
+            fence_async_smem();
+          }
+          named_bar_sync(bar_sync, kGroupThreads);
+          SEG(11);
+          // the S^T tiles computed with the old row (this one and the next) get ones x (R_old - R_new) added in place
+          if (gt == 0) {
+            tc_fence_after();
+            tc_mma(tmem + col_s(s, sbuf), ones_d, qfix_d, kIdescS, 1u);
+            if (t + 1 < it.ntiles) tc_mma(tmem + col_s(s, sbuf ^ 1u), ones_d, qfix_d, kIdescS, 1u);
+            tc_commit(sh.bar(bb + FIXED));
+          }
+          if (have_ref) {                                // row sums (and, after the first tile, O^T) accumulated so far
+            // a reference that moved by more than 2^30 makes everything accumulated so far negligible (and the value
+            // taken out above may not have been finite): start the column afresh
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+              const float4 a = *reinterpret_cast<const float4*>(&alpha[c]);
+              l_part[c] = a.x < 9.3e-10f ? 0.f : l_part[c] * a.x;
+              l_part[c + 1] = a.y < 9.3e-10f ? 0.f : l_part[c + 1] * a.y;
+              l_part[c + 2] = a.z < 9.3e-10f ? 0.f : l_part[c + 2] * a.z;
+              l_part[c + 3] = a.w < 9.3e-10f ? 0.f : l_part[c + 3] * a.w;
+            }
+#pragma unroll 1
+            for (int ch = 0; ch < (t >= 1 ? 4 : 0); ++ch) {
+              uint32_t ov[16];
+              tc_ld16(o_addr + ch * 16, ov);
+              tc_wait_ld(ov);
+#pragma unroll
+              for (int e = 0; e < 16; e += 4) {
+                const float4 a = *reinterpret_cast<const float4*>(&alpha[ch * 16 + e]);
+                ov[e] = __float_as_uint(__uint_as_float(ov[e]) * a.x);
+                ov[e + 1] = __float_as_uint(__uint_as_float(ov[e + 1]) * a.y);
+                ov[e + 2] = __float_as_uint(__uint_as_float(ov[e + 2]) * a.z);
+                ov[e + 3] = __float_as_uint(__uint_as_float(ov[e + 3]) * a.w);
+              }
+              tc_st16(o_addr + ch * 16, ov);
+            }
+            tc_wait_st();
+          }
+          SEG(12);
+          if (named_bar_or(bar_vote, kGroupThreads, !mbar_wait(sh, bb + FIXED, nfix & 1u, status))) { ok = false; break; }
+          SEG(13);
+          ++nfix;
+          tc_fence_after();
+          if (masked) tile_pass<true, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk);
+          else tile_pass<false, false>(s_addr, sl2, row_live, diag, key_local, it.q_valid, l_part, pk);
+          store_p();
+          fence_async_smem();
+          tc_fence_before();
+          named_bar_sync(bar_sync, kGroupThreads);
+          s_seen = false;
+          SEG(14);
+        }
+        SEG(5);
+        // every thread's stores are visible to the MMA: one arrival hands P^T over and the S^T buffer back
+        if (gt == 0) mbar_arrive(sh.bar(bb + P_FULL));
+        SEG(7);
       }
-      gbase += (uint32_t)it.ntiles;
+      if (!ok) break;
 
       // ------------------------------------------------------------------------------------------ epilogue
-      tr.sample(0); tr.ev(30, (uint32_t)(w / gridDim.x));
-      bool efail = !ok;
-      if (ok && my_tiles > 0) {                          // the last P V on each P^T buffer (cnt tiles so far in this CTA)
-        efail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)((cnt - 1) & 1u), ((cnt - 1) >> 1) & 1u, status);
-        if (!efail && cnt >= 2) efail = !mbar_wait(sh, PV_DONE + 2 * grp + (int)(cnt & 1u), ((cnt - 2) >> 1) & 1u, status);
-      }
+      tr.sample(0); tr.ev(30, 0);
+      const bool efail = !mbar_wait(sh, bb + PV_DONE, (cnt - 1) & 1u, status);   // the last P V of the item
       tc_fence_after();
       {
         float s0, s1; int base;
@@ -867,63 +646,50 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         lsum[gw * 64 + base] = s0;
         lsum[gw * 64 + base + 1] = s1;
       }
-      named_bar_sync(bar_sync, kGroupThreads);
-      if (gt < 64) lfin[gt] = (lsum[gt] + lsum[64 + gt]) + (lsum[128 + gt] + lsum[192 + gt]);
-      // both groups: partial sums and references published, all P V of the item finished (or a wait was lost)
-      if (named_bar_or(5, 2 * kGroupThreads, efail)) { ok = false; break; }
-      if (grp == 0 && gt < 64) {
-        const float la = lfin_a[gt], lb = tiles_b > 0 ? lfin_b[gt] : 0.f;
-        const float ma = la > 0.f ? mref_a[gt] : -CUDART_INF_F, mb = lb > 0.f ? mref_b[gt] : -CUDART_INF_F;
-        const float mm = fmaxf(ma, mb);
-        float wa = 0.f, wb = 0.f, out_lse = -CUDART_INF_F;
-        if (mm != -CUDART_INF_F) {
-          const float fa = la > 0.f ? exp2f(ma - mm) : 0.f, fb = lb > 0.f ? exp2f(mb - mm) : 0.f;
-          const float l = la * fa + lb * fb;
-          wa = fa / l; wb = fb / l;
-          out_lse = (mm + log2f(l)) * 0.6931471805599453f;
-        }
-        w_a[gt] = wa; w_b[gt] = wb;
-        if (lse != nullptr && gt < it.q_valid) lse[(int64_t)it.h * (kChunk ? m.total_q_tokens : m.total_tokens) + tok0 + gt] = out_lse;
+      if (named_bar_or(bar_vote, kGroupThreads, efail)) { ok = false; break; }
+      if (gt < 64) {
+        const float l = (lsum[gt] + lsum[64 + gt]) + (lsum[128 + gt] + lsum[192 + gt]);
+        alpha[gt] = l > 0.f ? 1.f / l : 0.f;
+        if (lse != nullptr && gt < it.q_valid)
+          lse[(int64_t)it.h * (kChunk ? m.total_q_tokens : m.total_tokens) + tok0 + gt] =
+              l > 0.f ? (rcur[gt] * sl2 + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
       }
-      named_bar_sync(5, 2 * kGroupThreads);
-      // each group merges and stores 32 of the 64 query columns: staging [32 q][128 d] bf16 in its own P^T buffer
+      named_bar_sync(bar_sync, kGroupThreads);
+      // O^T row r (one d of all 64 queries) -> staging [64 q][128 d] bf16 in the stream's P^T buffer
       {
-        uint16_t* stage = reinterpret_cast<uint16_t*>(smem + kOffP + 2 * grp * kPBytes);
-        const int c0 = grp * 32;
+        uint16_t* stage = reinterpret_cast<uint16_t*>(p_gen);
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          uint32_t oa[16], ob[16];
-          if (tiles_a > 0) { tc_ld16(tmem + lane_addr + col_o(0) + c0 + ch * 16, oa); tc_wait_ld(oa); }
-          if (tiles_b > 0) { tc_ld16(tmem + lane_addr + col_o(1) + c0 + ch * 16, ob); tc_wait_ld(ob); }
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t ov[16];
+          tc_ld16(o_addr + ch * 16, ov);
+          tc_wait_ld(ov);
 #pragma unroll
           for (int e = 0; e < 16; e += 4) {
-            const int c = c0 + ch * 16 + e;
-            const float4 fa = *reinterpret_cast<const float4*>(&w_a[c]), fb = *reinterpret_cast<const float4*>(&w_b[c]);
-            const float wa4[4] = {fa.x, fa.y, fa.z, fa.w}, wb4[4] = {fb.x, fb.y, fb.z, fb.w};
+            const float4 f = *reinterpret_cast<const float4*>(&alpha[ch * 16 + e]);
+            const float w4[4] = {f.x, f.y, f.z, f.w};
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              float val = 0.f;
-              if (tiles_a > 0) val = __uint_as_float(oa[e + u]) * wa4[u];
-              if (tiles_b > 0) val = fmaf(__uint_as_float(ob[e + u]), wb4[u], val);
-              stage[(ch * 16 + e + u) * 128 + r] = (uint16_t)(pack_bf16(val, 0.f) & 0xffffu);
-            }
+            for (int u = 0; u < 4; ++u)
+              stage[(ch * 16 + e + u) * 128 + r] = (uint16_t)(pack_bf16(__uint_as_float(ov[e + u]) * w4[u], 0.f) & 0xffffu);
           }
         }
       }
       tc_fence_before();
-      named_bar_sync(5, 2 * kGroupThreads);   // every TMEM read of the item is done: the next item may overwrite O^T
+      named_bar_sync(bar_sync, kGroupThreads);   // O^T has been read (the next item's first P V waits for this group's P^T anyway)
       {
-        const uint4* stage4 = reinterpret_cast<const uint4*>(smem + kOffP + 2 * grp * kPBytes);
-        for (int idx = gt; idx < 32 * 16; idx += kGroupThreads) {
-          const int qrow = grp * 32 + (idx >> 4), chunk = idx & 15;
+        const uint4* stage4 = reinterpret_cast<const uint4*>(p_gen);
+        for (int idx = gt; idx < 64 * 16; idx += kGroupThreads) {
+          const int qrow = idx >> 4, chunk = idx & 15;
           if (qrow < it.q_valid)
             *reinterpret_cast<uint4*>(o + ((tok0 + qrow) * m.num_q_heads + it.h) * kHeadDim + chunk * 8) = stage4[idx];
         }
       }
-      named_bar_sync(bar_sync, kGroupThreads);   // staging is free again before this group's next P^T
-      tr.ev(31, (uint32_t)(w / gridDim.x));
+      named_bar_sync(bar_sync, kGroupThreads);   // staging is free again before the next P^T
+      tr.ev(31, 0);
     }
+    if constexpr (kTrace) if (tr.p != nullptr)
+      for (int k = 0; k < 15; ++k) { tr.acc[2 * (32 + k)] = (unsigned long long)seg[k]; tr.acc[2 * (32 + k) + 1] = k >= 8 ? nreb : seg_n; }
     tr.flush();
+#undef SEG
   }
 
   // ------------------------------------------------------------------------------------------------ teardown
@@ -974,7 +740,7 @@ seer_status init_attn_tc(seer_ctx* ctx) {
 }
 
 int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
-                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream) {
+                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream) {
   if (m.rows == 0) return 0;
   // the input pointers must be 16-byte aligned for TMA
   if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15) != 0) return -(int)cudaErrorMisalignedAddress;
@@ -982,16 +748,14 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
   if (!tc::make_map(ctx, &mq, q, m.total_q_tokens, m.num_q_heads) || !tc::make_map(ctx, &mk, k, m.total_tokens, m.num_kv_heads) ||
       !tc::make_map(ctx, &mv, v, m.total_tokens, m.num_kv_heads))
     return -(int)cudaErrorInvalidValue;
-  const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, m.rows);
+  const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, (m.rows + 1) / 2);
+  unsigned long long* tb = (unsigned long long*)ctx->trace;
   if (m.chunked)               // chunked prefill (never instrumented)
-    tc::attn_tc_kernel<false, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
-                                                                          ctx->d_status, (unsigned long long*)ctx->trace);
-  else if (ctx->trace != nullptr)   // the instrumented instantiation
-    tc::attn_tc_kernel<true, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
-                                                                    ctx->d_status, (unsigned long long*)ctx->trace);
+    tc::attn_tc_kernel<false, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
+  else if (tb != nullptr)      // the instrumented instantiation
+    tc::attn_tc_kernel<true, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
   else
-    tc::attn_tc_kernel<false, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, k, v, (uint16_t*)o, lse,
-                                                                    ctx->d_status, (unsigned long long*)ctx->trace);
+    tc::attn_tc_kernel<false, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;
 }

@@ -10,7 +10,6 @@
 namespace seer {
 namespace tcc {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is declared lost
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -36,6 +35,7 @@ struct Shared {
   uint32_t base;         // 1024-aligned shared address
   uint32_t bar0;         // shared address of mbarrier 0
   uint32_t abort_addr;   // shared address of the abort flag
+  unsigned long long limit_ns;   // a wait that lasts this long is declared lost (2 s unless a test shortens it)
   __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
   __device__ __forceinline__ uint32_t abort_flag() const { return abort_addr; }
 };
@@ -65,25 +65,14 @@ __device__ __forceinline__ bool mbar_wait(const Shared& sh, int bar, uint32_t pa
                  : "=r"(done) : "r"(addr), "r"(parity) : "memory");
     if (done) return true;
   }
-#ifdef SEER_SPIN_TEST
-  const unsigned long long t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    {
-      uint32_t done;
-      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                   : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-      if (done) return true;
-    }
-#else
   if (mbar_try(addr, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try(addr, parity)) return true;
-#endif
     if (kSleepNs > 0) __nanosleep(kSleepNs);   // a waiting helper must not take issue slots from the softmax warps of its scheduler
     if ((it & 255u) == 0u) {
       if (ld_shared_u32(sh.abort_flag()) != 0u) return false;
-      if (global_ns() - t0 > kWaitLimitNs) break;
+      if (global_ns() - t0 > sh.limit_ns) break;
     }
   }
   st_shared_u32(sh.abort_flag(), 1u);

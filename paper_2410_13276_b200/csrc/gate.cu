@@ -580,8 +580,8 @@ int launch_gate_scores_band(const SeqMeta& m, const ScoreBand& band, const void*
 // bytes until the process exits.  Host code must never hand the symbol itself to a kernel; its device address is
 // looked up once per device with cudaGetSymbolAddress.
 constexpr int kStaticMaxBatch = SEER_STATIC_MAX_BATCH;
-constexpr size_t kStaticMetaBytes = 16 * 1024;                              // cu_seqlens + four offset arrays
-constexpr size_t kStaticScratchBytes = (size_t)SEER_STATIC_SCRATCH_BYTES;   // projected pooled Q and K (fp32)
+constexpr size_t kStaticMetaBytes = 16 * 1024;                              // cu_seqlens and the two offset arrays (block, score)
+constexpr size_t kStaticScratchBytes = (size_t)SEER_STATIC_SCRATCH_BYTES;   // projected pooled Q and K, three bf16 planes each (768 B per (head, block))
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticMetaBytes + kStaticScratchBytes];
 
 constexpr int kStaticMaxDevices = 64;
@@ -621,12 +621,16 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   st = static_setup(dev, &base);
   if (st != SEER_OK) return st;
 
-  // per-batch offsets, built on the host stack and copied into the head of the array
+  // per-batch offsets, built in a host staging area that lives as long as the library (one per device, so that the
+  // copy below never refers to a stack frame that has gone) and copied into the head of the array
   struct HostMeta {
     int32_t cu[kStaticMaxBatch + 4], blk[kStaticMaxBatch + 4];
     int64_t score[kStaticMaxBatch + 2];
-  } hm;
+  };
   static_assert(sizeof(HostMeta) <= kStaticMetaBytes, "metadata region too small");
+  static HostMeta g_host_meta[kStaticMaxDevices];
+  std::lock_guard<std::mutex> lock(g_static_mutex);   // (static_setup has released it)
+  HostMeta& hm = g_host_meta[dev];
   hm.blk[0] = 0;
   hm.score[0] = 0;
   for (int b = 0; b < shape->batch; ++b) {
@@ -636,7 +640,7 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
     hm.score[b + 1] = hm.score[b] + (int64_t)shape->num_q_heads * nb * nb;
   }
   hm.cu[shape->batch] = shape->cu_seqlens_host[shape->batch];
-  // pageable source: the runtime stages the bytes before returning, so the stack buffer may go out of scope
+  // pageable source: the runtime stages the bytes before returning, so the next call may refill the staging area
   if (cudaMemcpyAsync(base, &hm, sizeof(HostMeta), cudaMemcpyHostToDevice, stream) != cudaSuccess) return SEER_ERR_CUDA;
 
   SeqMeta m;
@@ -657,6 +661,7 @@ seer_status gate_scores_static(const seer_shape* shape, const void* q, const voi
   m.block = shape->block;
   m.qoff = nullptr; m.qdelta = nullptr; m.chunked = 0;
   m.total_q_tokens = (int32_t)t.total_tokens;
+  m.wait_limit_us = 0u; m.lose_v_copy = -1;   // unused by the gate
   // The two kernels below are the ones seer_gate_scores launches; only the scratch pointer differs.  Nothing in the
   // scratch has to start at zero: the first kernel writes every projected vector the second one reads.
   const int n = launch_gate(nullptr, m, q, k, Wq, Wk, scores, base + kStaticMetaBytes, stream);

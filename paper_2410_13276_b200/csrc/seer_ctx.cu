@@ -81,13 +81,24 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   for (int i = 0; i < kMetaSlots; ++i)
     if (ctx->slots[i].key == key) { slot = i; break; }
   if (slot < 0) {
-    slot = 0;
-    for (int i = 1; i < kMetaSlots; ++i)
-      if (ctx->slots[i].stamp < ctx->slots[slot].stamp) slot = i;
+    // the least recently used slot whose last reader and last upload have finished; only if every slot is still
+    // in flight (more than kMetaSlots shapes cycling faster than the GPU works through them) does the call wait
+    // for the oldest one
+    slot = -1;
+    int oldest = 0;
+    for (int i = 0; i < kMetaSlots; ++i) {
+      if (ctx->slots[i].stamp < ctx->slots[oldest].stamp) oldest = i;
+      if (cudaEventQuery(ctx->slots[i].last_use) == cudaSuccess && cudaEventQuery(ctx->slots[i].ready) == cudaSuccess &&
+          (slot < 0 || ctx->slots[i].stamp < ctx->slots[slot].stamp))
+        slot = i;
+    }
+    (void)cudaGetLastError();                        // cudaErrorNotReady from the queries is not an error
+    if (slot < 0) {
+      slot = oldest;
+      if (cudaEventSynchronize(ctx->slots[slot].last_use) != cudaSuccess) return SEER_ERR_CUDA;
+      if (cudaEventSynchronize(ctx->slots[slot].ready) != cudaSuccess) return SEER_ERR_CUDA;
+    }
     MetaSlot& s = ctx->slots[slot];
-    // The slot may still be read by kernels of earlier calls, and its staging buffer by an earlier upload.
-    if (cudaEventSynchronize(s.last_use) != cudaSuccess) return SEER_ERR_CUDA;
-    if (cudaEventSynchronize(s.ready) != cudaSuccess) return SEER_ERR_CUDA;
     char* h = (char*)s.pinned;
     int32_t* cu = (int32_t*)(h + kOffCu);
     int32_t* blk = (int32_t*)(h + kOffBlk);
@@ -137,6 +148,8 @@ seer_status prepare(seer_ctx* ctx, const seer_shape* shape, cudaStream_t stream,
   m->qdelta = (const int32_t*)(d + kOffQdelta);
   m->total_q_tokens = (int32_t)t.total_q_tokens;
   m->chunked = shape->cu_seqlens_q_host ? 1 : 0;
+  m->wait_limit_us = ctx->wait_limit_us;
+  m->lose_v_copy = ctx->lose_v_copy;
   *slot_out = slot;
   return SEER_OK;
 }
@@ -198,7 +211,7 @@ seer_status seer_create(seer_ctx** out, int device) {
          cudaEventCreateWithFlags(&ctx->ev_comp[i], cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&ctx->ev_d2h[i], cudaEventDisableTiming) == cudaSuccess;
   if (ok) ok = init_gate(ctx) == SEER_OK && init_mask(ctx) == SEER_OK && init_attn_mma(ctx) == SEER_OK &&
-              init_attn_tc(ctx) == SEER_OK && init_attn_tc2(ctx) == SEER_OK && init_attn_tcs(ctx) == SEER_OK;
+              init_attn_tc(ctx) == SEER_OK;
   if (!ok) { seer_destroy(ctx); return SEER_ERR_CUDA; }
   *out = ctx;
   return SEER_OK;
@@ -271,6 +284,26 @@ seer_status seer_gate_scores(seer_ctx* ctx, const seer_shape* shape, const void*
   return SEER_OK;
 }
 
+seer_status seer_gate_project(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k, const float* Wq,
+                              const float* Wk, void* ws, size_t ws_bytes, void* stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (!ctx || !shape) return SEER_ERR_INVALID_ARG;
+  ShapeTotals t;
+  seer_status st = shape_totals(shape, &t);
+  if (st != SEER_OK) return st;
+  if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;
+  if (!q || !k || !Wq || !Wk) return SEER_ERR_INVALID_ARG;
+  if (!ws_ok(ws, ws_bytes, gate_workspace_bytes(t, shape))) return SEER_ERR_WORKSPACE;
+  SeqMeta m; int slot;
+  st = prepare(ctx, shape, stream, &m, &slot);
+  if (st != SEER_OK) return st;
+  int n = launch_gate(ctx, m, q, k, Wq, Wk, nullptr, ws, stream);   // no score buffer: pooling and projection only
+  finish_call(ctx, slot, stream);
+  if (n < 0) return SEER_ERR_CUDA;
+  ctx->launches += n;
+  return SEER_OK;
+}
+
 seer_status seer_gate_scores_ex(seer_ctx* ctx, const seer_shape* shape, const seer_gate_options* opt, const void* q,
                                 const void* k, const float* Wq, const float* Wk, float* scores, void* ws, size_t ws_bytes,
                                 void* stream_) {
@@ -331,7 +364,7 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   if (st != SEER_OK) return st;
   if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;   // 128-token lists go through seer_expand_block_lists first
   if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;   // no output row
-  if (!q || !k || !v || !row_ptr || !o) return SEER_ERR_INVALID_ARG;
+  if (!q || !k || !v || !row_ptr || !col_idx || !o) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
   if (st != SEER_OK) return st;
@@ -339,9 +372,7 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   // per-row hand-over than the legacy kernel needs for the whole row.
   const bool legacy = ctx->attn_impl == 1 || (ctx->attn_impl == 2 && t.causal_blocks <= 8 * t.rows);
   int n = legacy ? launch_attn_mma(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
-          : ctx->attn_impl == 3 ? launch_attn_tc2(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
-          : ctx->attn_impl == 4 ? launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
-                                : launch_attn_tcs(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream);
+                 : launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream);
   finish_call(ctx, slot, stream);
   if (n < 0) return SEER_ERR_CUDA;
   ctx->launches += n;
@@ -358,7 +389,7 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
   if (st != SEER_OK) return st;
   if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;
   if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;
-  if (!q || !k || !row_ptr || !lse) return SEER_ERR_INVALID_ARG;
+  if (!q || !k || !row_ptr || !col_idx || !lse || !block_max) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
   if (st != SEER_OK) return st;
@@ -513,8 +544,15 @@ seer_status seer_expand_block_lists(seer_ctx* ctx, const seer_shape* shape, cons
   return SEER_OK;
 }
 
+seer_status seer_debug_lost_wait(seer_ctx* ctx, uint32_t wait_limit_us, int32_t lose_v_copy_of_tile) {
+  if (!ctx || wait_limit_us == 0u) return SEER_ERR_INVALID_ARG;
+  ctx->wait_limit_us = wait_limit_us;
+  ctx->lose_v_copy = lose_v_copy_of_tile;
+  return SEER_OK;
+}
+
 seer_status seer_set_attn_impl(seer_ctx* ctx, int impl) {
-  if (!ctx || impl < 0 || impl > 4) return SEER_ERR_INVALID_ARG;
+  if (!ctx || impl < 0 || impl > 2) return SEER_ERR_INVALID_ARG;
   ctx->attn_impl = impl;
   return SEER_OK;
 }

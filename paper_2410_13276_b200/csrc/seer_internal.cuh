@@ -40,6 +40,9 @@ struct SeqMeta {
   const int32_t* qdelta;       // [batch] token index in q / o / lse = token index in k / v + qdelta
   int32_t total_q_tokens;      // tokens in q / o / lse
   int32_t chunked;             // 1 if the shape carries cu_seqlens_q
+  // bounded waits of the tcgen05 attention kernel, and the test hook that makes one of them run out
+  uint32_t wait_limit_us;      // a barrier wait that lasts this long is declared lost
+  int32_t lose_v_copy;         // >= 0: stream 0 of CTA 0 never issues the V copy of its tile with this ordinal
 };
 
 // A rectangle of (block row of the packed batch, query head) pairs whose scores are produced and consumed together.
@@ -72,6 +75,8 @@ struct seer_ctx {
   seer::MetaSlot slots[seer::kMetaSlots];
   void* tmap_encode = nullptr;   // cuTensorMapEncodeTiled, resolved at run time
   void* trace = nullptr;         // optional device buffer for the attention kernel's timeline (diagnostics)
+  uint32_t wait_limit_us = 2000000u;   // seer_debug_lost_wait
+  int32_t lose_v_copy = -1;
   // seer_prefill_host: copy streams and the events of its two-deep pipeline over KV-head slices
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
   cudaEvent_t ev_start = nullptr, ev_h2d[2] = {nullptr, nullptr}, ev_comp[2] = {nullptr, nullptr},
@@ -120,13 +125,8 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
 seer_status init_gate(seer_ctx* ctx);
 seer_status init_mask(seer_ctx* ctx);
 seer_status init_attn_mma(seer_ctx* ctx);
-int launch_attn_tc2(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
-                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
 seer_status init_attn_tc(seer_ctx* ctx);
-seer_status init_attn_tc2(seer_ctx* ctx);
-int launch_attn_tcs(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
-                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
-seer_status init_attn_tcs(seer_ctx* ctx);
+
 
 // Sequence that owns global block index gb: largest b with blk_off[b] <= gb (empty sequences are skipped).
 __device__ __forceinline__ int find_sequence(const int32_t* __restrict__ off, int batch, int x) {

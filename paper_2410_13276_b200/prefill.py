@@ -82,6 +82,10 @@ class Prefill:
     def gate(self, stream=None):
         B.seer_gate_scores(self.ctx, self.shape, self.q, self.k, self.wq, self.wk, self.scores, self.ws, stream)
 
+    def gate_project(self, stream=None):
+        """Pooling and projection only (the first kernel of the gate)."""
+        B.seer_gate_project(self.ctx, self.shape, self.q, self.k, self.wq, self.wk, self.ws, stream)
+
     def gate_ex(self, options: B.seer_gate_options, wq, wk, stream=None):
         """Gate with composed pooling and / or block-level RoPE (Sec. 3.1); wq, wk are device tensors
         [heads, n * 128, 128] matching the pooling subsets in `options`."""

@@ -400,7 +400,7 @@ def test_attention_kernel_chosen_by_shape(rt):
             assert torch.equal(outs[2][0], outs[want][0]) and torch.equal(outs[2][1], outs[want][1])
             assert not torch.equal(outs[0][0], outs[1][0])                  # the two kernels round differently
         with pytest.raises(B.SeerError):
-            B.seer_set_attn_impl(ctx, 9)
+            B.seer_set_attn_impl(ctx, 3)
     finally:
         B.seer_set_attn_impl(ctx, 0)
 
@@ -465,7 +465,7 @@ def test_output_does_not_depend_on_the_neighbours_in_the_batch(rt):
     S, hq, hkv = 333, 2, 1
     w = W.make_small(seed=52_000, seqlens=[S], hq=hq, hkv=hkv, q_gain=2.0)
     rp, col = O.full_causal_lists([0, S], 64, hq)
-    for impl in (0, 3):
+    for impl in (0,):
         B.seer_set_attn_impl(ctx, impl)
         try:
             _neighbour_case(B, Prefill, ctx, w, rp, col, S, hq, hkv)

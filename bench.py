@@ -30,7 +30,8 @@ sys.path.insert(0, ROOT)
 
 FLOP_PER_BLOCK = 4 * 64 * 64 * 128
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of the default command, and the capture it is from
-TRAFFIC_C3_KEEP10 = (None, "not captured yet")
+TRAFFIC_C3_KEEP10 = (7.62e9, "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch of this command "
+                                 "(summary: profiles/attn_tc_kernel_c3_seq131072_keep10_dram.md)")
 METRIC = "sparse_prefill_attention_effective_tflops_128k_90pct_block_sparsity"
 
 
@@ -608,8 +609,7 @@ def main():
         achieved = flops / (attn_ms * 1e-3) / 1e12
         gate_pool_bytes = (w.num_q_heads + w.num_kv_heads) * (w.total_tokens * 256 + int(sum(w.num_blocks)) * 768)
         mask_bytes = (B.seer_causal_blocks(p.shape) + nnz + B.seer_mask_rows(p.shape)) * 4
-        # DRAM bytes of one attention launch from an ncu capture of this very command
-        # (profiles/attn_tc_kernel_c3_seq131072_keep10_dram.md); other workloads have no capture
+        # DRAM bytes of one attention launch from an ncu capture of this very command; other workloads have no capture
         traffic, traffic_source = None, "no ncu capture for this command"
         if w.name == "c3" and args.seq is None and (spec.keep_num, spec.keep_den) == (1, 10) and args.attn_impl == 0:
             traffic, traffic_source = TRAFFIC_C3_KEEP10

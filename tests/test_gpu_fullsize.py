@@ -1,8 +1,9 @@
 """Parity at the full sizes of the five workloads, in the launch configuration bench.py times (whole GPU path, default
-attention kernel).  The oracle cannot run attention in full at these sizes, so it checks (a) gate scores of a few heads,
-(b) the block lists of those heads, rebuilt from the GPU's own scores (bit-exact), (c) attention on a stratified sample
-of (head, query block) rows, one output element at a time, with the GPU's lists fed to both, and (d) properties that
-hold at any size (list lengths in closed form, ordering, range)."""
+attention kernel).  The oracle cannot run attention in full at these sizes, so it checks (a) the gate scores of every
+head, one head at a time, (b) the block lists of every head, rebuilt from the GPU's own scores (bit-exact), (c) attention
+on a stratified sample of rows of every (sequence, head) (the first two query blocks, the last, the longest and the
+shortest list, eight seeded-random ones) with the GPU's lists fed to both, (d) properties that hold at any size (list
+lengths in closed form, ordering, range), and (e) every output row against the independent mma.sync kernel."""
 import json
 import math
 import os
@@ -34,25 +35,22 @@ def golden_threshold(name):
         return float.fromhex(json.load(f)[name]["threshold_hex"])
 
 
-def head_slice_scores(flat, w, heads):
-    per_seq = O.unflatten_scores(flat, w.cu_seqlens, 64, w.num_q_heads)
-    return [s[heads] for s in per_seq]
-
-
-def check_workload(rt, name, specs, sample_heads, rows_per_head=3):
+def check_workload(rt, name, specs, sample_heads=None, rows_per_head=8, all_rows=False):
     B, Prefill, ctx = rt
     w = W.make_workload(name)
     G = w.num_q_heads // w.num_kv_heads
+    if sample_heads is None:
+        sample_heads = list(range(w.num_q_heads))
     p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx)
     p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
     p.gate()
-    gpu_scores = p.scores_host()
-    # (a) gate scores of the sampled heads against the oracle run on those heads alone
+    gpu_scores = O.unflatten_scores(p.scores_host(), w.cu_seqlens, 64, w.num_q_heads)   # per sequence [Hq, nb, nb] views
+    # (a) gate scores, head by head, against the oracle run on that head alone
     for h in sample_heads:
         g = h // G
         ref = O.gate_scores(np.ascontiguousarray(w.q[:, h:h + 1]), np.ascontiguousarray(w.k[:, g:g + 1]),
                             w.wq[h:h + 1], w.wk[g:g + 1], w.cu_seqlens, 64)
-        got = head_slice_scores(gpu_scores, w, [h])
+        got = [s[h:h + 1] for s in gpu_scores]
         for r, x in zip(ref, got):
             il = np.tril_indices(r.shape[-1])
             rr, xx = r[:, il[0], il[1]].astype(np.float64), x[:, il[0], il[1]].astype(np.float64)
@@ -94,7 +92,7 @@ def check_workload(rt, name, specs, sample_heads, rows_per_head=3):
         base = 0
         for b, nb in enumerate(nbs):
             for h in sample_heads:
-                s = head_slice_scores(gpu_scores, w, [h])[b]
+                s = gpu_scores[b][h:h + 1]
                 orp, ocol = O.block_mask([s], spec.mode, keep_num=spec.keep_num, keep_den=spec.keep_den, k=spec.k,
                                          threshold=spec.threshold or 0.0, flags=spec.flags)
                 r0 = base + h * nb
@@ -102,7 +100,8 @@ def check_workload(rt, name, specs, sample_heads, rows_per_head=3):
                 assert np.array_equal(col[rp[r0]:rp[r0 + nb]], ocol), (name, h)
             base += w.num_q_heads * nb
         # (c) attention on a stratified sample of rows with the GPU's lists
-        rows = W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=11, per_head_random=rows_per_head, heads=sample_heads)
+        rows = None if all_rows else W.sample_rows(w.cu_seqlens, w.num_q_heads, rp, seed=11,
+                                                   per_head_random=rows_per_head, heads=sample_heads)
         o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, w.num_q_heads, w.num_kv_heads, 64,
                                             1 / math.sqrt(128), rows=rows)
         done = ~np.isnan(o_ref[..., 0])
@@ -120,31 +119,40 @@ def check_workload(rt, name, specs, sample_heads, rows_per_head=3):
 def test_c3_128k_topk_bench_configuration(rt):
     specs = [W.MaskSpec(W.MODE_TOPK_RATIO, 1, 10, flags=W.FORCE_DIAG | W.FORCE_SINK),
              W.MaskSpec(W.MODE_TOPK_RATIO, 1, 2, flags=W.FORCE_DIAG | W.FORCE_SINK)]
-    check_workload(rt, "c3", specs, sample_heads=[0, 13, 31], rows_per_head=2)
+    check_workload(rt, "c3", specs)
 
 
-@pytest.mark.parametrize("name,heads", [("c2", [3, 28]), ("c4", [0, 22, 39]), ("c5", [5, 7, 16])])
-def test_threshold_workloads_full_size(rt, name, heads):
+def test_c1_full_size_every_row(rt):
+    """The smallest workload: the oracle runs the whole of it (every head, every attention row)."""
+    check_workload(rt, "c1", [W.make_workload("c1").masks[0]], all_rows=True)
+
+
+@pytest.mark.parametrize("name", ["c2", "c4", "c5"])
+def test_threshold_workloads_full_size(rt, name):
     w_spec = W.make_workload(name + "s").masks[0]            # same mask recipe as the full-size workload
     spec = W.MaskSpec(W.MODE_THRESHOLD, threshold=golden_threshold(name), flags=w_spec.flags)
-    check_workload(rt, name, [spec], sample_heads=heads, rows_per_head=2)
+    check_workload(rt, name, [spec])
 
 
-@pytest.mark.parametrize("impl", [0])
-def test_c3_bench_configuration_all_rows_cross_check(rt, impl):
-    """Every output row of the bench workload, not a sample: each tcgen05 kernel against the independent mma.sync kernel
-    (different tiling, layout and softmax scheme; itself checked against the oracle on the small cases) on the same
-    lists.  Both round P and o to bf16, so the bound is the attention tolerance between two results of that kind."""
+def full_size_params(B, name):
+    if name == "c3":
+        return B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=10, flags=3)
+    w_spec = W.make_workload(name + "s").masks[0]
+    return B.make_mask_params(B.SEER_THRESHOLD, threshold=golden_threshold(name), flags=w_spec.flags)
+
+
+@pytest.mark.parametrize("name", ["c3", "c2", "c4", "c5"])
+def test_full_size_all_rows_cross_check(rt, name):
+    """Every output row of the full-size workloads, not a sample: the tcgen05 kernel against the independent mma.sync
+    kernel (different tiling, layout and softmax scheme; itself checked against the oracle on the small cases) on the
+    same lists.  Both round P and o to bf16, so the bound is the attention tolerance between two results of that kind."""
     import torch
     B, Prefill, ctx = rt
-    w = W.make_workload("c3")
+    w = W.make_workload(name)
     p = Prefill(w.cu_seqlens, w.num_q_heads, w.num_kv_heads, ctx=ctx)
     p.set_inputs(w.q, w.k, w.v, w.wq, w.wk)
-    B.seer_set_attn_impl(ctx, impl)
-    try:
-        p.run(B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=10, flags=3))
-    finally:
-        B.seer_set_attn_impl(ctx, 0)
+    B.seer_set_attn_impl(ctx, 0)
+    p.run(full_size_params(B, name))
     assert p.status() == 0
     o_tc = p.o.float().clone()
     lse_tc = p.lse.clone()

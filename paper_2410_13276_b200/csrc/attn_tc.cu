@@ -655,9 +655,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
               l > 0.f ? (rcur[gt] * sl2 + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
       }
       named_bar_sync(bar_sync, kGroupThreads);
-      // O^T row r (one d of all 64 queries) -> staging [64 q][128 d] bf16 in the stream's P^T buffer
+      // O^T row r (one d of all 64 queries) -> staging in the stream's P^T buffer as [32 query pairs][128 d] words, a
+      // word holding the two queries of a pair for one d: every store is a full word per lane, a warp's stores one
+      // 128-byte line (two-byte stores of single elements cost two wavefronts each and twice as many instructions)
       {
-        uint16_t* stage = reinterpret_cast<uint16_t*>(p_gen);
+        uint32_t* stage = reinterpret_cast<uint32_t*>(p_gen);
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           uint32_t ov[16];
@@ -666,21 +668,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
           for (int e = 0; e < 16; e += 4) {
             const float4 f = *reinterpret_cast<const float4*>(&alpha[ch * 16 + e]);
-            const float w4[4] = {f.x, f.y, f.z, f.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-              stage[(ch * 16 + e + u) * 128 + r] = (uint16_t)(pack_bf16(__uint_as_float(ov[e + u]) * w4[u], 0.f) & 0xffffu);
+            stage[((ch * 16 + e) >> 1) * 128 + r] = pack_bf16(__uint_as_float(ov[e]) * f.x, __uint_as_float(ov[e + 1]) * f.y);
+            stage[((ch * 16 + e + 2) >> 1) * 128 + r] = pack_bf16(__uint_as_float(ov[e + 2]) * f.z, __uint_as_float(ov[e + 3]) * f.w);
           }
         }
       }
       tc_fence_before();
       named_bar_sync(bar_sync, kGroupThreads);   // O^T has been read (the next item's first P V waits for this group's P^T anyway)
       {
+        // a thread takes eight d of a query pair: eight words in, the low halves are query 2p, the high halves query 2p + 1
         const uint4* stage4 = reinterpret_cast<const uint4*>(p_gen);
-        for (int idx = gt; idx < 64 * 16; idx += kGroupThreads) {
-          const int qrow = idx >> 4, chunk = idx & 15;
-          if (qrow < it.q_valid)
-            *reinterpret_cast<uint4*>(o + ((tok0 + qrow) * m.num_q_heads + it.h) * kHeadDim + chunk * 8) = stage4[idx];
+        for (int idx = gt; idx < 32 * 16; idx += kGroupThreads) {
+          const int pair = idx >> 4, chunk = idx & 15;
+          const uint4 w0 = stage4[pair * 32 + chunk * 2], w1 = stage4[pair * 32 + chunk * 2 + 1];
+          const uint4 lo = make_uint4(__byte_perm(w0.x, w0.y, 0x5410), __byte_perm(w0.z, w0.w, 0x5410),
+                                      __byte_perm(w1.x, w1.y, 0x5410), __byte_perm(w1.z, w1.w, 0x5410));
+          const uint4 hi = make_uint4(__byte_perm(w0.x, w0.y, 0x7632), __byte_perm(w0.z, w0.w, 0x7632),
+                                      __byte_perm(w1.x, w1.y, 0x7632), __byte_perm(w1.z, w1.w, 0x7632));
+          uint16_t* dst = o + ((tok0 + 2 * pair) * m.num_q_heads + it.h) * kHeadDim + chunk * 8;
+          if (2 * pair < it.q_valid) *reinterpret_cast<uint4*>(dst) = lo;
+          if (2 * pair + 1 < it.q_valid) *reinterpret_cast<uint4*>(dst + (size_t)m.num_q_heads * kHeadDim) = hi;
         }
       }
       named_bar_sync(bar_sync, kGroupThreads);   // staging is free again before the next P^T

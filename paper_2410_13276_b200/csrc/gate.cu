@@ -510,7 +510,19 @@ gate_scores_kernel(SeqMeta m, ScoreBand band, const uint16_t* __restrict__ gq, c
     float* dst = scores + row_off[r];
     if ((row_off[r] & 3) == 0) {
       const int full = n & ~3;                         // columns 0 .. full-1 in whole float4s
-      for (int j = lane * 4; j < full; j += 128) {
+      int j = lane * 4;
+      for (; j + 384 < full; j += 512) {               // four loads in flight per lane (the loop is bound by their latency)
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<float4*>(dst + j + u * 128);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          v[u].x = __expf(v[u].x - mm) * inv; v[u].y = __expf(v[u].y - mm) * inv;
+          v[u].z = __expf(v[u].z - mm) * inv; v[u].w = __expf(v[u].w - mm) * inv;
+          *reinterpret_cast<float4*>(dst + j + u * 128) = v[u];
+        }
+      }
+      for (; j < full; j += 128) {
         float4 v = *reinterpret_cast<float4*>(dst + j);
         v.x = __expf(v.x - mm) * inv; v.y = __expf(v.y - mm) * inv; v.z = __expf(v.z - mm) * inv; v.w = __expf(v.w - mm) * inv;
         *reinterpret_cast<float4*>(dst + j) = v;

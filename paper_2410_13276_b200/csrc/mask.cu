@@ -194,7 +194,7 @@ scan_kernel(int64_t rows, int32_t* __restrict__ row_ptr, int first, int64_t col_
 __global__ void __launch_bounds__(kMaskWarps * 32)
 fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask_params p, const int32_t* __restrict__ row_ptr,
             int32_t* __restrict__ col_idx, int64_t col_capacity, int stage_cap) {
-  extern __shared__ uint32_t key_smem[];
+  extern __shared__ __align__(16) uint32_t key_smem[];
   uint32_t* hist_smem = key_smem + (size_t)kMaskWarps * stage_cap;   // 256 bins per warp
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t r = band.row_lo + (int64_t)blockIdx.x * kMaskWarps + warp;
@@ -253,28 +253,33 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   const bool staged = n <= stage_cap;
   int c = 0;
   uint32_t k_and = 0xffffffffu, k_or = 0u;     // over the candidates' keys: the bits all of them share are k_and | ~k_or
-  auto take_key = [&](int j, float sc) {
+  auto make_key = [&](int j, float sc) -> uint32_t {
     const uint32_t kk = is_forced(j, ri.i, p.flags) ? 0u : score_key(sc);
-    if (staged) keys[j] = kk;
     c += kk != 0u;
     if (kk != 0u) { k_and &= kk; k_or |= kk; }
+    return kk;
   };
-  // four scores per lane and load where the row is 16-byte aligned (the loop is bound by the latency of its loads)
-  int head = 0;
-  if ((reinterpret_cast<uintptr_t>(ri.s) & 15) == 0) {
-    head = n & ~3;
-    for (int j = lane * 4; j < head; j += 128) {
-      const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
-      take_key(j, v.x); take_key(j + 1, v.y); take_key(j + 2, v.z); take_key(j + 3, v.w);
-    }
+  // four scores per lane and load where the row is 16-byte aligned (the loop is bound by the latency of its loads);
+  // the staged row is padded with zero keys (never candidates) to a multiple of 128
+  const bool vec = (reinterpret_cast<uintptr_t>(ri.s) & 15) == 0;
+  const int head = vec ? (n & ~3) : 0;
+  for (int j = lane * 4; j < head; j += 128) {
+    const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
+    const uint4 kq = make_uint4(make_key(j, v.x), make_key(j + 1, v.y), make_key(j + 2, v.z), make_key(j + 3, v.w));
+    if (staged) *reinterpret_cast<uint4*>(keys + j) = kq;
   }
-  for (int j = head + lane; j < n; j += 32) take_key(j, ri.s[j]);
+  for (int j = head + lane; j < n; j += 32) {
+    const uint32_t kk = make_key(j, ri.s[j]);
+    if (staged) keys[j] = kk;
+  }
+  const int n_pad = (n + 127) & ~127;
+  if (staged) for (int j = n + lane; j < n_pad; j += 32) keys[j] = 0u;
   const int ncand = warp_sum(c);
   k_and = __reduce_and_sync(0xffffffffu, k_and);
   k_or = __reduce_or_sync(0xffffffffu, k_or);
   __syncwarp();
   auto key_at = [&](int j) -> uint32_t {
-    return staged ? keys[j] : (is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]));
+    return is_forced(j, ri.i, p.flags) ? 0u : score_key(ri.s[j]);
   };
 
   uint32_t T = 0u;      // key of the last kept candidate; kept: key > T, plus the first need_eq with key == T
@@ -284,28 +289,47 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   } else if (take == 0) {
     T = 0xffffffffu; need_eq = 0;   // nothing beyond the forced blocks
   } else {
-    // Radix select, 8 bits per pass from the top (rows too long to stage re-read their scores in every pass): histogram the current digit of the keys that match the prefix found
-    // so far (warp-private shared-memory bins), walk the bins from the largest digit down until `remaining` is covered.
+    // Radix select, up to 8 bits per pass from the top (rows too long to stage re-read their scores in every pass):
+    // histogram the current digit of the keys that match the prefix found so far (warp-private shared-memory bins), walk
+    // the bins from the largest digit down until `remaining` is covered.
     uint32_t* hist = hist_smem + warp * 256;
-    // The scores of a row are often close together; the leading bits all candidate keys share need no pass: the passes
-    // start at the first 8-bit digit in which two keys differ.
+    // The scores of a row are close together (probabilities of one softmax): the leading bits all candidate keys share
+    // need no pass, and the first digit starts at the highest bit in which two keys differ, so that it spreads the keys
+    // over all 256 bins (a byte-aligned first digit put a whole row into two or three bins: 32 lanes adding to one
+    // shared-memory word).
     const uint32_t differ = k_and ^ k_or;                                 // bit set: not all keys agree there
-    const int top_shift = differ == 0u ? 0 : ((31 - __clz(differ)) >> 3) << 3;   // shift of the highest differing digit
-    uint32_t prefix_mask = top_shift >= 24 ? 0u : ~((1u << (top_shift + 8)) - 1u);
-    uint32_t prefix = k_or & prefix_mask;                                 // the shared leading digits
+    int hi_bit = differ == 0u ? 0 : 31 - __clz(differ);                   // highest differing bit
+    uint32_t prefix_mask = hi_bit >= 31 ? 0u : ~((2u << hi_bit) - 1u);    // the shared leading bits
+    uint32_t prefix = k_or & prefix_mask;
     int remaining = take;           // rank (1-based, from the top) still to locate inside the current prefix class
-    for (int shift = top_shift; shift >= 0; shift -= 8) {
+    for (int top = hi_bit; top >= 0; top -= 8) {                          // this pass: bits top .. max(top - 7, 0)
+      const int shift = max(top - 7, 0);
+      const uint32_t dmask = (2u << (top - shift)) - 1u;
       for (int b = lane; b < 256; b += 32) hist[b] = 0u;
       __syncwarp();
-      for (int j = lane; j < n; j += 32) {
-        const uint32_t kk = key_at(j);
-        if (kk != 0u && (kk & prefix_mask) == prefix) atomicAdd(&hist[(kk >> shift) & 255u], 1u);
+      if (staged) {
+        for (int j = lane * 4; j < n_pad; j += 128) {
+          const uint4 kq = *reinterpret_cast<const uint4*>(keys + j);
+          if (kq.x != 0u && (kq.x & prefix_mask) == prefix) atomicAdd(&hist[(kq.x >> shift) & dmask], 1u);
+          if (kq.y != 0u && (kq.y & prefix_mask) == prefix) atomicAdd(&hist[(kq.y >> shift) & dmask], 1u);
+          if (kq.z != 0u && (kq.z & prefix_mask) == prefix) atomicAdd(&hist[(kq.z >> shift) & dmask], 1u);
+          if (kq.w != 0u && (kq.w & prefix_mask) == prefix) atomicAdd(&hist[(kq.w >> shift) & dmask], 1u);
+        }
+      } else {
+        for (int j = lane; j < n; j += 32) {
+          const uint32_t kk = key_at(j);
+          if (kk != 0u && (kk & prefix_mask) == prefix) atomicAdd(&hist[(kk >> shift) & dmask], 1u);
+        }
       }
       __syncwarp();
       // lane l owns digits 8l .. 8l+7; suffix sums over lanes give the number of keys with a larger digit
       uint32_t c[8], lane_total = 0u;
+      {
+        const uint4 h0 = *reinterpret_cast<const uint4*>(hist + lane * 8), h1 = *reinterpret_cast<const uint4*>(hist + lane * 8 + 4);
+        c[0] = h0.x; c[1] = h0.y; c[2] = h0.z; c[3] = h0.w; c[4] = h1.x; c[5] = h1.y; c[6] = h1.z; c[7] = h1.w;
+      }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) { c[e] = hist[lane * 8 + e]; lane_total += c[e]; }
+      for (int e = 0; e < 8; ++e) lane_total += c[e];
       uint32_t above = lane_total;                       // inclusive suffix sum over lanes >= this lane
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -329,13 +353,54 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
       digit = __shfl_sync(0xffffffffu, digit, src);
       remaining = __shfl_sync(0xffffffffu, new_remaining, src);
       prefix |= digit << shift;
-      prefix_mask |= 255u << shift;
+      prefix_mask |= dmask << shift;
       __syncwarp();
     }
     T = prefix;                      // the take-th largest key; `remaining` of the keys equal to it are kept
     need_eq = remaining;
   }
   int written = 0, eq_seen = 0;
+  if (staged) {
+    // 128 columns at a time, four consecutive ones per lane: a lane's kept columns follow those of the lanes below it
+    for (int base = 0; base < n_pad; base += 128) {
+      const int j = base + 4 * lane;
+      const uint4 kq = *reinterpret_cast<const uint4*>(keys + j);
+      const uint32_t kk[4] = {kq.x, kq.y, kq.z, kq.w};
+      bool eq[4], keep[4];
+      int my_eq = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { eq[u] = kk[u] != 0u && kk[u] == T; my_eq += (int)eq[u]; }
+      int eq_incl = my_eq;
+      if (__any_sync(0xffffffffu, my_eq != 0)) {          // ties at the selection key are rare
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int u = __shfl_up_sync(0xffffffffu, eq_incl, o);
+          if (lane >= o) eq_incl += u;
+        }
+      }
+      int eq_rank = eq_seen + eq_incl - my_eq;            // ties before this lane's first column
+      int mine = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool forced = j + u < n && is_forced(j + u, ri.i, p.flags);
+        keep[u] = forced || (kk[u] != 0u && kk[u] > T) || (eq[u] && eq_rank < need_eq);
+        eq_rank += (int)eq[u];
+        mine += (int)keep[u];
+      }
+      int incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += u;
+      }
+      int at = written + incl - mine;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) if (keep[u]) out[at++] = j + u;
+      written += __shfl_sync(0xffffffffu, incl, 31);
+      eq_seen += __shfl_sync(0xffffffffu, eq_incl, 31);
+    }
+    return;
+  }
   for (int base = 0; base < n; base += 32) {
     const int j = base + lane;
     const uint32_t kk = j < n ? key_at(j) : 0u;
@@ -358,7 +423,7 @@ int launch_mask_band(seer_ctx* ctx, const SeqMeta& m, const float* scores, int64
   const unsigned grid = (unsigned)((row_hi - row_lo + kMaskWarps - 1) / kMaskWarps);
   count_kernel<<<grid, kMaskWarps * 32, 0, stream>>>(m, band, scores, p, row_ptr);
   scan_kernel<<<1, 1024, 0, stream>>>(row_hi - row_lo, row_ptr + row_lo, first ? 1 : 0, col_capacity, nnz_out, ctx->d_status);
-  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? m.max_nb : 0;   // long rows re-read their scores instead
+  const int stage_cap = m.max_nb <= kMaskSmemRowMax ? (m.max_nb + 127) & ~127 : 0;   // long rows re-read their scores instead
   const size_t smem = (size_t)kMaskWarps * (stage_cap + 256) * sizeof(uint32_t);
   fill_kernel<<<grid, kMaskWarps * 32, smem, stream>>>(m, band, scores, p, row_ptr, col_idx, col_capacity, stage_cap);
   cudaError_t e = cudaGetLastError();

@@ -15,10 +15,11 @@
  *    work has finished, and only if all 8 are still in flight does it wait on the host for the oldest one.
  *    The library allocates device memory only in seer_create; per-call scratch comes from the caller's
  *    workspace `ws` (>= seer_workspace_bytes(shape), 256-byte aligned).
- *  - The tcgen05 attention kernel takes all 512 tensor-memory columns and 215 KB of shared memory of an SM, so
- *    one CTA is resident per SM and its tensor-memory allocation cannot wait on another CTA of this library.  A
- *    kernel of ANOTHER library that holds tensor memory on the same device at the same time (another stream or
- *    process) can make that allocation wait; it is the one wait in the kernel the library cannot bound.
+ *  - The tcgen05 attention kernel takes all 512 tensor-memory columns and 219 KB of shared memory of an SM, the
+ *    gate's score kernel 256 columns and 226 KB: one CTA of either is resident per SM (the two cannot share an SM
+ *    either), so a tensor-memory allocation never waits on another CTA of this library.  A kernel of ANOTHER
+ *    library that holds tensor memory on the same device at the same time (another stream or process) can make
+ *    that allocation wait; it is the one wait in these kernels the library cannot bound.
  *  - Nothing throws across the ABI.  Host-detectable errors are returned at once and enqueue nothing.
  *    Errors only the device can see (list capacity exceeded, a list entry out of range, a bounded wait
  *    that ran out) are recorded in a status word owned by the context; the offending work is skipped and

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libseer.so")
-SOURCES = ["seer_ctx.cu", "gate.cu", "mask.cu", "attn_mma.cu", "attn_tc.cu"]
+SOURCES = ["seer_ctx.cu", "gate.cu", "gate_scores.cu", "mask.cu", "attn_mma.cu", "attn_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -194,7 +194,7 @@ def _structured_layer(config, twin, S, hq, hkv):
     return cu, f32_to_bf16_bits(q), f32_to_bf16_bits(k), f32_to_bf16_bits(v), wq, wk
 
 
-# name -> (config id, twin?)   "cN" = full size of BASELINE config N, "cNs" = its reduced twin (~4096 tokens)
+# name -> (config id, twin?)   "cN" = full size of benchmark configuration N, "cNs" = its reduced twin (~4096 tokens)
 WORKLOADS = ("c1", "c2", "c3", "c4", "c5", "c2s", "c3s", "c4s", "c5s")
 
 C3_RATIOS = ((1, 2), (1, 4), (1, 10), (1, 20))

@@ -36,11 +36,12 @@ __device__ __forceinline__ RowInfo decode_row(const SeqMeta& m, const RowBand& b
   ri.skip = false;
   ri.nb = 0;
   if (!ri.valid) { ri.s = nullptr; ri.i = 0; return ri; }
-  const int b = find_sequence(m.blk_off, m.batch, (int)(r / m.num_q_heads));
+  // (the host refuses shapes with 2^31 rows or more: 32-bit divisions)
+  const int b = find_sequence(m.blk_off, m.batch, (int)((uint32_t)r / (uint32_t)m.num_q_heads));
   const int nb = m.blk_off[b + 1] - m.blk_off[b];
-  const int64_t local = r - (int64_t)m.num_q_heads * m.blk_off[b];
-  const int h = (int)(local / nb);
-  ri.i = (int)(local - (int64_t)h * nb);
+  const uint32_t local = (uint32_t)r - (uint32_t)m.num_q_heads * (uint32_t)m.blk_off[b];
+  const int h = (int)(local / (uint32_t)nb);
+  ri.i = (int)(local - (uint32_t)h * (uint32_t)nb);
   ri.s = scores + (m.score_off[b] + ((int64_t)h * nb + ri.i) * nb - band.score_base);
   ri.skip = m.chunked && ri.i < m.qoff[b];
   ri.nb = nb;
@@ -339,12 +340,12 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
       above -= lane_total;                               // keys in lanes with larger digits
       // the digit holding rank `remaining` lies in the lane where above < remaining <= above + lane_total
       const bool mine = (int)above < remaining && remaining <= (int)(above + lane_total);
-      uint32_t digit = 0u; int new_remaining = 0;
+      uint32_t digit = 0u, sel_cnt = 0u; int new_remaining = 0;
       if (mine) {
         uint32_t acc = above;
 #pragma unroll
         for (int e = 7; e >= 0; --e) {
-          if ((int)acc < remaining && remaining <= (int)(acc + c[e])) { digit = (uint32_t)(lane * 8 + e); new_remaining = remaining - (int)acc; }
+          if ((int)acc < remaining && remaining <= (int)(acc + c[e])) { digit = (uint32_t)(lane * 8 + e); new_remaining = remaining - (int)acc; sel_cnt = c[e]; }
           acc += c[e];
         }
       }
@@ -352,9 +353,40 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
       const int src = __ffs(owner) - 1;
       digit = __shfl_sync(0xffffffffu, digit, src);
       remaining = __shfl_sync(0xffffffffu, new_remaining, src);
+      const uint32_t class_cnt = __shfl_sync(0xffffffffu, sel_cnt, src);   // keys that share the prefix found so far
       prefix |= digit << shift;
       prefix_mask |= dmask << shift;
       __syncwarp();
+      // A class of at most 32 keys (the usual case after one pass: a row of <= 2048 keys over 256 bins) is finished in
+      // registers: one sweep gathers its keys, every lane ranks one of them against the others.
+      if (staged && shift > 0 && class_cnt <= 32u) {
+        int found = 0;
+        for (int j = lane * 4; j < n_pad; j += 128) {
+          const uint4 kq = *reinterpret_cast<const uint4*>(keys + j);
+          const uint32_t kk[4] = {kq.x, kq.y, kq.z, kq.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const bool mt = kk[u] != 0u && (kk[u] & prefix_mask) == prefix;
+            const uint32_t bal = __ballot_sync(0xffffffffu, mt);
+            if (mt) hist[found + __popc(bal & lt_mask)] = kk[u];
+            found += __popc(bal);
+          }
+        }
+        __syncwarp();
+        const uint32_t x = lane < (int)class_cnt ? hist[lane] : 0u;
+        int G = 0, E = 0;                              // keys of the class larger than / equal to this lane's
+#pragma unroll
+        for (int l = 0; l < 32; ++l) {
+          const uint32_t y = __shfl_sync(0xffffffffu, x, l);
+          G += y > x; E += y == x;
+        }
+        const bool is_t = x != 0u && G < remaining && remaining <= G + E;
+        const int ts = __ffs(__ballot_sync(0xffffffffu, is_t)) - 1;
+        prefix = __shfl_sync(0xffffffffu, x, ts);
+        remaining -= __shfl_sync(0xffffffffu, G, ts);
+        __syncwarp();
+        break;
+      }
     }
     T = prefix;                      // the take-th largest key; `remaining` of the keys equal to it are kept
     need_eq = remaining;

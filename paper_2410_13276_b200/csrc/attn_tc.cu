@@ -180,13 +180,17 @@ __device__ __forceinline__ uint32_t tile_pass(uint32_t s_addr, float sl2, bool r
 }
 
 // ------------------------------------------------------------------------------------------------ kernel
-template <bool kTrace, bool kChunk>
+// kBlockMax: the same pipeline without V: instead of softmax(S) V the kernel writes, for every list entry, the largest
+// probability exp(scale * s - lse) of its 64 x 64 tile (Sec. 3.2, Eq. 2 on the listed blocks), `lse` being an input.
+// The log-sum-exp of a query column is subtracted by the tensor core exactly like a softmax reference (as three bf16
+// terms, so exactly to fp32), a thread takes the maximum of its key row, a block's maximum is one redux per warp.
+template <bool kTrace, bool kChunk, bool kBlockMax = false>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, SeqMeta m,
                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                 uint16_t* __restrict__ o, float* __restrict__ lse, int* __restrict__ status,
-                unsigned long long* __restrict__ trace) {
+                unsigned long long* __restrict__ trace, float* __restrict__ block_max = nullptr) {
   extern __shared__ unsigned char smem_raw[];
   Shared sh;
   sh.base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -242,7 +246,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ========================================================================================== producers (TMA)
     // warps 0 / 2: Q and K of stream 0 / 1; warps 12 / 13: V of stream 0 / 1
     if (warp == 0 || warp == 2 || warp == 12 || warp == 13) {
-      if (lane == 0) {
+      if (lane == 0 && !(kBlockMax && warp >= 12)) {       // (no V in the block-maximum pass)
         const bool is_v = warp >= 12;
         const int s = is_v ? warp - 12 : warp >> 1, bb = s * kBarsPerStream;
         const uint32_t sbase = sh.base + (uint32_t)s * kStreamBytes;
@@ -340,6 +344,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (it.ntiles > 1 && !issue_s(it.ntiles == 2, false)) break;
           for (int t = 0; t < it.ntiles; ++t, ++cp) {
             tr.sample(cp); tr.ev(13, cp);
+            if constexpr (kBlockMax) {
+              // the group has taken the maxima of S^T buffer cp & 1: the buffer is free for the tile after next
+              if (!mbar_wait<kIssuerSleepNs>(sh, bb + P_FULL, cp & 1u, status)) { ok = false; break; }
+              if (t + 2 < it.ntiles && !issue_s(t + 3 == it.ntiles, true)) { ok = false; break; }
+              continue;
+            }
             if (!mbar_wait(sh, bb + V_FULL, cp & 1u, status)) { ok = false; break; }
             tr.ev(14, cp);
             // P^T of tile t is complete; the group has also finished with S^T buffer cp & 1 (and, at t = 0, with the
@@ -401,6 +411,83 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     unsigned seg_n = 0, nreb = 0;
 #define SEG(k) do { if constexpr (kTrace) { const long long now_ = clock64(); seg[k] += now_ - seg_last; seg_last = now_; } } while (0)
 
+    if constexpr (kBlockMax) {
+      int* wmax = reinterpret_cast<int*>(lsum);             // [2 tile parities][4 warps]: maxima as order-preserving integers
+      const float inv_scale = 1.0f / m.softmax_scale;
+      for (int64_t w = 2 * (int64_t)blockIdx.x + s; ok && w < m.rows; w += w_step) {
+        const Item it = decode_item<kChunk>(m, row_ptr, w);
+        if (it.ntiles == 0) continue;
+        const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock + (kChunk ? it.dq : 0);
+        // -R[c], R[c] = lse[c] / scale (the log-sum-exp in units of raw scores), as three truncated bf16 terms in
+        // columns 0..2 of both reference rows (the first two tiles are corrected in place, the later ones get it from the
+        // ninth K-step of their MMA)
+        if (gt < 64) {
+          float L = gt < it.q_valid ? lse[(int64_t)it.h * (kChunk ? m.total_q_tokens : m.total_tokens) + tok0 + gt] : 0.f;
+          if (!(fabsf(L) < 3.0e38f)) L = 0.f;               // a query without a key has no probabilities to report
+          const float d = -L * inv_scale;
+          const uint32_t hi = __float_as_uint(d) & 0xffff0000u;
+          const float r1 = d - __uint_as_float(hi);
+          const uint32_t mid = __float_as_uint(r1) & 0xffff0000u;
+          const uint32_t lo = __float_as_uint(r1 - __uint_as_float(mid)) & 0xffff0000u;
+          *reinterpret_cast<uint2*>(qfix + gt * 8) = make_uint2((hi >> 16) | mid, lo >> 16);
+          *reinterpret_cast<uint2*>(qext + gt * 8) = make_uint2((hi >> 16) | mid, lo >> 16);
+          fence_async_smem();
+        }
+        int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
+        for (int t = 0; t < it.ntiles; ++t, ++cnt) {
+          const uint32_t sbuf = cnt & 1u;
+          bool fail = !mbar_wait(sh, bb + S_FULL + (int)sbuf, (cnt >> 1) & 1u, status);
+          if (t == 0) {
+            if (!fail && it.ntiles > 1) fail = !mbar_wait(sh, bb + S_FULL + (int)(sbuf ^ 1u), ((cnt + 1) >> 1) & 1u, status);
+            tc_fence_after();
+            if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
+            if (gt == 0) {
+              tc_mma(tmem + col_s(s, sbuf), ones_d, qfix_d, kIdescS, 1u);
+              if (it.ntiles > 1) tc_mma(tmem + col_s(s, sbuf ^ 1u), ones_d, qfix_d, kIdescS, 1u);
+              tc_commit(sh.bar(bb + FIXED));
+            }
+            if (named_bar_or(bar_vote, kGroupThreads, !mbar_wait(sh, bb + FIXED, nfix & 1u, status))) { ok = false; break; }
+            ++nfix;
+          }
+          tc_fence_after();
+          const int na = list_block(it, col_idx, 2 * t + 2), nb2 = list_block(it, col_idx, 2 * t + 3);
+          const int my_j = r < 64 ? ja : jb;
+          const bool diag = my_j == it.i;
+          const uint32_t s_addr = tmem + lane_addr + col_s(s, sbuf);
+          float mx = -CUDART_INF_F;                         // largest s - R over the causal queries of this key row
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t sv[32];
+            tc_ld32(s_addr + ch * 32, sv);
+            tc_wait_ld32(sv);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int c = ch * 32 + e;
+              if (c < it.q_valid && !(diag && key_local > c)) mx = fmaxf(mx, __uint_as_float(sv[e]));
+            }
+          }
+          if (my_j < 0 || fail || !(mx == mx)) mx = -CUDART_INF_F;
+          int key = __float_as_int(mx);
+          key ^= (key >> 31) & 0x7fffffff;                  // order-preserving map float -> int
+          key = __reduce_max_sync(0xffffffffu, key);
+          if (lane == 0) wmax[sbuf * 4 + gw] = key;
+          tc_fence_before();
+          if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
+          if (gt == 0) {
+            mbar_arrive(sh.bar(bb + P_FULL));               // the S^T buffer may be overwritten
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              if (2 * t + half < it.nlist) {
+                int kx = max(wmax[sbuf * 4 + 2 * half], wmax[sbuf * 4 + 2 * half + 1]);
+                kx ^= (kx >> 31) & 0x7fffffff;
+                block_max[it.l0 + 2 * t + half] = exp2f(__int_as_float(kx) * sl2);   // 2^(-inf) = 0: no causal pair, or a rejected entry
+              }
+            }
+          }
+          ja = na; jb = nb2;
+        }
+      }
+    } else
     for (int64_t w = 2 * (int64_t)blockIdx.x + s; w < m.rows; w += w_step) {
       tr.sample(0);
       const Item it = decode_item<kChunk>(m, row_ptr, w);
@@ -743,6 +830,10 @@ seer_status init_attn_tc(seer_ctx* ctx) {
     e = cudaFuncSetAttribute(tc::attn_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(tc::attn_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::attn_tc_kernel<false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes);
   return e == cudaSuccess ? SEER_OK : SEER_ERR_CUDA;
 }
 
@@ -763,6 +854,24 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
     tc::attn_tc_kernel<true, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
   else
     tc::attn_tc_kernel<false, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
+  cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? 1 : -(int)e;
+}
+
+// Max-pooled attention map on the listed blocks (Sec. 3.2, Eq. 2): the attention pipeline without V.
+int launch_block_max_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const int32_t* row_ptr,
+                        const int32_t* col_idx, const float* lse, float* out, cudaStream_t stream) {
+  if (m.rows == 0) return 0;
+  if ((((uintptr_t)q | (uintptr_t)k) & 15) != 0) return -(int)cudaErrorMisalignedAddress;
+  CUtensorMap mq, mk;
+  if (!tc::make_map(ctx, &mq, q, m.total_q_tokens, m.num_q_heads) || !tc::make_map(ctx, &mk, k, m.total_tokens, m.num_kv_heads))
+    return -(int)cudaErrorInvalidValue;
+  const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, (m.rows + 1) / 2);
+  float* lse_in = const_cast<float*>(lse);   // read only in this mode
+  if (m.chunked)
+    tc::attn_tc_kernel<false, true, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mk, m, row_ptr, col_idx, nullptr, lse_in, ctx->d_status, nullptr, out);
+  else
+    tc::attn_tc_kernel<false, false, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mk, m, row_ptr, col_idx, nullptr, lse_in, ctx->d_status, nullptr, out);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;
 }

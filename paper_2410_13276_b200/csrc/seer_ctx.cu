@@ -393,7 +393,10 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
   SeqMeta m; int slot;
   st = prepare(ctx, shape, stream, &m, &slot);
   if (st != SEER_OK) return st;
-  int n = launch_block_max(ctx, m, q, k, row_ptr, col_idx, lse, block_max, stream);
+  // the same choice of kernel as seer_sparse_attn: the tcgen05 pipeline without V, or the mma.sync kernel
+  const bool legacy = ctx->attn_impl == 1 || (ctx->attn_impl == 2 && t.causal_blocks <= 8 * t.rows);
+  int n = legacy ? launch_block_max(ctx, m, q, k, row_ptr, col_idx, lse, block_max, stream)
+                 : launch_block_max_tc(ctx, m, q, k, row_ptr, col_idx, lse, block_max, stream);
   finish_call(ctx, slot, stream);
   if (n < 0) return SEER_ERR_CUDA;
   ctx->launches += n;

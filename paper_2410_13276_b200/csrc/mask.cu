@@ -254,20 +254,41 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   const bool staged = n <= stage_cap;
   int c = 0;
   uint32_t k_and = 0xffffffffu, k_or = 0u;     // over the candidates' keys: the bits all of them share are k_and | ~k_or
-  auto make_key = [&](int j, float sc) -> uint32_t {
-    const uint32_t kk = is_forced(j, ri.i, p.flags) ? 0u : score_key(sc);
+  // The same key as score_key in fewer instructions (this loop is bound by instruction issue); forced blocks are not
+  // told apart here: they are taken out again below.  (Their keys stay in k_and / k_or: the bits a superset shares are
+  // shared by the candidates too.)
+  auto lean_key = [](float sc) -> uint32_t {
+    const float z = sc + 0.0f;                                   // -0 -> +0
+    const uint32_t u = __float_as_uint(z);
+    const uint32_t kk = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+    return z != z ? 0u : kk;                                     // NaN: never a candidate
+  };
+  auto make_key = [&](int, float sc) -> uint32_t {
+    const uint32_t kk = lean_key(sc);
     c += kk != 0u;
-    if (kk != 0u) { k_and &= kk; k_or |= kk; }
+    k_or |= kk;
+    k_and &= kk != 0u ? kk : 0xffffffffu;
     return kk;
   };
   // four scores per lane and load where the row is 16-byte aligned (the loop is bound by the latency of its loads);
   // the staged row is padded with zero keys (never candidates) to a multiple of 128
   const bool vec = (reinterpret_cast<uintptr_t>(ri.s) & 15) == 0;
   const int head = vec ? (n & ~3) : 0;
-  for (int j = lane * 4; j < head; j += 128) {
-    const float4 v = *reinterpret_cast<const float4*>(ri.s + j);
-    const uint4 kq = make_uint4(make_key(j, v.x), make_key(j + 1, v.y), make_key(j + 2, v.z), make_key(j + 3, v.w));
-    if (staged) *reinterpret_cast<uint4*>(keys + j) = kq;
+  // (four loads in flight per lane: one load per step left the loop waiting a memory latency per 128 columns, 45 % of
+  // the kernel)
+  for (int j0 = lane * 4; j0 < head; j0 += 512) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      v[u] = j0 + u * 128 < head ? *reinterpret_cast<const float4*>(ri.s + j0 + u * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * 128;
+      if (j < head) {
+        const uint4 kq = make_uint4(make_key(j, v[u].x), make_key(j + 1, v[u].y), make_key(j + 2, v[u].z), make_key(j + 3, v[u].w));
+        if (staged) *reinterpret_cast<uint4*>(keys + j) = kq;
+      }
+    }
   }
   for (int j = head + lane; j < n; j += 32) {
     const uint32_t kk = make_key(j, ri.s[j]);
@@ -275,6 +296,15 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   }
   const int n_pad = (n + 127) & ~127;
   if (staged) for (int j = n + lane; j < n_pad; j += 32) keys[j] = 0u;
+  // forced blocks are not candidates: out of the count, and their staged keys blanked (a zero key is never kept by the
+  // selection; the list writer below puts the forced blocks in their places: block 0 first, block i last)
+  const bool sink_f = (p.flags & SEER_FORCE_SINK) != 0u;
+  const bool diag_f = (p.flags & SEER_FORCE_DIAG) != 0u && !(sink_f && ri.i == 0);
+  __syncwarp();
+  if (lane == 0) {                                  // (the staged key where there is one: a global load here costs a memory latency per row)
+    if (sink_f) { c -= (staged ? keys[0] : lean_key(ri.s[0])) != 0u; if (staged) keys[0] = 0u; }
+    if (diag_f) { c -= (staged ? keys[ri.i] : lean_key(ri.s[ri.i])) != 0u; if (staged) keys[ri.i] = 0u; }
+  }
   const int ncand = warp_sum(c);
   k_and = __reduce_and_sync(0xffffffffu, k_and);
   k_or = __reduce_or_sync(0xffffffffu, k_or);
@@ -393,6 +423,7 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
   }
   int written = 0, eq_seen = 0;
   if (staged) {
+    if (sink_f) { if (lane == 0) out[0] = 0; written = 1; }
     // 128 columns at a time, four consecutive ones per lane: a lane's kept columns follow those of the lanes below it
     for (int base = 0; base < n_pad; base += 128) {
       const int j = base + 4 * lane;
@@ -411,26 +442,21 @@ fill_kernel(SeqMeta m, RowBand band, const float* __restrict__ scores, seer_mask
         }
       }
       int eq_rank = eq_seen + eq_incl - my_eq;            // ties before this lane's first column
-      int mine = 0;
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const bool forced = j + u < n && is_forced(j + u, ri.i, p.flags);
-        keep[u] = forced || (kk[u] != 0u && kk[u] > T) || (eq[u] && eq_rank < need_eq);
+        keep[u] = (kk[u] != 0u && kk[u] > T) || (eq[u] && eq_rank < need_eq);
         eq_rank += (int)eq[u];
-        mine += (int)keep[u];
       }
-      int incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int u = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += u;
-      }
-      int at = written + incl - mine;
+      // kept columns of the lanes below this one: four independent ballots instead of a five-step scan
+      const uint32_t b0 = __ballot_sync(0xffffffffu, keep[0]), b1 = __ballot_sync(0xffffffffu, keep[1]);
+      const uint32_t b2 = __ballot_sync(0xffffffffu, keep[2]), b3 = __ballot_sync(0xffffffffu, keep[3]);
+      int at = written + __popc(b0 & lt_mask) + __popc(b1 & lt_mask) + __popc(b2 & lt_mask) + __popc(b3 & lt_mask);
 #pragma unroll
       for (int u = 0; u < 4; ++u) if (keep[u]) out[at++] = j + u;
-      written += __shfl_sync(0xffffffffu, incl, 31);
+      written += __popc(b0) + __popc(b1) + __popc(b2) + __popc(b3);
       eq_seen += __shfl_sync(0xffffffffu, eq_incl, 31);
     }
+    if (diag_f && lane == 0) out[written] = ri.i;
     return;
   }
   for (int base = 0; base < n; base += 32) {

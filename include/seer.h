@@ -171,7 +171,8 @@ seer_status seer_attn_block_max(seer_ctx* ctx, const seer_shape* shape, const vo
                                 const int32_t* row_ptr, const int32_t* col_idx, const float* lse, float* block_max,
                                 void* stream);
 
-/* Selects the attention kernel used by seer_sparse_attn: 0 = tcgen05 / TMEM / TMA kernel (default),
+/* Selects the attention kernel used by seer_sparse_attn (and, by the same rule, the kernel of seer_attn_block_max: the
+ * tcgen05 pipeline without V, or the mma.sync kernel): 0 = tcgen05 / TMEM / TMA kernel (default),
  * 1 = mma.sync kernel (on-device cross-check; also the faster one for very short lists), 2 = chosen per call from
  * the shape: the persistent tcgen05 kernel pays a few microseconds per (head, query block) row whatever its list
  * length, so batches whose rows have at most 8 causal blocks on average (many short sequences) go to the mma.sync

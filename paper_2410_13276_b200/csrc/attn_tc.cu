@@ -212,7 +212,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(sh.bar(b + V_EMPTY), 1);
       mbar_init(sh.bar(b + S_FULL), 1);
       mbar_init(sh.bar(b + S_FULL + 1), 1);
-      mbar_init(sh.bar(b + P_FULL), 1);                       // one arrival, after the softmax group has met
+      mbar_init(sh.bar(b + P_FULL), kBlockMax ? 4 : 1);       // one arrival, after the softmax group has met (block maxima: one per warp)
       mbar_init(sh.bar(b + PV_DONE), 1);
       mbar_init(sh.bar(b + FIXED), 1);
     }
@@ -413,6 +413,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
     if constexpr (kBlockMax) {
       int* wmax = reinterpret_cast<int*>(lsum);             // [2 tile parities][4 warps]: maxima as order-preserving integers
+      bool sticky_fail = false;
       const float inv_scale = 1.0f / m.softmax_scale;
       for (int64_t w = 2 * (int64_t)blockIdx.x + s; ok && w < m.rows; w += w_step) {
         const Item it = decode_item<kChunk>(m, row_ptr, w);
@@ -436,8 +437,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         int ja = list_block(it, col_idx, 0), jb = list_block(it, col_idx, 1);
         for (int t = 0; t < it.ntiles; ++t, ++cnt) {
           const uint32_t sbuf = cnt & 1u;
+          // (a lost wait does not leave the loop here: the warps of a group meet only at an item's first tile, and all
+          // of them have to get there; the failure is voted on at that point)
           bool fail = !mbar_wait(sh, bb + S_FULL + (int)sbuf, (cnt >> 1) & 1u, status);
           if (t == 0) {
+            fail = fail || sticky_fail;
             if (!fail && it.ntiles > 1) fail = !mbar_wait(sh, bb + S_FULL + (int)(sbuf ^ 1u), ((cnt + 1) >> 1) & 1u, status);
             tc_fence_after();
             if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
@@ -471,19 +475,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           key ^= (key >> 31) & 0x7fffffff;                  // order-preserving map float -> int
           key = __reduce_max_sync(0xffffffffu, key);
           if (lane == 0) wmax[sbuf * 4 + gw] = key;
+          // this warp is done with the S^T buffer (four arrivals free it); the two warps of a key block meet to
+          // combine their maxima, the group as a whole does not
           tc_fence_before();
-          if (named_bar_or(bar_vote, kGroupThreads, fail)) { ok = false; break; }
-          if (gt == 0) {
-            mbar_arrive(sh.bar(bb + P_FULL));               // the S^T buffer may be overwritten
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              if (2 * t + half < it.nlist) {
-                int kx = max(wmax[sbuf * 4 + 2 * half], wmax[sbuf * 4 + 2 * half + 1]);
-                kx ^= (kx >> 31) & 0x7fffffff;
-                block_max[it.l0 + 2 * t + half] = exp2f(__int_as_float(kx) * sl2);   // 2^(-inf) = 0: no causal pair, or a rejected entry
-              }
-            }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(sh.bar(bb + P_FULL));
+          const int half = gw >> 1;
+          named_bar_sync(5 + 2 * s + half, 64);
+          if ((gw & 1) == 0 && lane == 0 && 2 * t + half < it.nlist) {
+            int kx = max(wmax[sbuf * 4 + 2 * half], wmax[sbuf * 4 + 2 * half + 1]);
+            kx ^= (kx >> 31) & 0x7fffffff;
+            block_max[it.l0 + 2 * t + half] = exp2f(__int_as_float(kx) * sl2);   // 2^(-inf) = 0: no causal pair, or a rejected entry
           }
+          sticky_fail |= fail;
           ja = na; jb = nb2;
         }
       }

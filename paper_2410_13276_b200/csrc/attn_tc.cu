@@ -46,8 +46,9 @@ constexpr int kGroupThreads = 128;
 // a helper thread that polls a barrier shares its scheduler with two softmax warps: it sleeps between polls
 constexpr int kProducerSleepNs = 128, kIssuerSleepNs = 0;
 // of every eight column pairs of a pass this many take their exponentials on the FMA pipe, the others on the
-// special-function unit (measured optimum of the pass alone: 3)
-constexpr int kPolyPairsOf8 = 3;
+// special-function unit (the pass alone is fastest with 3; the kernel, where the pass shares its schedulers with the
+// other stream's, with 2: 19.9 ms against 20.4 with 3, 20.3 with 0 and 21.5 with 4 on the 128k TopK 1/10 workload)
+constexpr int kPolyPairsOf8 = 2;
 constexpr uint32_t kHalfQ = 64 * 128;            // bytes of one d-half of a 64-row tile (8 KB)
 constexpr uint32_t kHalfKV = 128 * 128;          // bytes of one d-half of a 128-row tile (16 KB)
 constexpr uint32_t kQBytes = 2 * kHalfQ;         // 16 KB

@@ -154,7 +154,11 @@ seer_status seer_block_mask(seer_ctx* ctx, const seer_shape* shape, const float*
  *    blocks listed for its (sequence, head, query block) row that are not later than the query.  bf16 operands, fp32
  *    accumulation and softmax, probabilities rounded to bf16 before the P V product, o written as bf16.
  *    lse (optional, may be NULL): [num_q_heads, T] fp32, natural log of the softmax denominator of the scaled logits.
- *    A row with an empty list yields o = 0 and lse = -inf. */
+ *    A row with an empty list yields o = 0 and lse = -inf.
+ *    ws (optional): with a workspace of at least 256 bytes (256-byte aligned, as for the other calls) the first word
+ *    becomes the counter from which the tcgen05 kernel's persistent CTAs draw their (head, query block) work items,
+ *    so that a CTA that finishes early takes more of them; without one (NULL) the items are dealt statically.  The
+ *    results are identical bit for bit.  Calls that may run at the same time must not share the workspace. */
 seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k, const void* v,
                              const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, void* ws,
                              size_t ws_bytes, void* stream);

@@ -64,15 +64,16 @@ constexpr uint32_t kOffGrp = kOffQfix + 2 * 2048;                 // per-group s
 constexpr uint32_t kGrpRcur = 0, kGrpAlpha = 256, kGrpLsum = 1024;   // lsum: 4 x 64 floats
 constexpr uint32_t kGrpBytes = 2048;
 constexpr uint32_t kOffBar = kOffGrp + 2 * kGrpBytes;             // mbarriers
-constexpr int kBarsPerStream = 12;
+constexpr int kBarsPerStream = 16;
 constexpr uint32_t kNumBars = 2 * kBarsPerStream;
-constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag
+constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag, the two streams' rings of work items (at +16, +32)
 constexpr uint32_t kOffTrace = kOffMisc + 64;                     // diagnostics: 6 roles x 48 tags x (sum, count)
 constexpr uint32_t kSmemBytes = kOffTrace + 6 * 48 * 16 + 1024;   // + alignment slack
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2, K_EMPTY = 3, V_FULL = 4, V_EMPTY = 5, S_FULL = 6 /* + buf */, P_FULL = 8,
-           PV_DONE = 9, FIXED = 10 };
+           PV_DONE = 9, FIXED = 10, ITEM_FULL = 12 /* + slot, 4 slots */ };
+constexpr int kItemRing = 4;
 
 constexpr uint32_t kTmemCols = 512;
 // TMEM columns of a stream: two S^T accumulators, O^T
@@ -191,7 +192,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const __grid_constant__ CUtensorMap map_v, SeqMeta m,
                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                 uint16_t* __restrict__ o, float* __restrict__ lse, int* __restrict__ status,
-                unsigned long long* __restrict__ trace, float* __restrict__ block_max = nullptr) {
+                unsigned long long* __restrict__ trace, float* __restrict__ block_max = nullptr,
+                int* __restrict__ work_counter = nullptr) {
   extern __shared__ unsigned char smem_raw[];
   Shared sh;
   sh.base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -216,6 +218,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(sh.bar(b + P_FULL), kBlockMax ? 4 : 1);       // one arrival, after the softmax group has met (block maxima: one per warp)
       mbar_init(sh.bar(b + PV_DONE), 1);
       mbar_init(sh.bar(b + FIXED), 1);
+      for (int i = 0; i < kItemRing; ++i) mbar_init(sh.bar(b + ITEM_FULL + i), 1);
     }
     st_shared_u32(sh.abort_flag(), 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -241,6 +244,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // Every role of stream s walks the same items w = 2 * blockIdx.x + s, + 2 * gridDim.x, ... and the same tiles, so
   // their ordinals (items seen, tiles seen) agree without communication.
   const int64_t w_step = 2 * (int64_t)gridDim.x;
+  // Work items.  Without a counter a stream takes the items 2 * CTA + stream, + 2 * grid, ... (static deal).  With one
+  // (`work_counter`, zero at launch) the stream's Q / K producer draws the next item number from it when it starts an
+  // item and passes it to the stream's other roles through a ring of four shared-memory words, one mbarrier each: the
+  // roles of a stream are never more than three items apart (Q is single-buffered), so a slot is not rewritten before
+  // its last reader has left it.  A negative number ends the stream.  Results do not depend on which stream runs an item.
+  const bool dyn = !kBlockMax && work_counter != nullptr;
+  auto ring_addr = [&](int s, uint32_t n) -> uint32_t { return sh.base + kOffMisc + 16u + (uint32_t)s * 16u + (n & 3u) * 4u; };
+  // consumer side: the n-th item of stream s (false: no more items, or a lost wait)
+  auto next_item = [&](int s, uint32_t n, int64_t& w) -> bool {
+    if (!dyn) { w = 2 * (int64_t)blockIdx.x + s + (int64_t)n * w_step; return w < m.rows; }
+    if (!mbar_wait<kProducerSleepNs>(sh, s * kBarsPerStream + ITEM_FULL + (int)(n & 3u), (n >> 2) & 1u, status)) return false;
+    w = (int64_t)(int32_t)ld_shared_u32(ring_addr(s, n));
+    return w >= 0;
+  };
 
   if (warp < 4 || warp >= 12) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kHelperRegs));
@@ -257,7 +274,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t dst = sbase + (is_v ? kStV : kStK);
         uint32_t nitem = 0, cnt = 0;
         bool ok = true;
-        for (int64_t w = 2 * (int64_t)blockIdx.x + s; ok && w < m.rows; w += w_step) {
+        int drawn = (dyn && !is_v) ? atomicAdd(work_counter, 1) : 0;   // the Q / K producer draws the stream's items
+        for (uint32_t n = 0; ok; ++n) {
+          int64_t w;
+          if (dyn && !is_v) {
+            w = drawn;
+            const bool more = w < m.rows;
+            st_shared_u32(ring_addr(s, n), more ? (uint32_t)drawn : 0xffffffffu);
+            mbar_arrive(sh.bar(bb + ITEM_FULL + (int)(n & 3u)));
+            if (!more) break;
+            drawn = atomicAdd(work_counter, 1);                        // the next one is on its way while this one is copied
+          } else if (!next_item(s, n, w)) break;
           const Item it = decode_item<kChunk>(m, row_ptr, w);
           if (it.ntiles == 0) continue;
           if (!is_v) {
@@ -332,7 +359,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           ++cs;
           return true;
         };
-        for (int64_t w = 2 * (int64_t)blockIdx.x + s; ok && w < m.rows; w += w_step) {
+        for (uint32_t n = 0; ok; ++n) {
+          int64_t w;
+          if (!next_item(s, n, w)) break;
           const Item it = decode_item<kChunk>(m, row_ptr, w);
           if (it.ntiles == 0) continue;
           tr.sample(cs);
@@ -493,8 +522,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
       }
     } else
-    for (int64_t w = 2 * (int64_t)blockIdx.x + s; w < m.rows; w += w_step) {
+    for (uint32_t n = 0;; ++n) {
       tr.sample(0);
+      int64_t w;
+      const bool more = next_item(s, n, w);
+      // (with a counter the answer comes from a wait, which can be lost: the group leaves together or not at all)
+      if (dyn ? named_bar_or(bar_vote, kGroupThreads, !more) : !more) break;
       const Item it = decode_item<kChunk>(m, row_ptr, w);
       const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock + (kChunk ? it.dq : 0);   // first row of the item in q / o / lse
       if (it.ntiles == 0) {                                 // no visible key: o = 0, lse = -inf
@@ -843,8 +876,11 @@ seer_status init_attn_tc(seer_ctx* ctx) {
 }
 
 int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
-                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream) {
+                    const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int* work_counter,
+                    cudaStream_t stream) {
   if (m.rows == 0) return 0;
+  // the counter the streams draw their work items from (in the caller's workspace; without one the deal is static)
+  if (work_counter != nullptr && cudaMemsetAsync(work_counter, 0, sizeof(int), stream) != cudaSuccess) return -(int)cudaErrorInvalidValue;
   // the input pointers must be 16-byte aligned for TMA
   if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o) & 15) != 0) return -(int)cudaErrorMisalignedAddress;
   CUtensorMap mq, mk, mv;
@@ -854,11 +890,11 @@ int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k
   const unsigned grid = (unsigned)min((int64_t)ctx->num_sms, (m.rows + 1) / 2);
   unsigned long long* tb = (unsigned long long*)ctx->trace;
   if (m.chunked)               // chunked prefill (never instrumented)
-    tc::attn_tc_kernel<false, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
+    tc::attn_tc_kernel<false, true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb, nullptr, work_counter);
   else if (tb != nullptr)      // the instrumented instantiation
-    tc::attn_tc_kernel<true, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
+    tc::attn_tc_kernel<true, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb, nullptr, work_counter);
   else
-    tc::attn_tc_kernel<false, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb);
+    tc::attn_tc_kernel<false, false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(mq, mk, mv, m, row_ptr, col_idx, (uint16_t*)o, lse, ctx->d_status, tb, nullptr, work_counter);
   cudaError_t e = cudaGetLastError();
   return e == cudaSuccess ? 1 : -(int)e;
 }

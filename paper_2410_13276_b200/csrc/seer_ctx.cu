@@ -356,13 +356,15 @@ seer_status seer_block_mask(seer_ctx* ctx, const seer_shape* shape, const float*
 seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void* q, const void* k, const void* v,
                              const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, void* ws,
                              size_t ws_bytes, void* stream_) {
-  (void)ws; (void)ws_bytes;
   cudaStream_t stream = (cudaStream_t)stream_;
   if (!ctx || !shape) return SEER_ERR_INVALID_ARG;
   ShapeTotals t;
   seer_status st = shape_totals(shape, &t);
   if (st != SEER_OK) return st;
   if (shape->block != kBlock) return SEER_ERR_UNSUPPORTED;   // 128-token lists go through seer_expand_block_lists first
+  // the first word of the workspace is the counter the tcgen05 kernel's streams draw their work items from; without
+  // a workspace the items are dealt statically
+  int* work_counter = ws_ok(ws, ws_bytes, 256) ? (int*)ws : nullptr;
   if (t.total_blocks == 0 || t.total_q_tokens == 0) return SEER_OK;   // no output row
   if (!q || !k || !v || !row_ptr || !col_idx || !o) return SEER_ERR_INVALID_ARG;
   SeqMeta m; int slot;
@@ -372,7 +374,7 @@ seer_status seer_sparse_attn(seer_ctx* ctx, const seer_shape* shape, const void*
   // per-row hand-over than the legacy kernel needs for the whole row.
   const bool legacy = ctx->attn_impl == 1 || (ctx->attn_impl == 2 && t.causal_blocks <= 8 * t.rows);
   int n = legacy ? launch_attn_mma(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream)
-                 : launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, stream);
+                 : launch_attn_tc(ctx, m, q, k, v, row_ptr, col_idx, o, lse, work_counter, stream);
   finish_call(ctx, slot, stream);
   if (n < 0) return SEER_ERR_CUDA;
   ctx->launches += n;
@@ -679,8 +681,8 @@ seer_status seer_prefill_host(seer_ctx* ctx, const seer_shape* shape, const void
                          (int32_t*)(d + a.col_idx), t.causal_blocks, (int64_t*)(d + a.nnz), nullptr, 0, stream);
     if (st != SEER_OK) return st;
     st = seer_sparse_attn(ctx, &slice, d + a.q[b], d + a.k[b], d + a.v[b], (const int32_t*)(d + a.row_ptr),
-                          (const int32_t*)(d + a.col_idx), d + a.o[b], lse_host ? (float*)(d + a.lse[b]) : nullptr, nullptr,
-                          0, stream);
+                          (const int32_t*)(d + a.col_idx), d + a.o[b], lse_host ? (float*)(d + a.lse[b]) : nullptr, d + a.ws,
+                          a.total - a.ws, stream);   // (the gate's workspace is free again: the attention's work counter)
     if (st != SEER_OK) return st;
     SEER_TRY(cudaEventRecord(ctx->ev_comp[b], stream));
     // ---- device -> host

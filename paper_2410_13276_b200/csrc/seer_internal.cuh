@@ -123,7 +123,8 @@ int launch_block_max(seer_ctx* ctx, const SeqMeta& m, const void* q, const void*
 int launch_block_max_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const int32_t* row_ptr,
                         const int32_t* col_idx, const float* lse, float* out, cudaStream_t stream);
 int launch_attn_tc(seer_ctx* ctx, const SeqMeta& m, const void* q, const void* k, const void* v,
-                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, cudaStream_t stream);
+                   const int32_t* row_ptr, const int32_t* col_idx, void* o, float* lse, int* work_counter,
+                   cudaStream_t stream);
 seer_status init_gate(seer_ctx* ctx);
 seer_status init_mask(seer_ctx* ctx);
 seer_status init_attn_mma(seer_ctx* ctx);

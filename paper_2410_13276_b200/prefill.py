@@ -126,9 +126,13 @@ class Prefill:
         B.seer_expand_block_lists(self.ctx, self.shape, self.row_ptr, self.col_idx, self.row_ptr64, self.col_idx64, None,
                                   self.nnz64, stream)
 
-    def attn(self, stream=None):
+    def attn(self, stream=None, dynamic=True):
+        """Block-sparse attention over the lists.  With `dynamic` the call gets the workspace, whose first word the
+        tcgen05 kernel uses as the counter its streams draw their work items from; without, the items are dealt
+        statically (the results are the same bit for bit)."""
         rp, col = (self.row_ptr, self.col_idx) if self.block == 64 else (self.row_ptr64, self.col_idx64)
-        B.seer_sparse_attn(self.ctx, self.attn_shape, self.q, self.k, self.v, rp, col, self.o, self.lse, None, stream)
+        B.seer_sparse_attn(self.ctx, self.attn_shape, self.q, self.k, self.v, rp, col, self.o, self.lse,
+                           self.ws if dynamic else None, stream)
 
     def run(self, params: B.seer_mask_params, stream=None):
         self.gate(stream)

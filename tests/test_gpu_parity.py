@@ -263,6 +263,25 @@ def test_attention_flags_out_of_range_index_without_touching_it(rt, impl):
     check_attention(o, lse, o_ref, lse_ref, w)      # the bad entries were skipped
 
 
+def test_attention_work_counter_and_static_deal_agree_bit_for_bit(rt):
+    """The tcgen05 kernel's streams either draw their work items from a counter in the workspace or take a static
+    share; an item's result does not depend on which stream ran it or on what ran before it."""
+    import torch
+    B, Prefill, ctx = rt
+    w = W.make_workload("c4s")                            # several sequences, ragged tails, 40 / 8 heads
+    p = make_prefill(rt, w)
+    p.gate(); p.mask(B.make_mask_params(B.SEER_TOPK_RATIO, keep_num=1, keep_den=3, flags=3))
+    p.o.fill_(float("nan")); p.attn(dynamic=False); torch.cuda.synchronize()
+    assert p.status() == 0
+    o_static, lse_static = p.o.clone(), None if p.lse is None else p.lse.clone()
+    for _ in range(3):
+        p.o.fill_(float("nan")); p.attn(dynamic=True); torch.cuda.synchronize()
+        assert p.status() == 0
+        assert torch.equal(p.o, o_static)
+        if lse_static is not None:
+            assert torch.equal(p.lse, lse_static)
+
+
 @pytest.mark.parametrize("name", ["c2s", "c3s", "c4s", "c5s"])
 def test_attention_reduced_twins_gpu_pipeline(rt, name):
     """Whole GPU path (gate -> mask -> attention); the oracle attends over the GPU's own lists."""

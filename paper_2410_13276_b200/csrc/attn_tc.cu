@@ -64,7 +64,7 @@ constexpr uint32_t kOffGrp = kOffQfix + 2 * 2048;                 // per-group s
 constexpr uint32_t kGrpRcur = 0, kGrpAlpha = 256, kGrpLsum = 1024;   // lsum: 4 x 64 floats
 constexpr uint32_t kGrpBytes = 2048;
 constexpr uint32_t kOffBar = kOffGrp + 2 * kGrpBytes;             // mbarriers
-constexpr int kBarsPerStream = 16;
+constexpr int kBarsPerStream = 20;
 constexpr uint32_t kNumBars = 2 * kBarsPerStream;
 constexpr uint32_t kOffMisc = kOffBar + kNumBars * 8;             // tmem base, abort flag, the two streams' rings of work items (at +16, +32)
 constexpr uint32_t kOffTrace = kOffMisc + 64;                     // diagnostics: 6 roles x 48 tags x (sum, count)
@@ -72,7 +72,7 @@ constexpr uint32_t kSmemBytes = kOffTrace + 6 * 48 * 16 + 1024;   // + alignment
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 enum Bar { Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2, K_EMPTY = 3, V_FULL = 4, V_EMPTY = 5, S_FULL = 6 /* + buf */, P_FULL = 8,
-           PV_DONE = 9, FIXED = 10, ITEM_FULL = 12 /* + slot, 4 slots */ };
+           PV_DONE = 9, FIXED = 10, ITEM_FULL = 12 /* + slot, 4 slots */, ITEM_EMPTY = 16 /* + slot */ };
 constexpr int kItemRing = 4;
 
 constexpr uint32_t kTmemCols = 512;
@@ -218,7 +218,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(sh.bar(b + P_FULL), kBlockMax ? 4 : 1);       // one arrival, after the softmax group has met (block maxima: one per warp)
       mbar_init(sh.bar(b + PV_DONE), 1);
       mbar_init(sh.bar(b + FIXED), 1);
-      for (int i = 0; i < kItemRing; ++i) mbar_init(sh.bar(b + ITEM_FULL + i), 1);
+      for (int i = 0; i < kItemRing; ++i) {
+        mbar_init(sh.bar(b + ITEM_FULL + i), 1);
+        mbar_init(sh.bar(b + ITEM_EMPTY + i), 3);             // the V producer, the issuer and the softmax group have read the slot
+      }
     }
     st_shared_u32(sh.abort_flag(), 0u);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -246,9 +249,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int64_t w_step = 2 * (int64_t)gridDim.x;
   // Work items.  Without a counter a stream takes the items 2 * CTA + stream, + 2 * grid, ... (static deal).  With one
   // (`work_counter`, zero at launch) the stream's Q / K producer draws the next item number from it when it starts an
-  // item and passes it to the stream's other roles through a ring of four shared-memory words, one mbarrier each: the
-  // roles of a stream are never more than three items apart (Q is single-buffered), so a slot is not rewritten before
-  // its last reader has left it.  A negative number ends the stream.  Results do not depend on which stream runs an item.
+  // item and passes it to the stream's other roles through a ring of four shared-memory words, each with a full and an
+  // empty mbarrier: a slot is rewritten only when the V producer, the issuer and the softmax group have all read it
+  // (items with empty lists cost their roles nothing, so without the empty barrier the producer could lap the ring).
+  // A negative number ends the stream.  Results do not depend on which stream runs an item.
   const bool dyn = !kBlockMax && work_counter != nullptr;
   auto ring_addr = [&](int s, uint32_t n) -> uint32_t { return sh.base + kOffMisc + 16u + (uint32_t)s * 16u + (n & 3u) * 4u; };
   // consumer side: the n-th item of stream s (false: no more items, or a lost wait)
@@ -257,6 +261,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (!mbar_wait<kProducerSleepNs>(sh, s * kBarsPerStream + ITEM_FULL + (int)(n & 3u), (n >> 2) & 1u, status)) return false;
     w = (int64_t)(int32_t)ld_shared_u32(ring_addr(s, n));
     return w >= 0;
+  };
+  // a single-thread role has read slot n (the softmax group arrives once, after it has met)
+  auto release_item = [&](int s, uint32_t n) {
+    if (dyn) mbar_arrive(sh.bar(s * kBarsPerStream + ITEM_EMPTY + (int)(n & 3u)));
   };
 
   if (warp < 4 || warp >= 12) {
@@ -280,11 +288,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (dyn && !is_v) {
             w = drawn;
             const bool more = w < m.rows;
+            // the slot's previous content (item n - 4) has been read by everyone
+            if (!mbar_wait<kProducerSleepNs>(sh, bb + ITEM_EMPTY + (int)(n & 3u), ((n >> 2) & 1u) ^ 1u, status)) break;
             st_shared_u32(ring_addr(s, n), more ? (uint32_t)drawn : 0xffffffffu);
             mbar_arrive(sh.bar(bb + ITEM_FULL + (int)(n & 3u)));
             if (!more) break;
             drawn = atomicAdd(work_counter, 1);                        // the next one is on its way while this one is copied
-          } else if (!next_item(s, n, w)) break;
+          } else {
+            const bool more = next_item(s, n, w);
+            release_item(s, n);
+            if (!more) break;
+          }
           const Item it = decode_item<kChunk>(m, row_ptr, w);
           if (it.ntiles == 0) continue;
           if (!is_v) {
@@ -361,7 +375,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         };
         for (uint32_t n = 0; ok; ++n) {
           int64_t w;
-          if (!next_item(s, n, w)) break;
+          const bool more = next_item(s, n, w);
+          release_item(s, n);
+          if (!more) break;
           const Item it = decode_item<kChunk>(m, row_ptr, w);
           if (it.ntiles == 0) continue;
           tr.sample(cs);
@@ -527,7 +543,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       int64_t w;
       const bool more = next_item(s, n, w);
       // (with a counter the answer comes from a wait, which can be lost: the group leaves together or not at all)
-      if (dyn ? named_bar_or(bar_vote, kGroupThreads, !more) : !more) break;
+      const bool stop = dyn ? named_bar_or(bar_vote, kGroupThreads, !more) : !more;
+      if (gt == 0) release_item(s, n);                      // (every thread of the group has read the slot)
+      if (stop) break;
       const Item it = decode_item<kChunk>(m, row_ptr, w);
       const int64_t tok0 = (int64_t)it.s0 + (int64_t)it.i * kBlock + (kChunk ? it.dq : 0);   // first row of the item in q / o / lse
       if (it.ntiles == 0) {                                 // no visible key: o = 0, lse = -inf

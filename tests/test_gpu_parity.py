@@ -282,6 +282,34 @@ def test_attention_work_counter_and_static_deal_agree_bit_for_bit(rt):
             assert torch.equal(p.lse, lse_static)
 
 
+def test_attention_long_runs_of_empty_rows_with_the_work_counter(rt):
+    """Rows with empty lists cost the kernel's roles nothing, so the role that draws the work items could run far
+    ahead of the others: the ring that passes the item numbers on must not be lapped.  Only every 37th row has a list."""
+    import torch
+    B, Prefill, ctx = rt
+    w = W.make_small(seed=120, seqlens=[4096, 1000], hq=8, hkv=2)
+    p = make_prefill(rt, w, want_lse=True)
+    nbs = [int(n) for n in w.num_blocks]
+    counts, cols, r = [], [], 0
+    for nb in nbs:
+        for h in range(8):
+            for i in range(nb):
+                if r % 37 == 0:
+                    lst = sorted({0, i // 2, i})
+                else:
+                    lst = []
+                counts.append(len(lst)); cols.extend(lst); r += 1
+    rp = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    col = np.array(cols, np.int32)
+    p.set_lists(rp, col)
+    o_ref, lse_ref = O.sparse_attention(w.q, w.k, w.v, w.cu_seqlens, rp, col, 8, 2, 64, 1 / math.sqrt(128))
+    for dynamic in (False, True, True):
+        p.o.fill_(float("nan")); p.lse.fill_(float("nan"))
+        p.attn(dynamic=dynamic); torch.cuda.synchronize()
+        assert p.status() == 0
+        check_attention(p.o_host(), p.lse_host(), o_ref, lse_ref, w)
+
+
 @pytest.mark.parametrize("name", ["c2s", "c3s", "c4s", "c5s"])
 def test_attention_reduced_twins_gpu_pipeline(rt, name):
     """Whole GPU path (gate -> mask -> attention); the oracle attends over the GPU's own lists."""

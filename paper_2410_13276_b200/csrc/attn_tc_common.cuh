@@ -120,23 +120,6 @@ __device__ __forceinline__ void tc_wait_ld32(uint32_t (&r)[32]) {
                  "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
                :: "memory");
 }
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&r)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-               : "r"(taddr) : "memory");
-}
-// Waits for the loads of this thread; the loaded registers are in/out operands so that no use of them moves above it.
-__device__ __forceinline__ void tc_wait_ld8(uint32_t (&a)[8], uint32_t (&b)[8]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
-                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7])
-               :: "memory");
-}
-__device__ __forceinline__ void tc_wait_ld8(uint32_t (&a)[8]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7])
-               :: "memory");
-}
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
@@ -364,53 +347,6 @@ constexpr uint32_t make_idesc(bool a_mn_major, bool b_mn_major, uint32_t n = 64u
          ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// One pass over a 128 x 64 S^T tile for the key row of this thread: p = 2^(s * sl2 - mref[c]).
-//   SUBTRACT == false: adds p to l[c], packs p to bf16 pairs in pk, returns the OR of the packed words: bit 14 or 30
-//                      set means some p >= 2 (the references sit kRefShift above the column maxima, so that is a score
-//                      2^(kRefShift + 1) above its reference maximum, or an infinity / NaN).
-//   SUBTRACT == true : removes p from l[c] again (used before a rebase; pk is not touched).
-// MASKED applies the causal mask of a diagonal block / drops a dead row.
-template <bool MASKED, bool SUBTRACT, class TR = Tracer<false>>
-__device__ __forceinline__ uint32_t softmax_pass(uint32_t s_addr, uint32_t m_addr, float sl2, bool row_live,
-                                              bool diag, int key_local, float (&l)[64], uint32_t (&pk)[32], TR* tr = nullptr) {
-  uint32_t ored = 0u;
-  uint32_t sv[2][8], mv[2][8];
-  tc_ld8(s_addr, sv[0]);
-  tc_ld8(m_addr, mv[0]);
-#pragma unroll
-  for (int ch = 0; ch < 8; ++ch) {
-    tc_wait_ld8(sv[ch & 1], mv[ch & 1]);
-    if (tr) tr->ev(40 + (ch >> 1), 0);
-    if (ch < 7) {
-      tc_ld8(s_addr + (ch + 1) * 8, sv[(ch + 1) & 1]);
-      tc_ld8(m_addr + (ch + 1) * 8, mv[(ch + 1) & 1]);
-    }
-#pragma unroll
-    for (int e = 0; e < 8; e += 4) {
-      const int c = ch * 8 + e;
-      float x0 = fmaf(__uint_as_float(sv[ch & 1][e]), sl2, -__uint_as_float(mv[ch & 1][e]));
-      float x1 = fmaf(__uint_as_float(sv[ch & 1][e + 1]), sl2, -__uint_as_float(mv[ch & 1][e + 1]));
-      float x2 = fmaf(__uint_as_float(sv[ch & 1][e + 2]), sl2, -__uint_as_float(mv[ch & 1][e + 2]));
-      float x3 = fmaf(__uint_as_float(sv[ch & 1][e + 3]), sl2, -__uint_as_float(mv[ch & 1][e + 3]));
-      if (MASKED) {
-        if (!row_live || (diag && key_local > c)) x0 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 1)) x1 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 2)) x2 = -CUDART_INF_F;
-        if (!row_live || (diag && key_local > c + 3)) x3 = -CUDART_INF_F;
-      }
-      const float p0 = ex2f(x0), p1 = ex2f(x1), p2 = ex2f(x2), p3 = ex2f(x3);
-      if (SUBTRACT) {
-        l[c] -= p0; l[c + 1] -= p1; l[c + 2] -= p2; l[c + 3] -= p3;
-      } else {
-        l[c] += p0; l[c + 1] += p1; l[c + 2] += p2; l[c + 3] += p3;
-        pk[c >> 1] = pack_bf16(p0, p1);
-        pk[(c >> 1) + 1] = pack_bf16(p2, p3);
-        ored |= pk[c >> 1] | pk[(c >> 1) + 1];
-      }
-    }
-  }
-  return ored;
-}
 
 }  // namespace tcc
 }  // namespace seer

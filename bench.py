@@ -619,6 +619,10 @@ def main():
                "kept_blocks": nnz, "stage_ms": {"gate": gate_ms, "mask": mask_ms, "attn": attn_ms,
                                                 "attn_min": float(min(attn_all)), "attn_median": float(np.median(attn_all))},
                "attn_kernel": {0: "tcgen05", 1: "mma.sync", 2: "chosen by shape"}[args.attn_impl],
+               # the same attention time with a row's diagonal block counted as (B + 1) / 2B of a block (what a causal
+               # kernel needs of it): the figure FlashAttention-style FLOP counts give
+               "attn_tflops_diag_counted_half": (nnz - B.seer_mask_rows(p.shape) * (1.0 - 65.0 / 128.0)) * FLOP_PER_BLOCK
+                                                / (attn_ms * 1e-3) / 1e12,
                "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
                             "frac": achieved / burst, "peak_source": f"bf16 dense burst, of {src}",
                             "frac_of_sustained": (achieved / sustained) if sustained else None, "traffic": traffic,

@@ -453,7 +453,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     uint32_t cnt = 0;                                       // tiles this stream has processed
     bool ok = true;
     // diagnostics (traced build): clocks of every steady-state tile by segment, kept in registers
-    long long seg[15] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, seg_last = 0;
+    long long seg[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, seg_last = 0;
     unsigned seg_n = 0, nreb = 0;
 #define SEG(k) do { if constexpr (kTrace) { const long long now_ = clock64(); seg[k] += now_ - seg_last; seg_last = now_; } } while (0)
 
@@ -662,6 +662,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         s_seen = t + 1 < it.ntiles && mbar_test(sh.bar(bb + S_FULL + (int)(sbuf ^ 1u)), ((cnt + 1) >> 1) & 1u);
         fence_async_smem();
         tc_fence_before();
+        SEG(15);
         const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
         SEG(4);
         if (slow) {
@@ -837,7 +838,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       tr.ev(31, 0);
     }
     if constexpr (kTrace) if (tr.p != nullptr)
-      for (int k = 0; k < 15; ++k) { tr.acc[2 * (32 + k)] = (unsigned long long)seg[k]; tr.acc[2 * (32 + k) + 1] = k >= 8 ? nreb : seg_n; }
+      for (int k = 0; k < 16; ++k) { tr.acc[2 * (32 + k)] = (unsigned long long)seg[k]; tr.acc[2 * (32 + k) + 1] = (k >= 8 && k < 15) ? nreb : seg_n; }
     tr.flush();
 #undef SEG
   }

@@ -215,7 +215,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(sh.bar(b + V_EMPTY), 1);
       mbar_init(sh.bar(b + S_FULL), 1);
       mbar_init(sh.bar(b + S_FULL + 1), 1);
-      mbar_init(sh.bar(b + P_FULL), kBlockMax ? 4 : 1);       // one arrival, after the softmax group has met (block maxima: one per warp)
+      mbar_init(sh.bar(b + P_FULL), 4);                       // one arrival per warp of the softmax group
       mbar_init(sh.bar(b + PV_DONE), 1);
       mbar_init(sh.bar(b + FIXED), 1);
       for (int i = 0; i < kItemRing; ++i) {
@@ -660,9 +660,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         SEG(6);
         // the next tile's S^T: asked now, looked at when the next tile starts
         s_seen = t + 1 < it.ntiles && mbar_test(sh.bar(bb + S_FULL + (int)(sbuf ^ 1u)), ((cnt + 1) >> 1) & 1u);
-        fence_async_smem();
         tc_fence_before();
         SEG(15);
+        // the vote comes before the proxy fence: the stores drain (behind the MMAs' operand reads) while the group meets
         const bool slow = named_bar_or(bar_vote, kGroupThreads, fail || (over & 0x40004000u) != 0u);
         SEG(4);
         if (slow) {
@@ -774,8 +774,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           SEG(14);
         }
         SEG(5);
-        // every thread's stores are visible to the MMA: one arrival hands P^T over and the S^T buffer back
-        if (gt == 0) mbar_arrive(sh.bar(bb + P_FULL));
+        // a warp whose stores are visible to the MMA arrives; four arrivals hand P^T over and the S^T buffer back
+        if (!slow) fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sh.bar(bb + P_FULL));
         SEG(7);
       }
       if (!ok) break;

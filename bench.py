@@ -196,9 +196,9 @@ TIMELINE_TAGS = {1: "loop", 2: "wait for an empty K / V buffer", 10: "before S^T
                  13: "before P V", 14: "wait V_FULL", 15: "wait P_FULL", 16: "P V MMAs + commits",
                  29: "item start (decode, first list entries)", 30: "tile loop of an item (all tiles)", 31: "epilogue",
                  32: "wait S_FULL", 33: "softmax pass (incl. first-tile references)", 34: "next list entries",
-                 35: "wait PV_DONE", 36: "vote (the group's barrier)", 37: "(branch)", 38: "P^T stores", 39: "arrive P_FULL",
+                 35: "wait PV_DONE", 36: "vote (the group's barrier)", 37: "(branch)", 38: "P^T stores", 39: "proxy fence, arrive P_FULL",
                  40: "rebase: wait next S^T + vote", 41: "rebase: TMEM reads", 42: "rebase: column maxima (shuffles)",
-                 43: "rebase: new references", 44: "rebase: fix MMAs, rescale", 45: "rebase: wait FIXED", 46: "rebase: pass + stores", 47: "S_FULL test, proxy fence"}
+                 43: "rebase: new references", 44: "rebase: fix MMAs, rescale", 45: "rebase: wait FIXED", 46: "rebase: pass + stores", 47: "next S_FULL test (waits behind the P^T stores)"}
 TIMELINE_ROLES = ["producer K+Q, stream 0", "issuer, stream 0", "producer V, stream 0", "issuer, stream 1",
                   "softmax group, stream 0", "softmax group, stream 1"]
 

@@ -30,7 +30,7 @@ sys.path.insert(0, ROOT)
 
 FLOP_PER_BLOCK = 4 * 64 * 64 * 128
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch of the default command, and the capture it is from
-TRAFFIC_C3_KEEP10 = (6.66e9, "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch of this command "
+TRAFFIC_C3_KEEP10 = (4.64e9, "ncu dram__bytes_read.sum + dram__bytes_write.sum, one launch of this command "
                                  "(summary: profiles/attn_tc_kernel_c3_seq131072_keep10_dram.md)")
 METRIC = "sparse_prefill_attention_effective_tflops_128k_90pct_block_sparsity"
 
